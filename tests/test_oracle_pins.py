@@ -1,0 +1,251 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU.
+
+Each test is chosen so that a plausible mistake in the oracle (dropped term, wrong sign or index,
+transposed operand, off-by-one in the accept rule) fails at least one of them.
+"""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2311_08263_b200 import workload as wl
+
+
+def _tiny():
+    cfg = wl.CONFIGS["tiny"]
+    return cfg, wl.make_weights(cfg), wl.make_prompts(cfg)[0][0].numpy()
+
+
+# ---------------------------------------------------------------- decoder forward vs the library
+def _hf_model(cfg, w):
+    from transformers import LlamaConfig, LlamaForCausalLM
+    hc = LlamaConfig(hidden_size=cfg.d_model, intermediate_size=cfg.d_ffn,
+                     num_hidden_layers=cfg.n_layers, num_attention_heads=cfg.n_heads,
+                     num_key_value_heads=cfg.n_kv_heads, head_dim=cfg.head_dim, vocab_size=cfg.vocab,
+                     rms_norm_eps=cfg.rms_eps, rope_theta=cfg.rope_theta, attention_bias=False,
+                     mlp_bias=False, tie_word_embeddings=False, max_position_embeddings=1024,
+                     attn_implementation="eager")
+    m = LlamaForCausalLM(hc).double().eval()
+    sd = {"model.embed_tokens.weight": w["tok_emb"], "model.norm.weight": w["g_final"],
+          "lm_head.weight": w["lm_head"]}
+    names = {"wq": "self_attn.q_proj", "wk": "self_attn.k_proj", "wv": "self_attn.v_proj",
+             "wo": "self_attn.o_proj", "w_gate": "mlp.gate_proj", "w_up": "mlp.up_proj",
+             "w_down": "mlp.down_proj", "g_attn": "input_layernorm", "g_ffn": "post_attention_layernorm"}
+    for l in range(cfg.n_layers):
+        for k, v in names.items():
+            sd[f"model.layers.{l}.{v}.weight"] = w[k][l]
+    res = m.load_state_dict({k: v.double() for k, v in sd.items()}, strict=False)
+    assert not res.missing_keys and not res.unexpected_keys
+    return m
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (4, 2), (4, 1)])
+def test_forward_matches_huggingface_llama_fp64(hq, hkv):
+    """The paper runs stock HuggingFace Llama (Section 5.1); the oracle's forward must be that
+    model: same logits for a causal forward, with and without a K/V-cache split."""
+    cfg = wl.small_config(dtype="f32", n_heads=hq, n_kv_heads=hkv, head_dim=32, d_model=128,
+                          d_ffn=256, vocab=300, bias_beta=0.0, n_layers=3)
+    w = wl.make_weights(cfg)
+    toks = wl.make_prompts(cfg, lens=[29])[0][0]
+    with torch.no_grad():
+        ref = _hf_model(cfg, w)(toks.long()[None]).logits[0].numpy()
+    o = oracle.Oracle(cfg, w, 64)
+    _, lg = o.forward(toks.numpy())
+    assert np.abs(lg - ref).max() < 2e-6
+    # same rows through the cache: commit the first 17 tokens, then a 12-row window
+    o2 = oracle.Oracle(cfg, w, 64)
+    o2.prefill(toks[:18].numpy(), c=12)
+    assert o2.kv_len == 17
+    _, lg2 = o2.forward(toks[17:].numpy())
+    assert np.abs(lg2 - ref[17:]).max() < 2e-6
+
+
+def test_bias_lands_on_permuted_input_token():
+    cfg = wl.small_config(dtype="f32", d_model=64, n_heads=2, n_kv_heads=2, head_dim=32, d_ffn=128,
+                          vocab=50, bias_beta=0.0)
+    w = wl.make_weights(cfg)
+    toks = np.array([3, 9, 41], np.int32)
+    _, base = oracle.Oracle(cfg, w, 16).forward(toks)
+    cfg_b = wl.small_config(dtype="f32", d_model=64, n_heads=2, n_kv_heads=2, head_dim=32, d_ffn=128,
+                            vocab=50, bias_beta=2.5)
+    _, biased = oracle.Oracle(cfg_b, w, 16).forward(toks)
+    diff = biased - base
+    perm = w["bias_perm"].numpy()
+    for r, t in enumerate(toks):
+        expect = np.zeros(50, np.float32)
+        expect[perm[t]] = 2.5
+        assert np.allclose(diff[r], expect, atol=1e-6)
+    assert sorted(perm.tolist()) == list(range(50))
+
+
+def test_bf16_weights_are_upconverted_exactly():
+    cfg = wl.small_config(dtype="bf16", d_model=64, n_heads=2, n_kv_heads=1, head_dim=32, d_ffn=128, vocab=80)
+    w = wl.make_weights(cfg)
+    w32 = {k: ([t.float() for t in v] if isinstance(v, list) else (v.float() if v.dtype != torch.int32 else v))
+           for k, v in w.items()}
+    cfg32 = wl.small_config(dtype="f32", d_model=64, n_heads=2, n_kv_heads=1, head_dim=32, d_ffn=128, vocab=80)
+    toks = np.arange(10, dtype=np.int32)
+    _, a = oracle.Oracle(cfg, w, 16).forward(toks)
+    _, b = oracle.Oracle(cfg32, w32, 16).forward(toks)
+    assert np.array_equal(a, b)
+
+
+# ---------------------------------------------------------------- losslessness (Section 3.1 / 3.2)
+@pytest.mark.parametrize("c", [1, 2, 3, 8, 16])
+@pytest.mark.parametrize("refill", [0, 1])
+def test_committed_stream_equals_greedy_autoregressive(c, refill):
+    cfg, w, prompt = _tiny()
+    o = oracle.Oracle(cfg, w, 160)
+    ar, _ = o.ar_generate(prompt, 64)
+    o.prefill(prompt, c, refill=refill, pad_id=7)
+    toks, counts = o.generate(64)
+    assert np.array_equal(toks, ar)
+    assert counts.min() >= 1 and counts.max() <= c
+    assert counts.sum() == 64
+    if c == 1:
+        assert len(counts) == 64     # window of one row is plain autoregressive decoding
+
+
+def test_window_contents_never_change_the_stream():
+    cfg, w, prompt = _tiny()
+    o = oracle.Oracle(cfg, w, 160)
+    ar, _ = o.ar_generate(prompt, 40)
+    o.prefill(prompt, 8)
+    rng = np.random.default_rng(0)
+    out, pending = [], prompt[-1]
+    while len(out) < 40:
+        win = rng.integers(0, cfg.vocab, 8).astype(np.int32)
+        win[0] = pending
+        k, acc, wnew = o.jacobi_step(win)
+        out.extend(acc.tolist())
+        pending = wnew[0]
+    assert out[:40] == ar.tolist()
+
+
+# ---------------------------------------------------------------- accept rule: closed form given AR
+def _expected_step(ar, n, window, c, prompt, refill_fn):
+    """Closed form: k = 1 + longest m with window[1..m] == ar[n..n+m-1]; emitted = ar[n..n+k-1]."""
+    k = 1
+    while k < c and window[k] == ar[n + k - 1]:
+        k += 1
+    return k, ar[n:n + k]
+
+
+@pytest.mark.parametrize("c", [2, 5, 8])
+def test_directed_accept_counts(c):
+    """Prime the window with m correct continuation tokens followed by a wrong one: the step must
+    accept exactly m + 1 tokens, for every m, and the refreshed window must carry the pending
+    token, the unverified outputs, and refill ids for the k-1 unseen positions."""
+    cfg, w, prompt = _tiny()
+    P = len(prompt)
+    o = oracle.Oracle(cfg, w, 200)
+    ar, _ = o.ar_generate(prompt, 80)
+    for m in range(c):
+        o.prefill(prompt, c)
+        n = 0
+        # advance a few plain steps so n_gen is not zero
+        for _ in range(3):
+            k, acc, wnew = o.jacobi_step()
+            n += k
+        win = wnew.copy()
+        win[1:1 + m] = ar[n:n + m]
+        if 1 + m < c:
+            win[1 + m] = (ar[n + m] + 1) % cfg.vocab
+        k, acc, w2, lg = o.jacobi_step(win, want_logits=True)
+        assert k == m + 1
+        assert np.array_equal(acc, ar[n:n + k])
+        a = lg.argmax(axis=1)
+        assert w2[0] == ar[n + k - 1]
+        assert np.array_equal(w2[1:c - k + 1], a[k:c])
+        n2 = n + k
+        for j in range(c - k + 1, c):
+            assert w2[j] == prompt[(n2 + j - 1) % P]
+        assert o.n_gen == n2 and o.kv_len == P - 1 + n2
+
+
+@pytest.mark.parametrize("V,c", [(4, 2), (4, 3), (4, 4), (8, 3)])
+def test_brute_force_all_windows_tiny_vocab(V, c):
+    """Enumerate every window over a tiny vocabulary and check the accepted count and tokens
+    against greedy decoding done one token at a time."""
+    cfg = wl.small_config(dtype="f32", n_layers=1, d_model=16, n_heads=2, n_kv_heads=1, head_dim=8,
+                          d_ffn=32, vocab=V, bias_beta=0.0, seed=5 + V + c)
+    w = wl.make_weights(cfg)
+    # larger weights so logits are well separated
+    for key in ("tok_emb", "lm_head"):
+        w[key] = w[key] * 40
+    prompt = np.array([1, 3 % V, 2, 0, 1], np.int32)
+    o = oracle.Oracle(cfg, w, 64)
+    ar, mar = o.ar_generate(prompt, c + 1)
+    assert mar.min() > 1e-4
+    seen_k = set()
+    for guess in itertools.product(range(V), repeat=c - 1):
+        o.prefill(prompt, c)
+        win = np.array((prompt[-1],) + guess, np.int32)
+        k, acc, w2 = o.jacobi_step(win)
+        kk, emitted = _expected_step(ar, 0, win, c, prompt, None)
+        assert k == kk and np.array_equal(acc, emitted)
+        assert w2[0] == ar[k - 1]
+        seen_k.add(k)
+    assert seen_k == set(range(1, c + 1))
+
+
+# ---------------------------------------------------------------- whole-stream closed forms
+def test_zero_matrices_stream_is_iterated_permutation():
+    cfg = wl.small_config(dtype="f32", d_model=32, n_heads=2, n_kv_heads=2, head_dim=16, d_ffn=64,
+                          vocab=97, bias_beta=4.0)
+    w = wl.make_weights(cfg, zero_matrices=True)
+    prompt = np.array([5, 11, 60], np.int32)
+    perm = w["bias_perm"].numpy()
+    o = oracle.Oracle(cfg, w, 128)
+    o.prefill(prompt, 6)
+    toks, counts = o.generate(50)
+    expect, t = [], prompt[-1]
+    for _ in range(50):
+        t = perm[t]
+        expect.append(t)
+    assert toks.tolist() == expect
+    # guesses that already follow the permutation are all accepted: k = c
+    o.prefill(prompt, 6)
+    win = np.array([prompt[-1]] + expect[:5], np.int32)
+    k, acc, _ = o.jacobi_step(win)
+    assert k == 6 and acc.tolist() == expect[:6]
+
+
+def test_all_equal_logits_pick_lowest_id():
+    cfg = wl.small_config(dtype="f32", d_model=32, n_heads=2, n_kv_heads=2, head_dim=16, d_ffn=64,
+                          vocab=33, bias_beta=0.0)
+    w = wl.make_weights(cfg, zero_matrices=True)
+    o = oracle.Oracle(cfg, w, 64)
+    o.prefill(np.array([4, 2], np.int32), 4)
+    toks, _ = o.generate(10)
+    assert toks.tolist() == [0] * 10
+
+
+# ---------------------------------------------------------------- stop rules
+def test_max_tokens_and_eos_truncation():
+    cfg, w, prompt = _tiny()
+    o = oracle.Oracle(cfg, w, 160)
+    ar, _ = o.ar_generate(prompt, 30)
+    eos = int(ar[12])
+    first = int(np.where(ar == eos)[0][0])
+    o.prefill(prompt, 8)
+    toks, counts = o.generate(30, eos_id=eos)
+    assert toks.tolist() == ar[:first + 1].tolist()
+    assert counts.sum() == first + 1
+    o.prefill(prompt, 8)
+    toks, counts = o.generate(5)
+    assert toks.tolist() == ar[:5].tolist()
+
+
+# ---------------------------------------------------------------- stored stream (drift guard)
+def test_golden_tiny_stream():
+    """tests/golden/tiny_ar_stream.txt is written by tests/golden/make_golden.py from the oracle
+    alone; it guards the oracle and the input generator against silent drift."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "tiny_ar_stream.txt")
+    want = [int(t) for t in open(path).read().split("\n")[-2].split()]
+    cfg, w, prompt = _tiny()
+    ar, _ = oracle.Oracle(cfg, w, 160).ar_generate(prompt, 64)
+    assert ar.tolist() == want
