@@ -1,0 +1,153 @@
+/*
+ * fastcot.h - C ABI of the Jacobi-window decode step (FastCoT, arXiv 2311.08263) for NVIDIA B200.
+ *
+ * One step = one causal decoder forward over (committed prefix held in a K/V cache) + (a window
+ * of c tokens: the pending exact token followed by c-1 approximate tokens), greedy argmax at
+ * every window row, verification of the previous guesses one by one, K/V commit of the accepted
+ * rows and shift + refill of the window (paper Section 3.3: Eq. 4 inference, Eq. 5 verification,
+ * "Cache Update"; buffer and index vector: Section 3.2).  With c = 1 the step is plain greedy
+ * autoregressive decoding (Eq. 1).
+ *
+ * Conventions
+ *   - "host"/"device" on every pointer says where the memory lives.  The library allocates NO
+ *     device memory: weights, K/V slab and workspace are caller-owned device buffers, BORROWED for
+ *     the lifetime of the context.  fc_destroy frees host state only.
+ *   - All matrices are row-major [out_features, in_features] in the model dtype.
+ *   - Every call returns FC_OK (0) or a negative fc_status; nothing aborts or throws, no device
+ *     trap is used, and a failed call leaves the committed state (tokens, kv_len) unchanged.
+ *   - Calls are synchronous with respect to their host outputs: they wait on the context's stream.
+ *   - A context is bound to one device and one stream and is not re-entrant.
+ */
+#ifndef FASTCOT_H_
+#define FASTCOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fc_ctx fc_ctx;
+
+typedef enum { FC_F32 = 0, FC_BF16 = 1 } fc_dtype;
+
+/* How window slots that no forward has predicted yet are filled (Section 3.2: the buffer is
+ * initialised from the prompt's own token ids; a pad token is the alternative it mentions). */
+typedef enum { FC_REFILL_PROMPT_CYCLE = 0, FC_REFILL_PAD = 1 } fc_refill;
+
+typedef enum {
+  FC_OK = 0,
+  FC_ERR_ARG = -1,            /* NULL pointer, non-positive size, bad enum */
+  FC_ERR_SHAPE = -2,          /* model shape the kernels cannot run (see fc_init) */
+  FC_ERR_CAPACITY = -3,       /* kv_len + c > max_seq, batch > max_batch, c > max_c, buffer too small */
+  FC_ERR_TOKEN_RANGE = -4,    /* token id outside [0, vocab) */
+  FC_ERR_STATE = -5,          /* step/generate before prefill */
+  FC_ERR_BAD_WINDOW = -6,     /* window_in[b][0] is not the pending exact token */
+  FC_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired; context must be re-prefilled */
+  FC_ERR_CUDA = -8            /* a CUDA runtime/driver call failed; see fc_last_cuda_error */
+} fc_status;
+
+enum {                        /* fc_model_shape.flags */
+  FC_FLAG_SIMT_GEMM = 1,      /* run projections on the plain FMA kernels even for bf16 (debug aid) */
+  FC_FLAG_NO_GRAPH = 2        /* never capture the step into a CUDA graph */
+};
+
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t dtype;              /* fc_dtype of the weights and of the K/V cache */
+  float rms_eps, rope_theta;  /* RMSNorm epsilon; rotary base (half-split pairing i <-> i+head_dim/2) */
+  int32_t max_batch, max_c;   /* capacity: sequences per step, window rows per sequence */
+  int32_t max_seq;            /* K/V capacity per sequence: committed tokens + window rows */
+  float bias_beta;            /* synthetic-workload logit bonus on token bias_perm[input]; 0 disables */
+  int32_t flags;
+} fc_model_shape;
+
+typedef struct {              /* DEVICE pointers, borrowed */
+  const void *tok_emb;                                   /* [vocab, d_model] */
+  const void *const *wq, *const *wk, *const *wv, *const *wo;   /* HOST arrays of n_layers device ptrs */
+  const void *const *w_gate, *const *w_up, *const *w_down;
+  const void *const *g_attn, *const *g_ffn;              /* RMSNorm gains [d_model] */
+  const void *g_final, *lm_head;                         /* [d_model], [vocab, d_model] */
+  const int32_t *bias_perm;                              /* device [vocab] or NULL */
+} fc_weights;
+
+typedef struct {              /* filled by fc_generate */
+  int64_t steps, tokens;      /* forwards run; tokens committed over all sequences */
+  int32_t accept_hist[65];    /* accept_hist[k] = (sequence, step) pairs that accepted k tokens; k>64 -> [64] */
+  float ms_prefill, ms_steps; /* device time; ms_prefill is 0 unless prefill ran inside the call */
+} fc_stats;
+
+/* Bytes the caller must provide.  K/V slab layout: [layer][K|V][max_batch][n_kv_heads][max_seq][head_dim]
+ * in the model dtype.  Both return 0 for an invalid shape. */
+size_t fc_kv_bytes(const fc_model_shape *shape);
+size_t fc_workspace_bytes(const fc_model_shape *shape);
+
+/* Create a context.  shape, weights: host structs (copied).  kv, ws: device, >= the sizes above,
+ * 256-byte aligned.  cuda_stream: a cudaStream_t (NULL = default stream).  Shape limits:
+ * head_dim in {32, 64, 128}; n_heads % n_kv_heads == 0; d_model, d_ffn, n_heads*head_dim multiples of 8;
+ * max_c <= 64.  The bf16 tensor-core path needs an sm_100a device; FC_F32 runs on FMA kernels. */
+int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weights *weights,
+            void *kv, size_t kv_bytes, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Start `batch` sequences.  prompt_ids: host [batch, p_stride]; prompt_lens: host [batch], each >= 1.
+ * Caches K/V of prompt[0 .. P-2]; prompt[P-1] becomes the pending exact token (window slot 0);
+ * slots 1..c-1 are filled by the refill rule.  Section 3.1 (prompt + window form the first input). */
+int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids, int32_t p_stride,
+               const int32_t *prompt_lens, int32_t c, int32_t refill, int32_t pad_id);
+
+/* One Jacobi-window iteration for every live sequence (Eq. 4, Eq. 5, cache update).
+ * window_in: host [batch, c] or NULL (keep the internal window); slot 0 of each row must be the
+ * pending exact token.  Outputs (host, each nullable): accepted_count [batch] (k in [1, c]; 0 for a
+ * finished sequence), accepted_tokens [batch, c] (first k valid), window_out [batch, c]. */
+int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *accepted_count,
+                   int32_t *accepted_tokens, int32_t *window_out);
+
+/* Iterate until every sequence has committed max_tokens tokens or eos_id (eos_id < 0: never).
+ * Streams are cut at max_tokens and just after the first EOS (Section 3.4, condition 2).
+ * out_tokens: host [batch, max_tokens]; out_lens: host [batch]; stats nullable. */
+int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t eos_id, int32_t *out_tokens,
+                int32_t *out_lens, fc_stats *stats);
+
+/* Benchmark/debug aids.  fc_debug_set_state: declare `batch` sequences with kv_lens[b] tokens
+ * already present in the K/V slab (written by the caller) and pending tokens pending[b]; windows are
+ * refilled with pad_id.  fc_debug_logits: device buffer [max_batch*max_c, vocab] fp32 that receives
+ * the logits of every following step (NULL turns it off).  fc_get_state: host copies of kv_len and
+ * n_gen per sequence (each nullable). */
+int fc_debug_set_state(fc_ctx *ctx, int32_t batch, const int32_t *kv_lens, const int32_t *pending,
+                       int32_t c, int32_t pad_id);
+int fc_debug_logits(fc_ctx *ctx, float *dev_logits);
+int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen);
+
+/* Enqueue `n_steps` iterations back to back without host round trips and without committing
+ * (kv_len is restored before each step), returning the device time in milliseconds between the
+ * first and the last kernel.  For latency measurement at a fixed K/V length. */
+int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, float *ms_total);
+
+/* Number of kernels the most recent step / prefill / bench call launched. */
+int64_t fc_last_launch_count(const fc_ctx *ctx);
+
+void fc_destroy(fc_ctx *ctx);
+const char *fc_strerror(int status);
+const char *fc_last_cuda_error(const fc_ctx *ctx);   /* text of the last CUDA failure, or "" */
+
+/* ---- single operations of the step, for unit parity tests (all pointers DEVICE unless noted) ---- */
+
+/* y[R, N] += x[R, K] . w[N, K]^T with fp32 x and y and weights in `dtype`; K % 8 == 0.
+ * use_tensor_cores != 0 selects the tcgen05 kernel (bf16 only).  The projections of the step
+ * (QKV, O, gate/up, down) are this contraction. */
+int fc_op_linear(const float *x, const void *w, float *y, int32_t R, int32_t N, int32_t K,
+                 int32_t dtype, int32_t use_tensor_cores, void *cuda_stream);
+
+/* Verification + cache update on given argmax results (Eq. 5).  All arrays device int32:
+ * window [batch, c] (in/out), argmax [batch, c], kv_len/n_gen [batch] (in/out),
+ * accepted_count [batch], accepted_tokens [batch, c]; prompt [batch, p_stride], prompt_lens [batch]. */
+int fc_op_accept(int32_t *window, const int32_t *argmax, int32_t *kv_len, int32_t *n_gen,
+                 int32_t *accepted_count, int32_t *accepted_tokens, const int32_t *prompt,
+                 const int32_t *prompt_lens, int32_t batch, int32_t c, int32_t p_stride,
+                 int32_t refill, int32_t pad_id, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* FASTCOT_H_ */

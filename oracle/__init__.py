@@ -58,6 +58,9 @@ def _load():
         lib.orc_generate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.orc_ar_generate.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                         C.c_void_p, C.c_void_p]
+        lib.orc_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int,
+                                   C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.orc_linear_add.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -72,6 +75,27 @@ def _host(t: torch.Tensor) -> torch.Tensor:
 
 def _i32(a) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def accept(window, argmax, n_gen: int, prompt, refill: int = 0, pad_id: int = 0):
+    """Verification + buffer update on plain arrays.  Returns (k, accepted[k], new_window[c])."""
+    w, a, p = _i32(window), _i32(argmax), _i32(prompt)
+    c = w.shape[0]
+    k = C.c_int32(0)
+    acc, w2 = np.empty(c, np.int32), np.empty(c, np.int32)
+    _load().orc_accept(w.ctypes.data, a.ctypes.data, c, n_gen, p.ctypes.data, p.shape[0], refill, pad_id,
+                       C.addressof(k), acc.ctypes.data, w2.ctypes.data)
+    return int(k.value), acc[:k.value].copy(), w2
+
+
+def linear_add(w: torch.Tensor, x: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """y + x . w^T with the oracle's fp32 dot product; w fp32 or bf16 [N, K], x [R, K], y [R, N]."""
+    wh = _host(w)
+    x = np.ascontiguousarray(x, np.float32)
+    out = np.ascontiguousarray(y, np.float32).copy()
+    _load().orc_linear_add(wh.data_ptr(), 0 if wh.dtype == torch.float32 else 1, wh.shape[0], wh.shape[1],
+                           x.ctypes.data, x.shape[0], out.ctypes.data)
+    return out
 
 
 class Oracle:

@@ -305,6 +305,35 @@ int orc_prefill(orc *o, const int32_t *prompt, int P, int c, int refill, int pad
   return 0;
 }
 
+/* Verification (Eq. 5) and buffer update (Section 3.3 "Cache Update") on plain arrays.
+ * w[0..c-1]: the window that was fed (w[0] exact); a[j]: greedy token following window slot j;
+ * n_gen: tokens generated before this step.  a[0] is always exact; a[j] is exact as long as every
+ * guess w[1..j] equalled the exact token before it: check one by one.  Outputs: *k in [1, c],
+ * accepted[0..k-1], and the new window: pending exact token a[k-1], then the still-unverified
+ * outputs a[k..c-1] as the next guesses, then fresh guesses for the k-1 positions that no forward
+ * has predicted yet (refill 0: prompt ids cycled by generated index; 1: pad_id). */
+void orc_accept(const int32_t *w, const int32_t *a, int c, int n_gen, const int32_t *prompt, int P,
+                int refill, int pad_id, int32_t *k_out, int32_t *accepted, int32_t *w_new) {
+  int k = 1;
+  while (k < c && w[k] == a[k - 1]) ++k;
+  for (int j = 0; j < k; ++j) accepted[j] = a[j];
+  *k_out = k;
+  const int n1 = n_gen + k;
+  w_new[0] = a[k - 1];
+  for (int j = 1; j < c; ++j) {
+    if (j <= c - k) w_new[j] = a[k - 1 + j];
+    else w_new[j] = refill == 1 ? pad_id : prompt[(n1 + j - 1) % P];
+  }
+}
+
+/* y[r, o] += dot(W[o, :], x[r, :]): the projection every GEMM of the step computes. */
+void orc_linear_add(const void *w, int wdtype, int out_f, int in_f, const float *x, int rows, float *y) {
+  float *t = malloc(sizeof(float) * (size_t)rows * out_f);
+  linear(w, wdtype, out_f, in_f, x, rows, t);
+  for (size_t i = 0; i < (size_t)rows * out_f; ++i) y[i] += t[i];
+  free(t);
+}
+
 /* One iteration (Eq. 4, Eq. 5, cache update).  window_in (or NULL = keep the internal window)
  * must carry the pending exact token in slot 0; slots 1.. are free guesses.
  * Outputs: *accepted = k in [1, c]; accepted_tokens[0..k-1]; window_out[0..c-1] (the refreshed
@@ -320,20 +349,13 @@ int orc_jacobi_step(orc *o, const int32_t *window_in, int32_t *accepted, int32_t
   int32_t *a = malloc(sizeof(int32_t) * c);
   int rc = orc_forward(o, o->window, c, logits_out, a);
   if (rc) { free(a); return rc; }
-  /* a[j] is the greedy token following window slot j.  a[0] is always exact; a[j] is exact as
-   * long as every guess w[1..j] equalled the exact token before it: check one by one. */
-  int k = 1;
-  while (k < c && o->window[k] == a[k - 1]) ++k;
-  for (int j = 0; j < k; ++j) accepted_tokens[j] = a[j];
+  int32_t *w2 = malloc(sizeof(int32_t) * c);
+  int32_t k;
+  orc_accept(o->window, a, c, o->n_gen, o->prompt, o->prompt_len, o->refill, o->pad_id, &k,
+             accepted_tokens, w2);
   *accepted = k;
   o->kv_len += k;                 /* K/V of rows 0..k-1 are already in place */
   o->n_gen += k;
-  /* new window: pending exact token a[k-1], then the still-unverified outputs a[k..c-1] as the
-   * next guesses, then fresh guesses for the k-1 positions no forward has predicted yet. */
-  int32_t *w2 = malloc(sizeof(int32_t) * c);
-  w2[0] = a[k - 1];
-  for (int j = 1; j < c; ++j)
-    w2[j] = (j <= c - k) ? a[k - 1 + j] : refill_token(o, o->n_gen + j - 1);
   memcpy(o->window, w2, sizeof(int32_t) * c);
   if (window_out) memcpy(window_out, w2, sizeof(int32_t) * c);
   free(a); free(w2);

@@ -1,0 +1,637 @@
+// C ABI of the Jacobi-window decode library: context, workspace carving, the per-step kernel chain.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "fc_internal.h"
+
+using namespace fc;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Carver {          // hands out aligned slices of the caller's workspace (or just counts bytes)
+  char *base; size_t off;
+  template <typename T> T *take(size_t n) {
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off = align_up(off + n * sizeof(T));
+    return p;
+  }
+};
+
+struct Buffers {
+  float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *part_o, *part_ml;
+  void *qb;
+  unsigned int *counters, *err;
+  unsigned long long *amax;
+  int32_t *window, *kv_len, *n_gen, *done, *acc_count, *acc_tokens, *prompt, *prompt_lens, *out_tokens;
+};
+
+struct Dims {
+  int rmax, qd, kvd, ldq, nsplit_max, tk;
+  size_t esz;
+};
+
+bool shape_ok(const fc_model_shape *s) {
+  if (!s) return false;
+  if (s->n_layers < 1 || s->d_model < 8 || s->n_heads < 1 || s->n_kv_heads < 1 || s->d_ffn < 8 || s->vocab < 1) return false;
+  if (s->dtype != FC_F32 && s->dtype != FC_BF16) return false;
+  if (s->head_dim != 32 && s->head_dim != 64 && s->head_dim != 128) return false;
+  if (s->n_heads % s->n_kv_heads) return false;
+  if (s->d_model % 8 || s->d_ffn % 8) return false;
+  if (s->max_batch < 1 || s->max_c < 1 || s->max_c > 64 || s->max_seq < s->max_c + 1) return false;
+  return true;
+}
+
+Dims dims_of(const fc_model_shape *s) {
+  Dims d;
+  d.rmax = s->max_batch * s->max_c;
+  d.qd = s->n_heads * s->head_dim;
+  d.kvd = s->n_kv_heads * s->head_dim;
+  d.ldq = d.qd + 2 * d.kvd;
+  d.tk = attn_tile_keys(s->dtype, s->head_dim);
+  d.nsplit_max = (s->max_seq + d.tk - 1) / d.tk;
+  d.esz = s->dtype == FC_F32 ? 4 : 2;
+  return d;
+}
+
+size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
+  Dims d = dims_of(s);
+  Carver c{base, 0};
+  Buffers t;
+  const size_t R = d.rmax;
+  t.x = c.take<float>(R * s->d_model);
+  t.qkv = c.take<float>(R * d.ldq);
+  t.qb = c.take<char>(R * d.qd * d.esz);
+  t.attn = c.take<float>(R * d.qd);
+  t.gu = c.take<float>(R * 2 * (size_t)s->d_ffn);
+  t.ss_attn = c.take<float>(R);
+  t.ss_ffn = c.take<float>(R);
+  t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
+  t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
+  t.counters = c.take<unsigned int>((size_t)s->max_batch * s->n_kv_heads);
+  t.err = c.take<unsigned int>(1);
+  t.amax = c.take<unsigned long long>(R);
+  t.window = c.take<int32_t>(R);
+  t.kv_len = c.take<int32_t>(s->max_batch);
+  t.n_gen = c.take<int32_t>(s->max_batch);
+  t.done = c.take<int32_t>(s->max_batch);
+  t.acc_count = c.take<int32_t>(s->max_batch);
+  t.acc_tokens = c.take<int32_t>(R);
+  t.prompt = c.take<int32_t>((size_t)s->max_batch * s->max_seq);
+  t.prompt_lens = c.take<int32_t>(s->max_batch);
+  t.out_tokens = c.take<int32_t>((size_t)s->max_batch * s->max_seq);
+  if (b) *b = t;
+  return c.off;
+}
+
+__global__ void bump_kernel(int32_t *v, int n) { if (threadIdx.x == 0 && blockIdx.x == 0) *v += n; }
+
+}  // namespace
+
+struct fc_ctx {
+  fc_model_shape s;
+  Dims d;
+  Buffers b;
+  // weights (host copies of the pointer tables)
+  const void *tok_emb, *g_final, *lm_head;
+  const int32_t *bias_perm;
+  std::vector<const void *> wq, wk, wv, wo, w_gate, w_up, w_down, g_attn, g_ffn;
+  char *kv; size_t kv_layer_stride, kv_half_stride;   // bytes
+  cudaStream_t st;
+  bool use_umma;
+  int n_sms;
+  std::vector<UmmaPlan *> plan_qkv, plan_o, plan_gu, plan_down;
+  UmmaPlan *plan_head = nullptr;
+  float *dbg_logits = nullptr;
+  // sequence state mirrored on the host
+  int batch = 0, c = 0, refill = 0, pad_id = 0, p_stride = 0;
+  bool ready = false;
+  std::vector<int32_t> kv_len_h, n_gen_h, pending_h, done_h;
+  int gen_max_tokens = 0, gen_eos = -1;
+  // pinned staging: [count | tokens | window | err]
+  int32_t *pin = nullptr;
+  int64_t launches = 0;
+  char cuda_err[256] = {0};
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+};
+
+#define FC_CK(call)                                                                      \
+  do {                                                                                   \
+    cudaError_t e_ = (call);                                                             \
+    if (e_ != cudaSuccess) {                                                             \
+      snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "%s: %s", #call, cudaGetErrorString(e_)); \
+      return FC_ERR_CUDA;                                                                \
+    }                                                                                    \
+  } while (0)
+
+extern "C" size_t fc_kv_bytes(const fc_model_shape *s) {
+  if (!shape_ok(s)) return 0;
+  Dims d = dims_of(s);
+  return (size_t)s->n_layers * 2 * s->max_batch * s->n_kv_heads * (size_t)s->max_seq * s->head_dim * d.esz;
+}
+
+extern "C" size_t fc_workspace_bytes(const fc_model_shape *s) {
+  if (!shape_ok(s)) return 0;
+  return carve(s, nullptr, nullptr);
+}
+
+extern "C" const char *fc_strerror(int st) {
+  switch (st) {
+    case FC_OK: return "ok";
+    case FC_ERR_ARG: return "bad argument";
+    case FC_ERR_SHAPE: return "unsupported model shape";
+    case FC_ERR_CAPACITY: return "capacity exceeded";
+    case FC_ERR_TOKEN_RANGE: return "token id out of range";
+    case FC_ERR_STATE: return "no prefilled sequences";
+    case FC_ERR_BAD_WINDOW: return "window slot 0 is not the pending exact token";
+    case FC_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case FC_ERR_CUDA: return "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+extern "C" const char *fc_last_cuda_error(const fc_ctx *ctx) { return ctx ? ctx->cuda_err : ""; }
+extern "C" int64_t fc_last_launch_count(const fc_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+static void destroy_plans(fc_ctx *ctx) {
+  for (auto *v : {&ctx->plan_qkv, &ctx->plan_o, &ctx->plan_gu, &ctx->plan_down}) {
+    for (UmmaPlan *p : *v) umma_plan_destroy(p);
+    v->clear();
+  }
+  umma_plan_destroy(ctx->plan_head);
+  ctx->plan_head = nullptr;
+}
+
+extern "C" void fc_destroy(fc_ctx *ctx) {
+  if (!ctx) return;
+  destroy_plans(ctx);
+  if (ctx->pin) cudaFreeHost(ctx->pin);
+  if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+  if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+  delete ctx;
+}
+
+// GEMM argument templates for layer l (buffers filled in; R set per forward)
+static GemmArgs args_qkv(const fc_ctx *c, int l) {
+  GemmArgs a; memset(&a, 0, sizeof(a));
+  a.x = c->b.x; a.ldx = c->s.d_model; a.gain = c->g_attn[l]; a.ss_out = c->b.ss_attn;
+  a.eps = c->s.rms_eps; a.dn = c->s.d_model;
+  a.w[0] = c->wq[l]; a.w[1] = c->wk[l]; a.w[2] = c->wv[l];
+  a.n_rows[0] = c->d.qd; a.n_rows[1] = c->d.kvd; a.n_rows[2] = c->d.kvd;
+  a.y_off[0] = 0; a.y_off[1] = c->d.qd; a.y_off[2] = c->d.qd + c->d.kvd;
+  a.n_mats = 3; a.y = c->b.qkv; a.ldy = c->d.ldq; a.K = c->s.d_model;
+  return a;
+}
+static GemmArgs args_o(const fc_ctx *c, int l) {
+  GemmArgs a; memset(&a, 0, sizeof(a));
+  a.x = c->b.attn; a.ldx = c->d.qd; a.eps = c->s.rms_eps; a.dn = c->s.d_model;
+  a.w[0] = c->wo[l]; a.n_rows[0] = c->s.d_model; a.n_mats = 1;
+  a.y = c->b.x; a.ldy = c->s.d_model; a.K = c->d.qd;
+  return a;
+}
+static GemmArgs args_gu(const fc_ctx *c, int l) {
+  GemmArgs a; memset(&a, 0, sizeof(a));
+  a.x = c->b.x; a.ldx = c->s.d_model; a.gain = c->g_ffn[l]; a.ss_out = c->b.ss_ffn;
+  a.eps = c->s.rms_eps; a.dn = c->s.d_model;
+  a.w[0] = c->w_gate[l]; a.w[1] = c->w_up[l];
+  a.n_rows[0] = c->s.d_ffn; a.n_rows[1] = c->s.d_ffn; a.y_off[0] = 0; a.y_off[1] = c->s.d_ffn;
+  a.n_mats = 2; a.y = c->b.gu; a.ldy = 2 * c->s.d_ffn; a.K = c->s.d_model;
+  return a;
+}
+static GemmArgs args_down(const fc_ctx *c, int l) {
+  GemmArgs a; memset(&a, 0, sizeof(a));
+  a.x = c->b.gu; a.x2 = c->b.gu + c->s.d_ffn; a.ldx = 2 * c->s.d_ffn; a.ss_in = c->b.ss_ffn;
+  a.eps = c->s.rms_eps; a.dn = c->s.d_model;
+  a.w[0] = c->w_down[l]; a.n_rows[0] = c->s.d_model; a.n_mats = 1;
+  a.y = c->b.x; a.ldy = c->s.d_model; a.K = c->s.d_ffn;
+  return a;
+}
+static GemmArgs args_head(const fc_ctx *c) {
+  GemmArgs a; memset(&a, 0, sizeof(a));
+  a.x = c->b.x; a.ldx = c->s.d_model; a.gain = c->g_final; a.eps = c->s.rms_eps; a.dn = c->s.d_model;
+  a.w[0] = c->lm_head; a.n_rows[0] = c->s.vocab; a.n_mats = 1; a.K = c->s.d_model;
+  a.tokens = c->b.window; a.perm = c->s.bias_beta != 0.f ? c->bias_perm : nullptr; a.beta = c->s.bias_beta;
+  a.amax = c->b.amax; a.logits = c->dbg_logits; a.vocab = c->s.vocab; a.ldy = c->s.vocab;
+  return a;
+}
+
+extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weights *w, void *kv, size_t kv_bytes,
+                       void *ws, size_t ws_bytes, void *cuda_stream) {
+  if (!out || !shape || !w || !kv || !ws) return FC_ERR_ARG;
+  *out = nullptr;
+  if (!shape_ok(shape)) return FC_ERR_SHAPE;
+  if (kv_bytes < fc_kv_bytes(shape) || ws_bytes < fc_workspace_bytes(shape)) return FC_ERR_CAPACITY;
+  if (((uintptr_t)kv | (uintptr_t)ws) % kAlign) return FC_ERR_ARG;
+  if (!w->tok_emb || !w->g_final || !w->lm_head || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate ||
+      !w->w_up || !w->w_down || !w->g_attn || !w->g_ffn) return FC_ERR_ARG;
+  fc_ctx *ctx = new (std::nothrow) fc_ctx();
+  if (!ctx) return FC_ERR_ARG;
+  ctx->s = *shape;
+  ctx->d = dims_of(shape);
+  carve(shape, (char *)ws, &ctx->b);
+  ctx->tok_emb = w->tok_emb; ctx->g_final = w->g_final; ctx->lm_head = w->lm_head; ctx->bias_perm = w->bias_perm;
+  const int L = shape->n_layers;
+  auto copy = [&](std::vector<const void *> &dst, const void *const *src) { dst.assign(src, src + L); };
+  copy(ctx->wq, w->wq); copy(ctx->wk, w->wk); copy(ctx->wv, w->wv); copy(ctx->wo, w->wo);
+  copy(ctx->w_gate, w->w_gate); copy(ctx->w_up, w->w_up); copy(ctx->w_down, w->w_down);
+  copy(ctx->g_attn, w->g_attn); copy(ctx->g_ffn, w->g_ffn);
+  for (int l = 0; l < L; ++l)
+    if (!ctx->wq[l] || !ctx->wk[l] || !ctx->wv[l] || !ctx->wo[l] || !ctx->w_gate[l] || !ctx->w_up[l] ||
+        !ctx->w_down[l] || !ctx->g_attn[l] || !ctx->g_ffn[l]) { delete ctx; return FC_ERR_ARG; }
+  ctx->kv = (char *)kv;
+  ctx->kv_half_stride = (size_t)shape->max_batch * shape->n_kv_heads * shape->max_seq * shape->head_dim * ctx->d.esz;
+  ctx->kv_layer_stride = 2 * ctx->kv_half_stride;
+  ctx->st = (cudaStream_t)cuda_stream;
+  ctx->use_umma = shape->dtype == FC_BF16 && !(shape->flags & FC_FLAG_SIMT_GEMM);
+
+  int rc = FC_OK;
+  auto fail = [&](int code) { fc_destroy(ctx); return code; };
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return fail(FC_ERR_CUDA);
+  ctx->n_sms = prop.multiProcessorCount;
+  if (ctx->use_umma) {
+    if (prop.major != 10) return fail(FC_ERR_SHAPE);
+    if (shape->d_model < 64 || shape->d_ffn < 64 || ctx->d.qd < 64) return fail(FC_ERR_SHAPE);
+    char msg[200];
+    for (int l = 0; l < L && rc == FC_OK; ++l) {
+      UmmaPlan *p;
+      if (!(p = umma_plan_create(args_qkv(ctx, l), PRO_GAIN, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_qkv.push_back(p);
+      if (rc == FC_OK) { if (!(p = umma_plan_create(args_o(ctx, l), PRO_NONE, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_o.push_back(p); }
+      if (rc == FC_OK) { if (!(p = umma_plan_create(args_gu(ctx, l), PRO_GAIN, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_gu.push_back(p); }
+      if (rc == FC_OK) { if (!(p = umma_plan_create(args_down(ctx, l), PRO_SILU_MUL, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_down.push_back(p); }
+    }
+    if (rc == FC_OK && !(ctx->plan_head = umma_plan_create(args_head(ctx), PRO_GAIN, EPI_ARGMAX, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA;
+    if (rc != FC_OK) { fprintf(stderr, "fc_init: %s\n", msg); return fail(rc); }
+  }
+  const size_t pin_ints = (size_t)shape->max_batch * (1 + 2 * shape->max_c) + 4;
+  if (cudaMallocHost((void **)&ctx->pin, pin_ints * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
+  if (cudaEventCreate(&ctx->ev0) != cudaSuccess || cudaEventCreate(&ctx->ev1) != cudaSuccess) return fail(FC_ERR_CUDA);
+  if (cudaMemsetAsync(ws, 0, fc_workspace_bytes(shape), ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
+  if (cudaStreamSynchronize(ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
+  const int B = shape->max_batch;
+  ctx->kv_len_h.assign(B, 0); ctx->n_gen_h.assign(B, 0); ctx->pending_h.assign(B, 0); ctx->done_h.assign(B, 0);
+  *out = ctx;
+  return FC_OK;
+}
+
+static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi) {
+  a.R = R;
+  ++ctx->launches;
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, ctx->st);
+  return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
+}
+
+// One decoder forward over nb sequences (b0 .. b0+nb-1) with `rows` rows each.  tokens: device [nb*rows].
+// with_head: LM head + argmax + accept (a decode step); otherwise the rows are committed (prefill chunk).
+static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens, bool with_head, int max_len_host,
+                   int commit) {
+  const fc_model_shape &s = ctx->s;
+  const Dims &d = ctx->d;
+  const int R = nb * rows;
+  const size_t Rz = R;
+  EmbedArgs ea; memset(&ea, 0, sizeof ea);
+  ea.tokens = tokens; ea.emb = ctx->tok_emb; ea.x = ctx->b.x; ea.R = R; ea.d = s.d_model;
+  ea.z.p[0] = ctx->b.qkv; ea.z.n[0] = Rz * d.ldq;
+  ea.z.p[1] = ctx->b.gu; ea.z.n[1] = Rz * 2 * s.d_ffn;
+  ea.z.p[2] = ctx->b.ss_attn; ea.z.n[2] = Rz;
+  ea.z.p[3] = ctx->b.ss_ffn; ea.z.n[3] = Rz;
+  ++ctx->launches;
+  FC_CK(launch_embed(ea, s.dtype, ctx->st));
+
+  const int nsplit = (max_len_host + rows + d.tk - 1) / d.tk;
+  const long long stride_h = (long long)s.max_seq * s.head_dim;
+  const long long stride_b = (long long)s.n_kv_heads * stride_h;
+  for (int l = 0; l < s.n_layers; ++l) {
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD));
+    RopeArgs ra; memset(&ra, 0, sizeof ra);
+    ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
+    ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows;
+    ra.hq = s.n_heads; ra.hkv = s.n_kv_heads; ra.hd = s.head_dim; ra.theta = s.rope_theta;
+    ra.q_out = ctx->b.qb;
+    ra.kcache = ctx->kv + (size_t)l * ctx->kv_layer_stride;
+    ra.vcache = ctx->kv + (size_t)l * ctx->kv_layer_stride + ctx->kv_half_stride;
+    ra.stride_b = stride_b; ra.stride_h = stride_h;
+    ra.z.p[0] = ctx->b.gu; ra.z.n[0] = Rz * 2 * s.d_ffn;
+    ra.z.p[1] = ctx->b.ss_ffn; ra.z.n[1] = Rz;
+    ++ctx->launches;
+    FC_CK(launch_rope_kv(ra, s.dtype, ctx->st));
+    AttnArgs aa; memset(&aa, 0, sizeof aa);
+    aa.q = ctx->b.qb; aa.kcache = ra.kcache; aa.vcache = ra.vcache; aa.stride_b = stride_b; aa.stride_h = stride_h;
+    aa.kv_len = ctx->b.kv_len; aa.b0 = b0; aa.nb = nb; aa.c = rows; aa.hq = s.n_heads; aa.hkv = s.n_kv_heads;
+    aa.nsplit = nsplit; aa.part_o = ctx->b.part_o; aa.part_ml = ctx->b.part_ml; aa.counters = ctx->b.counters;
+    aa.out = ctx->b.attn;
+    aa.z.p[0] = ctx->b.ss_attn; aa.z.n[0] = Rz;
+    ++ctx->launches;
+    FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st));
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD));
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD));
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD));
+  }
+  if (with_head) {
+    GemmArgs ha = args_head(ctx);
+    ha.tokens = tokens;
+    FC_CK(run_gemm(ctx, ctx->plan_head, ha, R, PRO_GAIN, EPI_ARGMAX));
+    AcceptArgs ac; memset(&ac, 0, sizeof ac);
+    ac.window = ctx->b.window; ac.amax = ctx->b.amax; ac.amax_clear = ctx->b.amax;
+    ac.kv_len = ctx->b.kv_len; ac.n_gen = ctx->b.n_gen; ac.done = ctx->b.done;
+    ac.accepted_count = ctx->b.acc_count; ac.accepted_tokens = ctx->b.acc_tokens;
+    ac.prompt = ctx->b.prompt; ac.prompt_lens = ctx->b.prompt_lens;
+    ac.out_tokens = ctx->b.out_tokens; ac.out_stride = s.max_seq;
+    ac.b0 = b0; ac.nb = nb; ac.c = rows; ac.p_stride = s.max_seq; ac.refill = ctx->refill; ac.pad_id = ctx->pad_id;
+    ac.max_tokens = ctx->gen_max_tokens; ac.eos_id = ctx->gen_eos; ac.commit = commit;
+    ++ctx->launches;
+    FC_CK(launch_accept(ac, ctx->st));
+  } else {
+    for (int b = b0; b < b0 + nb; ++b) {
+      ++ctx->launches;
+      bump_kernel<<<1, 32, 0, ctx->st>>>(ctx->b.kv_len + b, rows);
+      FC_CK(cudaGetLastError());
+    }
+  }
+  return FC_OK;
+}
+
+static int check_device_error(fc_ctx *ctx) {
+  unsigned int e = 0;
+  FC_CK(cudaMemcpyAsync(&ctx->pin[0], ctx->b.err, sizeof(e), cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  e = (unsigned int)ctx->pin[0];
+  if (e) {
+    cudaMemsetAsync(ctx->b.err, 0, sizeof(e), ctx->st);
+    ctx->ready = false;
+    return FC_ERR_DEVICE_TIMEOUT;
+  }
+  return FC_OK;
+}
+
+extern "C" int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids, int32_t p_stride,
+                          const int32_t *prompt_lens, int32_t c, int32_t refill, int32_t pad_id) {
+  if (!ctx || !prompt_ids || !prompt_lens || batch < 1 || c < 1 || p_stride < 1) return FC_ERR_ARG;
+  if (refill != FC_REFILL_PROMPT_CYCLE && refill != FC_REFILL_PAD) return FC_ERR_ARG;
+  const fc_model_shape &s = ctx->s;
+  if (batch > s.max_batch || c > s.max_c) return FC_ERR_CAPACITY;
+  if (refill == FC_REFILL_PAD && (pad_id < 0 || pad_id >= s.vocab)) return FC_ERR_TOKEN_RANGE;
+  for (int b = 0; b < batch; ++b) {
+    const int P = prompt_lens[b];
+    if (P < 1 || P > p_stride) return FC_ERR_ARG;
+    if (P - 1 + c > s.max_seq) return FC_ERR_CAPACITY;
+    for (int i = 0; i < P; ++i) {
+      const int t = prompt_ids[(size_t)b * p_stride + i];
+      if (t < 0 || t >= s.vocab) return FC_ERR_TOKEN_RANGE;
+    }
+  }
+  ctx->ready = false;
+  ctx->launches = 0;
+  ctx->batch = batch; ctx->c = c; ctx->refill = refill; ctx->pad_id = pad_id;
+  ctx->gen_max_tokens = 0; ctx->gen_eos = -1;
+  // device copies of the prompts, zeroed sequence state, initial windows
+  std::vector<int32_t> win((size_t)batch * c), zeros(batch, 0);
+  for (int b = 0; b < batch; ++b) {
+    const int P = prompt_lens[b];
+    FC_CK(cudaMemcpyAsync(ctx->b.prompt + (size_t)b * s.max_seq, prompt_ids + (size_t)b * p_stride,
+                          sizeof(int32_t) * P, cudaMemcpyHostToDevice, ctx->st));
+    win[(size_t)b * c] = prompt_ids[(size_t)b * p_stride + P - 1];
+    for (int j = 1; j < c; ++j)
+      win[(size_t)b * c + j] = refill == FC_REFILL_PAD ? pad_id : prompt_ids[(size_t)b * p_stride + (j - 1) % P];
+    ctx->kv_len_h[b] = 0; ctx->n_gen_h[b] = 0; ctx->done_h[b] = 0; ctx->pending_h[b] = win[(size_t)b * c];
+  }
+  FC_CK(cudaMemcpyAsync(ctx->b.prompt_lens, prompt_lens, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.window, win.data(), sizeof(int32_t) * win.size(), cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.kv_len, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.n_gen, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.done, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));   // host vectors above go out of scope
+  // K/V of prompt[0 .. P-2], one sequence at a time in chunks of up to rmax rows
+  for (int b = 0; b < batch; ++b) {
+    const int n = prompt_lens[b] - 1;
+    for (int start = 0; start < n; start += ctx->d.rmax) {
+      const int rows = n - start < ctx->d.rmax ? n - start : ctx->d.rmax;
+      int rc = forward(ctx, b, 1, rows, ctx->b.prompt + (size_t)b * s.max_seq + start, false, start, 1);
+      if (rc != FC_OK) return rc;
+    }
+    ctx->kv_len_h[b] = n;
+  }
+  int rc = check_device_error(ctx);
+  if (rc != FC_OK) return rc;
+  ctx->ready = true;
+  return FC_OK;
+}
+
+// Copy (count | tokens | window | err) of the finished step to the host and refresh the host mirrors.
+static int collect_step(fc_ctx *ctx, int32_t *accepted_count, int32_t *accepted_tokens, int32_t *window_out) {
+  const int B = ctx->batch, c = ctx->c;
+  int32_t *p_cnt = ctx->pin, *p_tok = p_cnt + B, *p_win = p_tok + (size_t)B * c, *p_err = p_win + (size_t)B * c;
+  FC_CK(cudaMemcpyAsync(p_cnt, ctx->b.acc_count, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaMemcpyAsync(p_tok, ctx->b.acc_tokens, sizeof(int32_t) * B * c, cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaMemcpyAsync(p_win, ctx->b.window, sizeof(int32_t) * B * c, cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaMemcpyAsync(p_err, ctx->b.err, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  if (*p_err) {
+    cudaMemsetAsync(ctx->b.err, 0, sizeof(int32_t), ctx->st);
+    ctx->ready = false;
+    return FC_ERR_DEVICE_TIMEOUT;
+  }
+  for (int b = 0; b < B; ++b) {
+    const int k = p_cnt[b];
+    ctx->kv_len_h[b] += k; ctx->n_gen_h[b] += k; ctx->pending_h[b] = p_win[(size_t)b * c];
+    if (k > 0) {
+      if (ctx->gen_max_tokens > 0 && ctx->n_gen_h[b] >= ctx->gen_max_tokens) ctx->done_h[b] = 1;
+      if (ctx->gen_eos >= 0 && p_tok[(size_t)b * c + k - 1] == ctx->gen_eos) ctx->done_h[b] = 1;
+    }
+  }
+  if (accepted_count) memcpy(accepted_count, p_cnt, sizeof(int32_t) * B);
+  if (accepted_tokens) memcpy(accepted_tokens, p_tok, sizeof(int32_t) * B * c);
+  if (window_out) memcpy(window_out, p_win, sizeof(int32_t) * B * c);
+  return FC_OK;
+}
+
+static int max_live_len(const fc_ctx *ctx) {
+  int m = 0;
+  for (int b = 0; b < ctx->batch; ++b) m = ctx->kv_len_h[b] > m ? ctx->kv_len_h[b] : m;
+  return m;
+}
+
+extern "C" int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *accepted_count,
+                              int32_t *accepted_tokens, int32_t *window_out) {
+  if (!ctx) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  const int B = ctx->batch, c = ctx->c;
+  for (int b = 0; b < B; ++b)
+    if (ctx->kv_len_h[b] + c > ctx->s.max_seq) return FC_ERR_CAPACITY;
+  if (window_in) {
+    for (int b = 0; b < B; ++b) {
+      if (window_in[(size_t)b * c] != ctx->pending_h[b]) return FC_ERR_BAD_WINDOW;
+      for (int j = 0; j < c; ++j) {
+        const int t = window_in[(size_t)b * c + j];
+        if (t < 0 || t >= ctx->s.vocab) return FC_ERR_TOKEN_RANGE;
+      }
+    }
+    memcpy(ctx->pin, window_in, sizeof(int32_t) * B * c);
+    FC_CK(cudaMemcpyAsync(ctx->b.window, ctx->pin, sizeof(int32_t) * B * c, cudaMemcpyHostToDevice, ctx->st));
+  }
+  ctx->launches = 0;
+  int rc = forward(ctx, 0, B, c, ctx->b.window, true, max_live_len(ctx), 1);
+  if (rc != FC_OK) return rc;
+  return collect_step(ctx, accepted_count, accepted_tokens, window_out);
+}
+
+extern "C" int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t eos_id, int32_t *out_tokens, int32_t *out_lens,
+                           fc_stats *stats) {
+  if (!ctx || !out_tokens || !out_lens || max_tokens < 1) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  const int B = ctx->batch, c = ctx->c;
+  for (int b = 0; b < B; ++b)
+    if (ctx->kv_len_h[b] + (max_tokens - ctx->n_gen_h[b]) + c > ctx->s.max_seq) return FC_ERR_CAPACITY;
+  ctx->gen_max_tokens = max_tokens; ctx->gen_eos = eos_id;
+  if (stats) memset(stats, 0, sizeof(*stats));
+  std::vector<int32_t> cnt(B), tok((size_t)B * c);
+  for (int b = 0; b < B; ++b) {
+    out_lens[b] = 0;
+    if (ctx->n_gen_h[b] >= max_tokens) ctx->done_h[b] = 1;
+  }
+  int64_t launches = 0;
+  FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
+  int rc = FC_OK;
+  for (;;) {
+    bool live = false;
+    for (int b = 0; b < B; ++b) live |= !ctx->done_h[b];
+    if (!live) break;
+    ctx->launches = 0;
+    rc = forward(ctx, 0, B, c, ctx->b.window, true, max_live_len(ctx), 1);
+    if (rc != FC_OK) break;
+    launches += ctx->launches;
+    rc = collect_step(ctx, cnt.data(), tok.data(), nullptr);
+    if (rc != FC_OK) break;
+    for (int b = 0; b < B; ++b) {
+      const int k = cnt[b];
+      for (int j = 0; j < k && out_lens[b] < max_tokens; ++j) out_tokens[(size_t)b * max_tokens + out_lens[b]++] = tok[(size_t)b * c + j];
+      if (stats && k > 0) { stats->accept_hist[k > 64 ? 64 : k]++; stats->tokens += k; }
+    }
+    if (stats) stats->steps++;
+  }
+  ctx->launches = launches;
+  ctx->gen_max_tokens = 0; ctx->gen_eos = -1;
+  if (rc != FC_OK) return rc;
+  FC_CK(cudaEventRecord(ctx->ev1, ctx->st));
+  FC_CK(cudaEventSynchronize(ctx->ev1));
+  if (stats) FC_CK(cudaEventElapsedTime(&stats->ms_steps, ctx->ev0, ctx->ev1));
+  return FC_OK;
+}
+
+extern "C" int fc_debug_set_state(fc_ctx *ctx, int32_t batch, const int32_t *kv_lens, const int32_t *pending,
+                                  int32_t c, int32_t pad_id) {
+  if (!ctx || !kv_lens || !pending || batch < 1 || c < 1) return FC_ERR_ARG;
+  const fc_model_shape &s = ctx->s;
+  if (batch > s.max_batch || c > s.max_c) return FC_ERR_CAPACITY;
+  if (pad_id < 0 || pad_id >= s.vocab) return FC_ERR_TOKEN_RANGE;
+  for (int b = 0; b < batch; ++b) {
+    if (kv_lens[b] < 0 || kv_lens[b] + c > s.max_seq) return FC_ERR_CAPACITY;
+    if (pending[b] < 0 || pending[b] >= s.vocab) return FC_ERR_TOKEN_RANGE;
+  }
+  ctx->ready = false;
+  ctx->batch = batch; ctx->c = c; ctx->refill = FC_REFILL_PAD; ctx->pad_id = pad_id;
+  ctx->gen_max_tokens = 0; ctx->gen_eos = -1;
+  std::vector<int32_t> win((size_t)batch * c, pad_id), zeros(batch, 0), ones(batch, 1);
+  for (int b = 0; b < batch; ++b) {
+    win[(size_t)b * c] = pending[b];
+    ctx->kv_len_h[b] = kv_lens[b]; ctx->n_gen_h[b] = 0; ctx->done_h[b] = 0; ctx->pending_h[b] = pending[b];
+  }
+  FC_CK(cudaMemcpyAsync(ctx->b.window, win.data(), sizeof(int32_t) * win.size(), cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.kv_len, kv_lens, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.n_gen, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.done, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.prompt_lens, ones.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  ctx->ready = true;
+  return FC_OK;
+}
+
+extern "C" int fc_debug_logits(fc_ctx *ctx, float *dev_logits) {
+  if (!ctx) return FC_ERR_ARG;
+  ctx->dbg_logits = dev_logits;
+  return FC_OK;
+}
+
+extern "C" int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen) {
+  if (!ctx) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  for (int b = 0; b < ctx->batch; ++b) {
+    if (kv_lens) kv_lens[b] = ctx->kv_len_h[b];
+    if (n_gen) n_gen[b] = ctx->n_gen_h[b];
+  }
+  return FC_OK;
+}
+
+extern "C" int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, float *ms_total) {
+  if (!ctx || n_steps < 1 || !ms_total) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  for (int b = 0; b < ctx->batch; ++b)
+    if (ctx->kv_len_h[b] + ctx->c > ctx->s.max_seq) return FC_ERR_CAPACITY;
+  ctx->launches = 0;
+  const int maxlen = max_live_len(ctx);
+  FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
+  for (int i = 0; i < n_steps; ++i) {
+    int rc = forward(ctx, 0, ctx->batch, ctx->c, ctx->b.window, true, maxlen, 0);
+    if (rc != FC_OK) return rc;
+  }
+  FC_CK(cudaEventRecord(ctx->ev1, ctx->st));
+  FC_CK(cudaEventSynchronize(ctx->ev1));
+  FC_CK(cudaEventElapsedTime(ms_total, ctx->ev0, ctx->ev1));
+  return check_device_error(ctx);
+}
+
+// ------------------------------------------------------------------------------------ single operations
+static __device__ unsigned int g_op_err;
+
+extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, int32_t N, int32_t K, int32_t dtype,
+                            int32_t use_tensor_cores, void *cuda_stream) {
+  if (!x || !w || !y || R < 1 || N < 1 || K < 8 || K % 8) return FC_ERR_ARG;
+  if (dtype != FC_F32 && dtype != FC_BF16) return FC_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  GemmArgs a; memset(&a, 0, sizeof a);
+  a.x = x; a.ldx = K; a.w[0] = w; a.n_rows[0] = N; a.n_mats = 1; a.y = y; a.ldy = N; a.R = R; a.K = K;
+  a.eps = 1e-5f; a.dn = K;
+  if (!use_tensor_cores) {
+    if (launch_gemm_simt(a, dtype, PRO_NONE, EPI_ATOMIC_ADD, st) != cudaSuccess) return FC_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+  }
+  if (dtype != FC_BF16 || K < 64) return FC_ERR_SHAPE;
+  int dev = 0, sms = 0;
+  unsigned int *err_word = nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaGetSymbolAddress((void **)&err_word, g_op_err) != cudaSuccess) return FC_ERR_CUDA;
+  if (cudaMemsetAsync(err_word, 0, sizeof(unsigned int), st) != cudaSuccess) return FC_ERR_CUDA;
+  char msg[200];
+  UmmaPlan *pl = umma_plan_create(a, PRO_NONE, EPI_ATOMIC_ADD, sms, err_word, msg, sizeof msg);
+  if (!pl) { fprintf(stderr, "fc_op_linear: %s\n", msg); return FC_ERR_CUDA; }
+  cudaError_t e = launch_gemm_umma(pl, a, st);
+  unsigned int herr = 0;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&herr, err_word, sizeof herr, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  umma_plan_destroy(pl);
+  if (e != cudaSuccess) { fprintf(stderr, "fc_op_linear: %s\n", cudaGetErrorString(e)); return FC_ERR_CUDA; }
+  return herr ? FC_ERR_DEVICE_TIMEOUT : FC_OK;
+}
+
+extern "C" int fc_op_accept(int32_t *window, const int32_t *argmax, int32_t *kv_len, int32_t *n_gen,
+                            int32_t *accepted_count, int32_t *accepted_tokens, const int32_t *prompt,
+                            const int32_t *prompt_lens, int32_t batch, int32_t c, int32_t p_stride, int32_t refill,
+                            int32_t pad_id, void *cuda_stream) {
+  if (!window || !argmax || !kv_len || !n_gen || !accepted_count || !accepted_tokens) return FC_ERR_ARG;
+  if (batch < 1 || c < 1 || c > 64) return FC_ERR_ARG;
+  if (refill == FC_REFILL_PROMPT_CYCLE && (!prompt || !prompt_lens || p_stride < 1)) return FC_ERR_ARG;
+  AcceptArgs ac; memset(&ac, 0, sizeof ac);
+  ac.window = window; ac.argmax = argmax; ac.kv_len = kv_len; ac.n_gen = n_gen;
+  ac.accepted_count = accepted_count; ac.accepted_tokens = accepted_tokens; ac.prompt = prompt; ac.prompt_lens = prompt_lens;
+  ac.nb = batch; ac.c = c; ac.p_stride = p_stride; ac.refill = refill; ac.pad_id = pad_id; ac.eos_id = -1; ac.commit = 1;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (launch_accept(ac, st) != cudaSuccess) return FC_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+}

@@ -1,0 +1,124 @@
+// Internal declarations shared by the CUDA sources of the Jacobi-window decode library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fastcot.h"
+
+namespace fc {
+
+// ---- activation transform applied while an fp32 buffer is staged as the GEMM's row operand ----
+enum ProOp : int {
+  PRO_NONE = 0,      // x
+  PRO_GAIN = 1,      // x * gain[k]                (RMSNorm gain; the 1/rms row factor is applied by the consumer)
+  PRO_SILU_MUL = 2   // silu(s_r * g) * (s_r * u)  (SwiGLU on gate/up accumulators that still lack 1/rms)
+};
+enum EpiOp : int {
+  EPI_ATOMIC_ADD = 0,  // y[r, n] += acc  (split-K partial sums, or += onto the residual stream)
+  EPI_ARGMAX = 1       // logits = s_r * acc + bias; per-row running (max, lowest index) via 64-bit atomicMax
+};
+
+constexpr int kMaxMats = 3;
+
+struct GemmArgs {
+  // row operand: fp32 [R, K] with leading dimension ldx
+  const float *x;
+  const float *x2;        // PRO_SILU_MUL: the "up" half (x is the "gate" half)
+  int ldx;
+  const void *gain;       // PRO_GAIN: [K] in the weight dtype
+  const float *ss_in;     // PRO_SILU_MUL: per-row sum of squares of the normalised input; s_r = rsqrt(ss/dn + eps)
+  float *ss_out;          // PRO_GAIN: if non-null, sum_k x[r,k]^2 is accumulated here (once per k)
+  float eps;
+  int dn;                 // width the sums of squares are means over (d_model)
+  // weights: up to three matrices [n_rows[m], K], outputs concatenated at column offsets y_off[m]
+  const void *w[kMaxMats];
+  int n_rows[kMaxMats];
+  int y_off[kMaxMats];
+  int n_mats;
+  float *y;
+  int ldy;
+  int R, K;
+  // EPI_ARGMAX
+  const int32_t *tokens;          // [R] input token of each row (bias lookup)
+  const int32_t *perm;            // [vocab] or null
+  float beta;
+  unsigned long long *amax;       // [R] packed (ordered logit << 32 | ~index)
+  float *logits;                  // optional dump [R, vocab]
+  int vocab;
+};
+
+struct ZeroList {       // buffers a kernel clears on the side (fp32 words)
+  float *p[4];
+  unsigned long long n[4];
+};
+
+struct RopeArgs {
+  float *qkv;             // [R, ldq] accumulators: q | k | v, unscaled by 1/rms; cleared after reading
+  int ldq;
+  const float *ss;        // [R] sums of squares for the 1/rms factor
+  float eps; int dn;
+  const int32_t *kv_len;  // [batch] device
+  int b0, nb, c;          // rows r = (b - b0) * c + j
+  int hq, hkv, hd;
+  float theta;
+  void *q_out;            // [R, hq*hd] in the cache dtype
+  void *kcache, *vcache;  // layer base; element strides below
+  long long stride_b, stride_h;   // per sequence, per kv head (elements); token stride is hd
+  ZeroList z;
+};
+
+struct AttnArgs {
+  const void *q;          // [R, hq*hd] cache dtype, already rotated
+  const void *kcache, *vcache;
+  long long stride_b, stride_h;
+  const int32_t *kv_len;
+  int b0, nb, c, hq, hkv;
+  int nsplit;
+  float *part_o;          // [R*hq, nsplit, hd]
+  float *part_ml;         // [R*hq, nsplit, 2]
+  unsigned int *counters; // [batch*hkv], zero on entry, zero on exit
+  float *out;             // [R, hq*hd] fp32
+  ZeroList z;
+};
+
+struct AcceptArgs {
+  int32_t *window;                 // [batch, c] in/out
+  const unsigned long long *amax;  // packed argmax per row, or null
+  unsigned long long *amax_clear;  // cleared after reading (may be null)
+  const int32_t *argmax;           // plain argmax per row (used when amax is null)
+  int32_t *kv_len, *n_gen, *done;  // [batch]; done may be null
+  int32_t *accepted_count, *accepted_tokens;   // [batch], [batch, c]
+  const int32_t *prompt, *prompt_lens;
+  int32_t *out_tokens;             // [batch, out_stride] or null
+  int out_stride;
+  int b0, nb, c, p_stride, refill, pad_id;
+  int max_tokens, eos_id;          // max_tokens <= 0: unlimited
+  int commit;                      // 0: leave kv_len / n_gen / window untouched (latency measurement)
+};
+
+struct EmbedArgs {
+  const int32_t *tokens;   // [R]
+  const void *emb;         // [vocab, d]
+  float *x;                // [R, d]
+  int R, d;
+  ZeroList z;
+};
+
+// ---- launchers (each returns the cudaError_t of the launch) ----
+cudaError_t launch_embed(const EmbedArgs &a, int dtype, cudaStream_t st);
+cudaError_t launch_gemm_simt(const GemmArgs &a, int dtype, int pro, int epi, cudaStream_t st);
+cudaError_t launch_rope_kv(const RopeArgs &a, int dtype, cudaStream_t st);
+cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st);
+cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
+int attn_tile_keys(int dtype, int hd);   // keys per split tile
+
+// tcgen05 path (bf16 only).  `maps` points at prebuilt tensor maps for the weight matrices.
+struct UmmaPlan;
+UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsigned int *err_word,
+                           char *err, int errlen);
+void umma_plan_destroy(UmmaPlan *p);
+// x/x2/y/ss pointers and R may differ per launch from those the plan was created with.
+cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, cudaStream_t st);
+
+}  // namespace fc

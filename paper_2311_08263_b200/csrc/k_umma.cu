@@ -1,0 +1,565 @@
+// Weight-streaming skinny GEMM for sm_100a:  y[R, N] (+)= pro(x)[R, K] . W[N, K]^T,  R = batch * c rows.
+//
+// The contraction is computed "swapped": a 128-row tile of W is the M operand of tcgen05.mma, the
+// R window rows (padded to BN) are the N operand, and the fp32 accumulator [128 x BN] lives in
+// tensor memory.  W tiles (128 rows x 64 k, 16 KB) arrive by TMA into a 128B-swizzled shared-memory
+// ring; the activation operand is produced on chip: four staging warps read the fp32 activations,
+// apply the fused transform (RMSNorm gain, or SwiGLU of the gate/up accumulators), round to bf16 and
+// store them in the same swizzled K-major layout.  Work is split stream-K style: the (tile, k-block)
+// items are dealt out in equal contiguous ranges to a fixed grid, every partial accumulator is added
+// to y with fp32 reductions in L2, so no second pass is needed and HBM traffic is W exactly once.
+//
+// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer + TMEM owner, 2-5 = activation staging,
+// 6-9 = epilogue (TMEM -> registers -> global).  Two accumulators alternate so the epilogue of one
+// segment overlaps the MMAs of the next.  Every mbarrier wait is bounded; on expiry the CTA records
+// an error word, drains its own copies and MMAs (bounded too), frees TMEM and returns.
+#include <cuda.h>
+
+#include <cstdio>
+#include <cstring>
+
+#include "fc_internal.h"
+
+namespace fc {
+
+constexpr int kTileM = 128;       // weight rows per tile
+constexpr int kTileK = 64;        // k elements per stage (128 bytes of bf16 = one swizzle row)
+constexpr int kWBytes = kTileM * kTileK * 2;
+constexpr int kThreads = 320;
+constexpr unsigned long long kSpinBudget = 4000000000ull;   // clock64 ticks (~2 s)
+
+struct UmmaParams {
+  GemmArgs g;
+  int n_tiles, nkb;               // 128-row tiles over all matrices; 64-wide k blocks
+  int tiles_m[kMaxMats];
+  int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
+  int stages;
+  int items_per_cta_mode;         // 0: stream-K ranges, 1: whole tiles round-robin (argmax epilogue)
+  unsigned int *err;              // device error word (0 = ok)
+};
+
+struct UmmaPlan {
+  UmmaParams p;
+  CUtensorMap maps[kMaxMats];
+  int pro, epi, grid, n_sms;
+  unsigned int *err;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the budget ran out or another role raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  unsigned int spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 0xFFu) == 0u) {
+      if (*abort_flag) return false;
+      if ((unsigned long long)(clock64() - t0) > kSpinBudget) { *abort_flag = 1; return false; }
+    }
+  }
+  return true;
+}
+// Same for a converged warp: every lane waits, and the verdict is made uniform so that the lanes of a
+// warp can never part ways around a later warp-level synchronisation.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B apart, 8-row groups
+// 1024 B apart (the tile base is 1024-byte aligned; k sub-blocks advance the start address by 32 B).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024u >> 4) << 32;                 // stride byte offset
+  d |= (uint64_t)1 << 46;                            // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = bn.
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ unsigned int ordered_key_u(float v) {
+  if (v != v) return 0u;
+  unsigned int u = __float_as_uint(v);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+struct Segment { int tile, kb0, kb1; };
+
+// Work of one CTA: stream-K mode deals contiguous (tile, k-block) ranges; tile mode deals whole tiles.
+struct SegIter {
+  long long w, w1;      // stream-K cursor
+  int tile, tile_step, n_tiles, nkb, mode;
+  __device__ SegIter(const UmmaParams &p) {
+    mode = p.items_per_cta_mode; nkb = p.nkb; n_tiles = p.n_tiles;
+    if (mode == 0) {
+      const long long W = (long long)p.n_tiles * p.nkb;
+      w = W * blockIdx.x / gridDim.x;
+      w1 = W * (blockIdx.x + 1) / gridDim.x;
+    } else { tile = blockIdx.x; tile_step = gridDim.x; w = w1 = 0; }
+  }
+  __device__ bool next(Segment &s) {
+    if (mode == 0) {
+      if (w >= w1) return false;
+      s.tile = (int)(w / nkb); s.kb0 = (int)(w % nkb);
+      long long rem = w1 - w;
+      s.kb1 = (int)((nkb - s.kb0 < rem) ? nkb : s.kb0 + rem);
+      w += s.kb1 - s.kb0;
+      return true;
+    }
+    if (tile >= n_tiles) return false;
+    s.tile = tile; s.kb0 = 0; s.kb1 = nkb; tile += tile_step;
+    return true;
+  }
+};
+
+__device__ __forceinline__ void tile_info(const UmmaParams &p, int tile, int &m, int &row0, int &rows_valid, int &ycol0) {
+  m = 0;
+  int lt = tile;
+  while (m + 1 < p.g.n_mats && lt >= p.tiles_m[m]) { lt -= p.tiles_m[m]; ++m; }
+  row0 = lt * kTileM;
+  rows_valid = min(kTileM, p.g.n_rows[m] - row0);
+  ycol0 = p.g.y_off[m] + row0;
+}
+
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o);
+    v = t > v ? t : v;
+  }
+  return v;
+}
+
+template <int PRO, int EPI, int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
+                 const __grid_constant__ CUtensorMap map2, const UmmaParams p) {
+  constexpr int kStageBytes = kWBytes + BN * 128;
+  constexpr int kUnits = BN / 16;                 // (row, 16-byte chunk) units per staging thread per stage
+  constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
+  constexpr uint32_t kIdesc = make_idesc(BN);
+
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  __shared__ float ss_s[2][BN];
+
+  const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int S = p.stages;
+  const GemmArgs &g = p.g;
+  const int nrb = (g.R + BN - 1) / BN;
+  volatile int *abort_flag = &abort_s;
+
+  if (threadIdx.x == 0) {
+    abort_s = 0;
+    for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&full_w[i]), 1); mbar_init(smem_u32(&full_x[i]), 4); mbar_init(smem_u32(&empty_b[i]), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
+    mbar_init(smem_u32(&drain_bar), 1);
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), kCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  int issued = 0;   // producer: k-block loads issued (for the drain on abort)
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int rb = 0; rb < nrb && ok; ++rb) {
+        SegIter si(p);
+        Segment s;
+        while (ok && si.next(s)) {
+          int m, row0, rows_valid, ycol0;
+          tile_info(p, s.tile, m, row0, rows_valid, ycol0);
+          const CUtensorMap *mp = (m == 0) ? &map0 : (m == 1 ? &map1 : &map2);
+          for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+            const int stage = it % S;
+            const uint32_t ph = (uint32_t)(it / S) & 1u;
+            if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t bar = smem_u32(&full_w[stage]);
+            mbar_expect_tx(bar, (uint32_t)p.tx_bytes[m]);
+            tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
+            issued = it + 1;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int it = 0, seg = 0;
+      bool ok = true;
+      for (int rb = 0; rb < nrb && ok; ++rb) {
+        SegIter si(p);
+        Segment s;
+        while (ok && si.next(s)) {
+          const int acc = seg & 1;
+          if (!mbar_wait(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+          for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+            const int stage = it % S;
+            const uint32_t ph = (uint32_t)(it / S) & 1u;
+            if (!mbar_wait(smem_u32(&full_w[stage]), ph, abort_flag) ||
+                !mbar_wait(smem_u32(&full_x[stage]), ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_base = smem_base + stage * kStageBytes;
+            const uint32_t b_base = a_base + kWBytes;
+#pragma unroll
+            for (int kk = 0; kk < kTileK / 16; ++kk)
+              umma_bf16(d_tmem, smem_desc_sw128(a_base + kk * 32), smem_desc_sw128(b_base + kk * 32), kIdesc,
+                        (kb > s.kb0 || kk > 0) ? 1u : 0u);
+            umma_commit(smem_u32(&empty_b[stage]));
+          }
+          if (ok) umma_commit(smem_u32(&accum_full[acc]));
+          ++seg;
+        }
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------ activation staging
+    const int tid_s = threadIdx.x - 64;
+    int it = 0, seg = 0;
+    bool ok = true;
+    for (int rb = 0; rb < nrb && ok; ++rb) {
+      SegIter si(p);
+      Segment s;
+      while (ok && si.next(s)) {
+        const int acc = seg & 1;
+        float ssq[kUnits], srow[kUnits];
+#pragma unroll
+        for (int u = 0; u < kUnits; ++u) {
+          ssq[u] = 0.f; srow[u] = 1.f;
+          if (PRO == PRO_SILU_MUL) {
+            const int r = rb * BN + ((u * 128 + tid_s) >> 3);
+            if (r < g.R) srow[u] = rsqrtf(g.ss_in[r] / (float)g.dn + g.eps);
+          }
+        }
+        for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+          const int stage = it % S;
+          const uint32_t ph = (uint32_t)(it / S) & 1u;
+          if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+          unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
+#pragma unroll
+          for (int u = 0; u < kUnits; ++u) {
+            const int unit = u * 128 + tid_s;
+            const int row = unit >> 3, chunk = unit & 7;
+            const int r = rb * BN + row, k = kb * kTileK + chunk * 8;
+            float v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+            if (r < g.R && k < g.K) {
+              const float4 a0 = *reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k);
+              const float4 a1 = *reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k + 4);
+              v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+              if (PRO == PRO_GAIN) {
+                const uint4 gq = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
+                const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float2 gf = __bfloat1622float2(gp[i]);
+                  ssq[u] = fmaf(v[2 * i], v[2 * i], ssq[u]); ssq[u] = fmaf(v[2 * i + 1], v[2 * i + 1], ssq[u]);
+                  v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
+                }
+              } else if (PRO == PRO_SILU_MUL) {
+                const float4 u0 = *reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k);
+                const float4 u1 = *reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k + 4);
+                const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float gt = srow[u] * v[i];
+                  v[i] = (gt / (1.0f + __expf(-gt))) * (srow[u] * uu[i]);
+                }
+              }
+            }
+            uint4 pk;
+            __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
+            pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+            pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+            *reinterpret_cast<uint4 *>(xs + (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+          }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&full_x[stage]));
+        }
+        if (!ok) break;
+        if (PRO == PRO_GAIN && (EPI == EPI_ARGMAX || (g.ss_out != nullptr && s.tile == 0))) {
+          if (EPI == EPI_ARGMAX) {   // ss_s[acc] is free once the epilogue two segments back has let go of it
+            if (!mbar_wait_warp(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          }
+#pragma unroll
+          for (int u = 0; u < kUnits; ++u) {
+            float t = ssq[u];
+            t += __shfl_xor_sync(0xffffffffu, t, 1);
+            t += __shfl_xor_sync(0xffffffffu, t, 2);
+            t += __shfl_xor_sync(0xffffffffu, t, 4);
+            const int unit = u * 128 + tid_s;
+            const int row = unit >> 3, r = rb * BN + row;
+            if ((unit & 7) == 0) {
+              if (EPI == EPI_ARGMAX) ss_s[acc][row] = t;
+              else if (r < g.R) atomicAdd(&g.ss_out[r], t);
+            }
+          }
+          if (EPI == EPI_ARGMAX) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ss_ready[acc]));
+          }
+        }
+        ++seg;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue
+    const int q = warp & 3;
+    const int n_local = q * 32 + lane;
+    int seg = 0;
+    bool ok = true;
+    for (int rb = 0; rb < nrb && ok; ++rb) {
+      SegIter si(p);
+      Segment s;
+      while (ok && si.next(s)) {
+        int m, row0, rows_valid, ycol0;
+        tile_info(p, s.tile, m, row0, rows_valid, ycol0);
+        const int acc = seg & 1;
+        const uint32_t ph = ((uint32_t)seg >> 1) & 1u;
+        if (!mbar_wait_warp(smem_u32(&accum_full[acc]), ph, abort_flag)) { ok = false; break; }
+        if (EPI == EPI_ARGMAX && !mbar_wait_warp(smem_u32(&ss_ready[acc]), ph, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const bool valid = n_local < rows_valid;
+        const int col = ycol0 + n_local;
+        for (int c0 = 0; c0 < BN; c0 += 16) {
+          if (rb * BN + c0 >= g.R) break;
+          float v[16];
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int r = rb * BN + c0 + j;
+            if (r >= g.R) break;
+            if (EPI == EPI_ATOMIC_ADD) {
+              if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
+            } else {
+              float logit = v[j] * rsqrtf(ss_s[acc][c0 + j] / (float)g.dn + g.eps);
+              unsigned long long key = 0ull;
+              if (valid) {
+                if (g.perm && g.perm[g.tokens[r]] == col) logit += g.beta;
+                if (g.logits) g.logits[(long long)r * g.vocab + col] = logit;
+                key = ((unsigned long long)ordered_key_u(logit) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned int)col);
+              }
+              key = warp_max_u64(key);
+              if (lane == 0) atomicMax(&g.amax[r], key);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[acc]));
+        ++seg;
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  __syncthreads();
+  if (abort_s) {
+    if (threadIdx.x == 0) {
+      atomicExch(p.err, 1u);
+      // wait (bounded) for this CTA's own TMA copies still in flight
+      const unsigned long long t0 = clock64();
+      for (int i = (issued > S ? issued - S : 0); i < issued; ++i) {
+        const uint32_t bar = smem_u32(&full_w[i % S]);
+        while (!mbar_try(bar, (uint32_t)(i / S) & 1u))
+          if ((unsigned long long)(clock64() - t0) > kSpinBudget / 4) break;
+      }
+    }
+    if (warp == 1 && lane == 0) {
+      // and for MMAs already issued
+      umma_commit(smem_u32(&drain_bar));
+      const unsigned long long t0 = clock64();
+      while (!mbar_try(smem_u32(&drain_bar), 0u))
+        if ((unsigned long long)(clock64() - t0) > kSpinBudget / 4) break;
+    }
+    __syncthreads();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, kCols); }
+}
+
+// ------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)sym;
+  }
+  return fn;
+}
+
+static void bn_config(int R, int &bn, int &stages, int &ctas_per_sm) {
+  if (R <= 16) { bn = 16; stages = 6; ctas_per_sm = 2; }
+  else if (R <= 32) { bn = 32; stages = 5; ctas_per_sm = 2; }
+  else if (R <= 64) { bn = 64; stages = 4; ctas_per_sm = 2; }
+  else if (R <= 128) { bn = 128; stages = 6; ctas_per_sm = 1; }
+  else { bn = 256; stages = 4; ctas_per_sm = 1; }
+}
+
+UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsigned int *err_word,
+                           char *err, int errlen) {
+  auto fail = [&](const char *msg) -> UmmaPlan * { if (err) snprintf(err, errlen, "%s", msg); return nullptr; };
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return fail("cuTensorMapEncodeTiled entry point not available");
+  if (a.K < kTileK || a.K % 8) return fail("tensor-core path needs K >= 64 and K % 8 == 0");
+  if (a.n_mats < 1 || a.n_mats > kMaxMats) return fail("bad matrix count");
+  UmmaPlan *pl = new UmmaPlan();
+  memset(pl, 0, sizeof(*pl));
+  pl->p.g = a;
+  pl->pro = pro; pl->epi = epi; pl->n_sms = n_sms; pl->err = err_word;
+  pl->p.err = err_word;
+  pl->p.nkb = (a.K + kTileK - 1) / kTileK;
+  pl->p.n_tiles = 0;
+  for (int m = 0; m < a.n_mats; ++m) {
+    if (a.n_rows[m] < 1) { delete pl; return fail("empty weight matrix"); }
+    pl->p.tiles_m[m] = (a.n_rows[m] + kTileM - 1) / kTileM;
+    pl->p.n_tiles += pl->p.tiles_m[m];
+    const cuuint32_t box_rows = (cuuint32_t)(a.n_rows[m] < kTileM ? a.n_rows[m] : kTileM);
+    pl->p.tx_bytes[m] = (int)(box_rows * kTileK * 2);
+    cuuint64_t gdim[2] = {(cuuint64_t)a.K, (cuuint64_t)a.n_rows[m]};
+    cuuint64_t gstr[1] = {(cuuint64_t)a.K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTileK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(&pl->maps[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(a.w[m]), gdim, gstr, box,
+                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { delete pl; return fail("cuTensorMapEncodeTiled failed (weight pointer must be 16-byte aligned)"); }
+  }
+  for (int m = a.n_mats; m < kMaxMats; ++m) pl->maps[m] = pl->maps[0];
+  pl->p.items_per_cta_mode = (epi == EPI_ARGMAX) ? 1 : 0;
+  return pl;
+}
+
+void umma_plan_destroy(UmmaPlan *p) { delete p; }
+
+template <int PRO, int EPI, int BN>
+static cudaError_t launch_one(const UmmaPlan *pl, const UmmaParams &p, int grid, cudaStream_t st) {
+  const size_t smem = (size_t)p.stages * (kWBytes + BN * 128) + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<PRO, EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  gemm_umma_kernel<PRO, EPI, BN><<<grid, kThreads, smem, st>>>(pl->maps[0], pl->maps[1], pl->maps[2], p);
+  return cudaGetLastError();
+}
+
+template <int PRO, int EPI>
+static cudaError_t launch_bn(const UmmaPlan *pl, const UmmaParams &p, int bn, int grid, cudaStream_t st) {
+  switch (bn) {
+    case 16: return launch_one<PRO, EPI, 16>(pl, p, grid, st);
+    case 32: return launch_one<PRO, EPI, 32>(pl, p, grid, st);
+    case 64: return launch_one<PRO, EPI, 64>(pl, p, grid, st);
+    case 128: return launch_one<PRO, EPI, 128>(pl, p, grid, st);
+    default: return launch_one<PRO, EPI, 256>(pl, p, grid, st);
+  }
+}
+
+cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, cudaStream_t st) {
+  UmmaParams p = pl->p;
+  // per-launch fields (buffers and row count); weights, K and the matrix split stay as planned
+  p.g.x = a.x; p.g.x2 = a.x2; p.g.ldx = a.ldx; p.g.ss_in = a.ss_in; p.g.ss_out = a.ss_out;
+  p.g.y = a.y; p.g.ldy = a.ldy; p.g.R = a.R; p.g.tokens = a.tokens; p.g.amax = a.amax; p.g.logits = a.logits;
+  int bn, cps;
+  bn_config(a.R, bn, p.stages, cps);
+  int grid;
+  if (p.items_per_cta_mode == 0) {
+    const long long W = (long long)p.n_tiles * p.nkb;
+    long long cap = W / 4 > 0 ? W / 4 : 1;
+    grid = (int)((long long)pl->n_sms * cps < cap ? (long long)pl->n_sms * cps : cap);
+  } else {
+    grid = p.n_tiles < pl->n_sms * cps ? p.n_tiles : pl->n_sms * cps;
+  }
+  if (pl->epi == EPI_ARGMAX) return launch_bn<PRO_GAIN, EPI_ARGMAX>(pl, p, bn, grid, st);
+  if (pl->pro == PRO_NONE) return launch_bn<PRO_NONE, EPI_ATOMIC_ADD>(pl, p, bn, grid, st);
+  if (pl->pro == PRO_GAIN) return launch_bn<PRO_GAIN, EPI_ATOMIC_ADD>(pl, p, bn, grid, st);
+  return launch_bn<PRO_SILU_MUL, EPI_ATOMIC_ADD>(pl, p, bn, grid, st);
+}
+
+}  // namespace fc

@@ -249,3 +249,36 @@ def test_golden_tiny_stream():
     cfg, w, prompt = _tiny()
     ar, _ = oracle.Oracle(cfg, w, 160).ar_generate(prompt, 64)
     assert ar.tolist() == want
+
+
+# ---------------------------------------------------------------- the accept rule alone, exhaustively
+@pytest.mark.parametrize("c", [1, 2, 3, 4, 5])
+def test_accept_rule_exhaustive_small_vocab(c):
+    """All (window, argmax) pairs over a 3-token vocabulary: properties that define the rule."""
+    V, prompt = 3, np.array([2, 0, 1, 1], np.int32)
+    for w in itertools.product(range(V), repeat=c):
+        for a in itertools.product(range(V), repeat=c):
+            for n_gen in (0, 3):
+                k, acc, w2 = oracle.accept(w, a, n_gen, prompt)
+                assert 1 <= k <= c
+                assert all(w[j] == a[j - 1] for j in range(1, k))          # accepted guesses were right
+                assert k == c or w[k] != a[k - 1]                           # and the run is maximal
+                assert acc.tolist() == list(a[:k])
+                assert w2[0] == a[k - 1]
+                assert w2[1:c - k + 1].tolist() == list(a[k:c])
+                assert w2[c - k + 1:].tolist() == [prompt[(n_gen + k + j - 1) % 4] for j in range(c - k + 1, c)]
+                _, _, w3 = oracle.accept(w, a, n_gen, prompt, refill=1, pad_id=2)
+                assert w3[c - k + 1:].tolist() == [2] * (k - 1)
+
+
+def test_linear_matches_fp64_matmul():
+    rng = np.random.default_rng(3)
+    w = torch.from_numpy(rng.standard_normal((37, 72)).astype(np.float32))
+    x = rng.standard_normal((5, 72)).astype(np.float32)
+    y = rng.standard_normal((5, 37)).astype(np.float32)
+    got = oracle.linear_add(w, x, y)
+    want = y.astype(np.float64) + x.astype(np.float64) @ w.numpy().astype(np.float64).T
+    assert np.abs(got - want).max() < 1e-5
+    got_b = oracle.linear_add(w.to(torch.bfloat16), x, y)
+    want_b = y.astype(np.float64) + x.astype(np.float64) @ w.to(torch.bfloat16).double().numpy().T
+    assert np.abs(got_b - want_b).max() < 1e-5
