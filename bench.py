@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the Jacobi-window decode step: accepted tokens/s and step latency.
+
+    python bench.py --gpus N --steps K --warmup W [--workload 7b] [--impl reference]
+
+One "step" is one fc_jacobi_step: a decoder forward over the K/V-cached prefix plus a window of c
+tokens, greedy argmax, verification, K/V commit and window shift.  The default workload is the
+7B Llama-shape bf16 model, prompt of 800 random ids, c = 16, batch 1, random-init weights
+(synthetic: stands in for the Llama-2 checkpoints and few-shot prompts of the paper's Section 5.1).
+The path does not shard: with N > 1 every rank runs an independent replica ("weak" scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2311_08263_b200 import workload as wl  # noqa: E402
+
+METRIC = "accepted_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def step_bytes(cfg, batch, c, kv_lens):
+    """Algorithmic bytes of one step: weights once, K/V read + write, embedding rows."""
+    s = cfg.elem_bytes
+    weights = cfg.weight_params() * s
+    kv_tok = cfg.kv_bytes_per_token()
+    kv_read = sum((L + c) * kv_tok for L in kv_lens)
+    kv_write = batch * c * kv_tok
+    return weights + kv_read + kv_write + batch * c * cfg.d_model * s
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def reduce_max_sum(world, t_ms, tokens, device):
+    if world == 1:
+        return t_ms, tokens
+    import torch.distributed as dist
+    a = torch.tensor([t_ms], dtype=torch.float64, device=device)
+    b = torch.tensor([tokens], dtype=torch.float64, device=device)
+    dist.all_reduce(a, op=dist.ReduceOp.MAX)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(a.item()), float(b.item())
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sample(cfg, weights_host, c, kv_len, reps, layers=None):
+    """Times `reps` oracle Jacobi steps (c rows) at K/V length kv_len filled with seeded random K/V.
+
+    This is the one place (besides tests and smoke) where the benchmark touches oracle/.
+    Returns (seconds per step, accepted tokens per step, threads used).
+    """
+    import dataclasses
+    import oracle
+    ocfg = cfg if layers is None else dataclasses.replace(cfg, n_layers=layers)
+    o = oracle.Oracle(ocfg, weights_host, kv_len + c + 8)
+    kvd = cfg.n_kv_heads * cfg.head_dim
+    kv = wl.hash_normal(cfg.seed, 6, kv_len * kvd).view(kv_len, kvd).numpy()
+    for l in range(ocfg.n_layers):
+        o.set_kv(l, kv, kv)
+    # Jacobi state without a prefill: pending token + prompt-cycled guesses, then the oracle's own
+    # forward and accept rule
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    window = np.concatenate([prompt[-1:], prompt[:c - 1]]).astype(np.int32)
+    times, acc = [], 0
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        a, _ = o.forward(window, want_logits=False)
+        k, _, window2 = oracle.accept(window, a, 0, prompt)
+        times.append(time.perf_counter() - t0)
+        acc += k
+    return sum(times) / len(times), acc / reps, oracle.threads()
+
+
+def run_reference(args, cfg, rank, world):
+    """--impl reference: the CPU oracle, as it stands, on this host's cores (rank 0 only)."""
+    if rank != 0:
+        return
+    L, c = cfg.prompt_len, cfg.c
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    w = wl.make_weights(cfg, device=dev)
+    wh = {k: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for k, v in w.items()}
+    del w
+    # size the per-step sample so the whole run stays within a few minutes
+    t_probe, _, threads = oracle_sample(cfg, wh, c, L, 1, layers=1)
+    head_frac = cfg.vocab * cfg.d_model / ((cfg.weight_params() - cfg.vocab * cfg.d_model) / cfg.n_layers + cfg.vocab * cfg.d_model)
+    t_layer = t_probe * (1 - head_frac)
+    t_head = t_probe * head_frac
+    budget = 180.0 / max(1, args.steps + args.warmup)
+    layers = int(max(1, min(cfg.n_layers, (budget - t_head) / max(t_layer, 1e-9))))
+    for _ in range(args.warmup):
+        oracle_sample(cfg, wh, c, L, 1, layers=layers)
+    t, k, threads = oracle_sample(cfg, wh, c, L, args.steps, layers=layers)
+    # a partial-depth sample is scaled to the full depth (cost is linear in layers; the head is counted once)
+    t_full = (t - t_head) * cfg.n_layers / layers + t_head if layers < cfg.n_layers else t
+    value = k / t_full
+    sample = (f"{args.steps} oracle Jacobi steps (c={c}, kv_len={L}, seeded random K/V) over {layers} of "
+              f"{cfg.n_layers} layers + LM head" + (", time scaled to full depth" if layers < cfg.n_layers else ""))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_full * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "batch": 1, "c": c, "kv_len": L},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(cfg):
+    return (f"{cfg.name} Llama-shape {cfg.dtype}: {cfg.n_layers} layers, d_model {cfg.d_model}, "
+            f"{cfg.n_heads}q/{cfg.n_kv_heads}kv heads x {cfg.head_dim}, FFN {cfg.d_ffn}, vocab {cfg.vocab}; "
+            f"prompt {cfg.prompt_len} random ids, c={cfg.c}, batch {cfg.batch}")
+
+
+# ------------------------------------------------------------------------------------------ CUDA leg
+def run_ours(args, cfg, rank, world, local):
+    from paper_2311_08263_b200 import engine
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    c, B, P = cfg.c, cfg.batch, cfg.prompt_len
+    steps, warm = args.steps, args.warmup
+    e2e_steps = min(steps, 50)
+    max_seq = P + (steps + warm + 2 * e2e_steps + 8) * c + 16
+
+    t0 = time.time()
+    w = wl.make_weights(cfg, device=device)
+    dec = engine.Decoder(cfg, w, B, c, max_seq, device=str(device))
+    ids, lens = wl.make_prompts(cfg, batch=B)
+    dec.fc_prefill(ids.numpy(), lens.numpy(), c)
+    setup_s = time.time() - t0
+
+    # ---- device-resident timing: K committed steps back to back, CUDA events, max over ranks
+    dec.fc_bench_steps(warm, commit=True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier(world)
+    torch.cuda.synchronize()
+    kv0 = dec.fc_get_state()[0].copy()
+    ms, tokens = dec.fc_bench_steps(steps, commit=True)
+    launches = dec.fc_last_launch_count()
+    torch.cuda.synchronize()
+    barrier(world)
+    kv1 = dec.fc_get_state()[0].copy()
+    # keep the GPU under the same load while nvidia-smi catches a few more samples
+    if ms < 1500:
+        dec.fc_bench_steps(max(1, int(steps * 1500 / max(ms, 1))), commit=False)
+    clocks = sampler.stop()
+    ms_max, tok_sum = reduce_max_sum(world, ms, tokens, device)
+
+    # ---- end to end: host window in, host results out, every step (wall clock)
+    win = dec.fc_jacobi_step()[2]
+    for _ in range(3):
+        win = dec.fc_jacobi_step(win)[2]
+    barrier(world)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    e2e_tok = 0
+    for _ in range(e2e_steps):
+        cnt, _, win = dec.fc_jacobi_step(win)
+        e2e_tok += int(cnt.sum())
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t1
+    e2e_ms_max, e2e_tok_sum = reduce_max_sum(world, e2e_s * 1e3, e2e_tok, device)
+
+    # ---- per-kernel-class device times (events around every launch of one step)
+    prof = dec.fc_profile_step()
+    prof = dec.fc_profile_step()
+    kv_mid = [int((a + b) // 2) for a, b in zip(kv0, kv1)]
+    sbytes = step_bytes(cfg, B, c, kv_mid)
+    peak, peak_kind = measured_peaks()
+    s = cfg.elem_bytes
+    d, f = cfg.d_model, cfg.d_ffn
+    qd, kvd = cfg.n_heads * cfg.head_dim, cfg.n_kv_heads * cfg.head_dim
+    # dominant kernel: the gate/up projection GEMM (largest share of the streamed bytes)
+    gu_bytes = 2 * d * f * s + B * c * d * 4 + B * c * 2 * f * 4
+    gu_ms, gu_n = prof["gateup"]
+    achieved = gu_bytes * gu_n / (gu_ms * 1e-3) / 1e9 if gu_ms > 0 else 0.0
+    roofline = {"bound": "hbm", "kernel": "gemm_umma_kernel<PRO_GAIN,EPI_ATOMIC_ADD> (gate/up projection)",
+                "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"of {peak_kind}", "traffic": None,
+                "bytes_per_launch": gu_bytes, "ms_per_launch": gu_ms / max(gu_n, 1)}
+    step_ms = ms_max / steps
+    step_gbs = sbytes / (step_ms * 1e-3) / 1e9
+    line = {"metric": METRIC, "value": tok_sum / (ms_max * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warm, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "batch": B, "c": c, "kv_len_start": int(kv0[0]),
+                       "kv_len_end": int(kv1[0]), "l2": "inputs larger than L2 (weights streamed every step)",
+                       "multi_gpu": "replicas only"},
+            "mean_accept": tok_sum / (steps * B * world),
+            "clocks": clocks,
+            "e2e": {"value": e2e_tok_sum / (e2e_ms_max * 1e-3), "unit": UNIT, "steps": e2e_steps,
+                    "ms_per_step": e2e_ms_max / e2e_steps,
+                    "h2d_bytes_per_step": B * c * 4, "d2h_bytes_per_step": B * (1 + 2 * c) * 4 + 4},
+            "gpu_launches": launches,
+            "roofline": roofline,
+            "step_roofline": {"bytes_per_step": sbytes, "achieved_gbs": step_gbs, "frac_of_peak": step_gbs / peak,
+                              "peak_gbs": peak, "peak_kind": peak_kind, "frac_of_8tbs": step_gbs / 8000.0},
+            "kernel_ms": {k: round(v[0], 4) for k, v in prof.items()},
+            "kernel_launches": {k: v[1] for k, v in prof.items()},
+            "setup_s": round(setup_s, 1)}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        wh = {k: ([t.cpu() for t in v] if isinstance(v, list) else v.cpu()) for k, v in w.items()}
+        del dec
+        t_probe, _, threads = oracle_sample(cfg, wh, c, P, 1, layers=1)
+        layers = int(max(1, min(cfg.n_layers, 20.0 / max(t_probe, 1e-9))))
+        t, k, threads = oracle_sample(cfg, wh, c, P, 1, layers=layers)
+        head_frac = cfg.vocab * d / ((cfg.weight_params() - cfg.vocab * d) / cfg.n_layers + cfg.vocab * d)
+        t_head = t_probe * head_frac
+        t_full = (t - t_head) * cfg.n_layers / layers + t_head if layers < cfg.n_layers else t
+        line["cpu_baseline"] = {"value": k / t_full, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"1 oracle Jacobi step (c={c}, kv_len={P}, seeded random K/V) over "
+                                          f"{layers} of {cfg.n_layers} layers + LM head"
+                                          + (", time scaled to full depth" if layers < cfg.n_layers else ""),
+                                "ms_per_step": t_full * 1e3}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="7b", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    cfg = wl.CONFIGS[args.workload]
+    rank, world, local = dist_setup(args.gpus)
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+    else:
+        run_ours(args, cfg, rank, world, local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

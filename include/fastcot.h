@@ -119,10 +119,19 @@ int fc_debug_set_state(fc_ctx *ctx, int32_t batch, const int32_t *kv_lens, const
 int fc_debug_logits(fc_ctx *ctx, float *dev_logits);
 int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen);
 
-/* Enqueue `n_steps` iterations back to back without host round trips and without committing
- * (kv_len is restored before each step), returning the device time in milliseconds between the
- * first and the last kernel.  For latency measurement at a fixed K/V length. */
-int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, float *ms_total);
+/* Enqueue `n_steps` iterations back to back with no host round trip in between and return the
+ * device time in milliseconds from the first to the last kernel (CUDA events on the context's
+ * stream).  commit != 0: every step commits its accepted tokens on the device (needs
+ * kv_len + n_steps * c <= max_seq); host mirrors are refreshed afterwards and *tokens_out (nullable)
+ * gets the tokens committed over all sequences.  commit == 0: kv_len, n_gen and the window are left
+ * untouched, so every step runs at the same K/V length (latency sweeps). */
+int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, int32_t commit, float *ms_total, int64_t *tokens_out);
+
+/* One non-committing step with CUDA events around every launch.  ms_by_class / launches_by_class
+ * (host, FC_N_CLASSES entries each) receive device time and launch count per kernel class. */
+enum { FC_CLS_EMBED = 0, FC_CLS_QKV, FC_CLS_ROPE, FC_CLS_ATTN, FC_CLS_OPROJ, FC_CLS_GATEUP, FC_CLS_DOWN,
+       FC_CLS_HEAD, FC_CLS_ACCEPT, FC_N_CLASSES };
+int fc_profile_step(fc_ctx *ctx, float *ms_by_class, int32_t *launches_by_class);
 
 /* Number of kernels the most recent step / prefill / bench call launched. */
 int64_t fc_last_launch_count(const fc_ctx *ctx);

@@ -118,6 +118,10 @@ struct fc_ctx {
   int64_t launches = 0;
   char cuda_err[256] = {0};
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  // per-launch profiling (fc_profile_step)
+  bool prof = false;
+  std::vector<cudaEvent_t> prof_ev;
+  std::vector<int> prof_cls;
 };
 
 #define FC_CK(call)                                                                      \
@@ -280,7 +284,22 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   return FC_OK;
 }
 
-static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi) {
+static void prof_mark(fc_ctx *ctx, int cls, bool begin) {
+  if (!ctx->prof) return;
+  cudaEvent_t e;
+  if (cudaEventCreate(&e) != cudaSuccess) return;
+  cudaEventRecord(e, ctx->st);
+  ctx->prof_ev.push_back(e);
+  if (begin) ctx->prof_cls.push_back(cls);
+}
+struct ProfScope {
+  fc_ctx *c; int cls;
+  ProfScope(fc_ctx *ctx, int k) : c(ctx), cls(k) { prof_mark(c, cls, true); }
+  ~ProfScope() { prof_mark(c, cls, false); }
+};
+
+static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls) {
+  ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
   if (ctx->use_umma) return launch_gemm_umma(plan, a, ctx->st);
@@ -302,13 +321,13 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   ea.z.p[2] = ctx->b.ss_attn; ea.z.n[2] = Rz;
   ea.z.p[3] = ctx->b.ss_ffn; ea.z.n[3] = Rz;
   ++ctx->launches;
-  FC_CK(launch_embed(ea, s.dtype, ctx->st));
+  { ProfScope ps(ctx, FC_CLS_EMBED); FC_CK(launch_embed(ea, s.dtype, ctx->st)); }
 
   const int nsplit = (max_len_host + rows + d.tk - 1) / d.tk;
   const long long stride_h = (long long)s.max_seq * s.head_dim;
   const long long stride_b = (long long)s.n_kv_heads * stride_h;
   for (int l = 0; l < s.n_layers; ++l) {
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD));
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV));
     RopeArgs ra; memset(&ra, 0, sizeof ra);
     ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
     ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows;
@@ -320,7 +339,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     ra.z.p[0] = ctx->b.gu; ra.z.n[0] = Rz * 2 * s.d_ffn;
     ra.z.p[1] = ctx->b.ss_ffn; ra.z.n[1] = Rz;
     ++ctx->launches;
-    FC_CK(launch_rope_kv(ra, s.dtype, ctx->st));
+    { ProfScope ps(ctx, FC_CLS_ROPE); FC_CK(launch_rope_kv(ra, s.dtype, ctx->st)); }
     AttnArgs aa; memset(&aa, 0, sizeof aa);
     aa.q = ctx->b.qb; aa.kcache = ra.kcache; aa.vcache = ra.vcache; aa.stride_b = stride_b; aa.stride_h = stride_h;
     aa.kv_len = ctx->b.kv_len; aa.b0 = b0; aa.nb = nb; aa.c = rows; aa.hq = s.n_heads; aa.hkv = s.n_kv_heads;
@@ -328,15 +347,15 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     aa.out = ctx->b.attn;
     aa.z.p[0] = ctx->b.ss_attn; aa.z.n[0] = Rz;
     ++ctx->launches;
-    FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st));
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD));
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD));
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD));
+    { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st)); }
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ));
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP));
+    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN));
   }
   if (with_head) {
     GemmArgs ha = args_head(ctx);
     ha.tokens = tokens;
-    FC_CK(run_gemm(ctx, ctx->plan_head, ha, R, PRO_GAIN, EPI_ARGMAX));
+    FC_CK(run_gemm(ctx, ctx->plan_head, ha, R, PRO_GAIN, EPI_ARGMAX, FC_CLS_HEAD));
     AcceptArgs ac; memset(&ac, 0, sizeof ac);
     ac.window = ctx->b.window; ac.amax = ctx->b.amax; ac.amax_clear = ctx->b.amax;
     ac.kv_len = ctx->b.kv_len; ac.n_gen = ctx->b.n_gen; ac.done = ctx->b.done;
@@ -346,7 +365,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     ac.b0 = b0; ac.nb = nb; ac.c = rows; ac.p_stride = s.max_seq; ac.refill = ctx->refill; ac.pad_id = ctx->pad_id;
     ac.max_tokens = ctx->gen_max_tokens; ac.eos_id = ctx->gen_eos; ac.commit = commit;
     ++ctx->launches;
-    FC_CK(launch_accept(ac, ctx->st));
+    { ProfScope ps(ctx, FC_CLS_ACCEPT); FC_CK(launch_accept(ac, ctx->st)); }
   } else {
     for (int b = b0; b < b0 + nb; ++b) {
       ++ctx->launches;
@@ -568,21 +587,63 @@ extern "C" int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen) {
   return FC_OK;
 }
 
-extern "C" int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, float *ms_total) {
+extern "C" int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, int32_t commit, float *ms_total, int64_t *tokens_out) {
   if (!ctx || n_steps < 1 || !ms_total) return FC_ERR_ARG;
   if (!ctx->ready) return FC_ERR_STATE;
-  for (int b = 0; b < ctx->batch; ++b)
-    if (ctx->kv_len_h[b] + ctx->c > ctx->s.max_seq) return FC_ERR_CAPACITY;
+  const int B = ctx->batch, c = ctx->c;
+  const int growth = commit ? n_steps * c : c;
+  for (int b = 0; b < B; ++b)
+    if (ctx->kv_len_h[b] + growth > ctx->s.max_seq) return FC_ERR_CAPACITY;
   ctx->launches = 0;
   const int maxlen = max_live_len(ctx);
   FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
   for (int i = 0; i < n_steps; ++i) {
-    int rc = forward(ctx, 0, ctx->batch, ctx->c, ctx->b.window, true, maxlen, 0);
+    // committed steps grow the cache by at most c tokens each: size the split count for that bound
+    int rc = forward(ctx, 0, B, c, ctx->b.window, true, commit ? maxlen + i * c : maxlen, commit ? 1 : 0);
     if (rc != FC_OK) return rc;
   }
   FC_CK(cudaEventRecord(ctx->ev1, ctx->st));
   FC_CK(cudaEventSynchronize(ctx->ev1));
   FC_CK(cudaEventElapsedTime(ms_total, ctx->ev0, ctx->ev1));
+  if (tokens_out) *tokens_out = 0;
+  if (commit) {
+    int32_t *p_kv = ctx->pin, *p_ng = p_kv + B, *p_win = p_ng + B;   // pin holds B * (1 + 2c) + 4 ints
+    FC_CK(cudaMemcpyAsync(p_kv, ctx->b.kv_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, ctx->st));
+    FC_CK(cudaMemcpyAsync(p_ng, ctx->b.n_gen, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, ctx->st));
+    FC_CK(cudaMemcpyAsync(p_win, ctx->b.window, sizeof(int32_t) * B * c, cudaMemcpyDeviceToHost, ctx->st));
+    FC_CK(cudaStreamSynchronize(ctx->st));
+    for (int b = 0; b < B; ++b) {
+      if (tokens_out) *tokens_out += p_ng[b] - ctx->n_gen_h[b];
+      ctx->kv_len_h[b] = p_kv[b]; ctx->n_gen_h[b] = p_ng[b]; ctx->pending_h[b] = p_win[(size_t)b * c];
+    }
+  }
+  return check_device_error(ctx);
+}
+
+extern "C" int fc_profile_step(fc_ctx *ctx, float *ms_by_class, int32_t *launches_by_class) {
+  if (!ctx || !ms_by_class || !launches_by_class) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  for (int b = 0; b < ctx->batch; ++b)
+    if (ctx->kv_len_h[b] + ctx->c > ctx->s.max_seq) return FC_ERR_CAPACITY;
+  for (int i = 0; i < FC_N_CLASSES; ++i) { ms_by_class[i] = 0.f; launches_by_class[i] = 0; }
+  ctx->prof = true; ctx->prof_ev.clear(); ctx->prof_cls.clear();
+  ctx->launches = 0;
+  int rc = forward(ctx, 0, ctx->batch, ctx->c, ctx->b.window, true, max_live_len(ctx), 0);
+  ctx->prof = false;
+  cudaError_t e = cudaStreamSynchronize(ctx->st);
+  if (rc == FC_OK && e == cudaSuccess) {
+    for (size_t i = 0; i < ctx->prof_cls.size() && 2 * i + 1 < ctx->prof_ev.size(); ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]) == cudaSuccess) {
+        ms_by_class[ctx->prof_cls[i]] += ms;
+        launches_by_class[ctx->prof_cls[i]] += 1;
+      }
+    }
+  }
+  for (cudaEvent_t ev : ctx->prof_ev) cudaEventDestroy(ev);
+  ctx->prof_ev.clear(); ctx->prof_cls.clear();
+  if (rc != FC_OK) return rc;
+  if (e != cudaSuccess) { snprintf(ctx->cuda_err, sizeof ctx->cuda_err, "%s", cudaGetErrorString(e)); return FC_ERR_CUDA; }
   return check_device_error(ctx);
 }
 

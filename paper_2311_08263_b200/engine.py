@@ -136,10 +136,19 @@ class Decoder:
         self._check(self.lib.fc_get_state(self.h, kl.ctypes.data, ng.ctypes.data), "fc_get_state")
         return kl, ng
 
-    def fc_bench_steps(self, n_steps: int) -> float:
-        ms = C.c_float(0)
-        self._check(self.lib.fc_bench_steps(self.h, n_steps, C.byref(ms)), "fc_bench_steps")
-        return float(ms.value)
+    def fc_bench_steps(self, n_steps: int, commit: bool = False):
+        """Returns (device milliseconds for n_steps back-to-back steps, tokens committed)."""
+        ms, tok = C.c_float(0), C.c_int64(0)
+        self._check(self.lib.fc_bench_steps(self.h, n_steps, int(commit), C.byref(ms), C.byref(tok)),
+                    "fc_bench_steps")
+        return float(ms.value), int(tok.value)
+
+    def fc_profile_step(self):
+        """Returns {class name: (milliseconds, launches)} for one non-committing step."""
+        n = len(_l.FC_CLASSES)
+        ms, cnt = (C.c_float * n)(), (C.c_int32 * n)()
+        self._check(self.lib.fc_profile_step(self.h, ms, cnt), "fc_profile_step")
+        return {name: (float(ms[i]), int(cnt[i])) for i, name in enumerate(_l.FC_CLASSES)}
 
     def fc_last_launch_count(self) -> int:
         return int(self.lib.fc_last_launch_count(self.h))

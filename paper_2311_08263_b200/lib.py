@@ -15,11 +15,12 @@ FC_F32, FC_BF16 = 0, 1
 FC_REFILL_PROMPT_CYCLE, FC_REFILL_PAD = 0, 1
 FC_FLAG_SIMT_GEMM, FC_FLAG_NO_GRAPH = 1, 2
 FC_OK = 0
+FC_CLASSES = ["embed", "qkv", "rope", "attn", "oproj", "gateup", "down", "head", "accept"]
 FC_ERR_ARG, FC_ERR_SHAPE, FC_ERR_CAPACITY, FC_ERR_TOKEN_RANGE = -1, -2, -3, -4
 FC_ERR_STATE, FC_ERR_BAD_WINDOW, FC_ERR_DEVICE_TIMEOUT, FC_ERR_CUDA = -5, -6, -7, -8
 
 EXPORTS = ["fc_kv_bytes", "fc_workspace_bytes", "fc_init", "fc_prefill", "fc_jacobi_step", "fc_generate",
-           "fc_debug_set_state", "fc_debug_logits", "fc_get_state", "fc_bench_steps",
+           "fc_debug_set_state", "fc_debug_logits", "fc_get_state", "fc_bench_steps", "fc_profile_step",
            "fc_last_launch_count", "fc_destroy", "fc_strerror", "fc_last_cuda_error",
            "fc_op_linear", "fc_op_accept"]
 
@@ -71,7 +72,8 @@ def load() -> C.CDLL:
     lib.fc_debug_set_state.argtypes = [vp, i32, i32p, i32p, i32, i32]
     lib.fc_debug_logits.argtypes = [vp, vp]
     lib.fc_get_state.argtypes = [vp, i32p, i32p]
-    lib.fc_bench_steps.argtypes = [vp, i32, C.POINTER(C.c_float)]
+    lib.fc_bench_steps.argtypes = [vp, i32, i32, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+    lib.fc_profile_step.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
     lib.fc_last_launch_count.restype = C.c_int64
     lib.fc_last_launch_count.argtypes = [vp]
     lib.fc_destroy.restype = None
