@@ -156,6 +156,21 @@ int fc_op_accept(int32_t *window, const int32_t *argmax, int32_t *kv_len, int32_
                  const int32_t *prompt_lens, int32_t batch, int32_t c, int32_t p_stride,
                  int32_t refill, int32_t pad_id, void *cuda_stream);
 
+/* Window attention of one layer (the attention inside Eq. 4's single causal forward): for sequence b,
+ * window row j and query head h, softmax over keys 0 .. kv_len[b] + j of q.k / sqrt(head_dim), times V;
+ * kv head = h / (n_heads / n_kv_heads).  q: [batch*c, n_heads*head_dim], kcache/vcache:
+ * [batch][n_kv_heads][max_seq][head_dim], all in `dtype`, rotary embedding already applied, the window's
+ * own K/V already stored at slots kv_len[b] .. kv_len[b]+c-1.  kv_len: device [batch]; max_len: host upper
+ * bound on kv_len[b].  out: fp32 [batch*c, n_heads*head_dim].  scratch: device, at least
+ * fc_op_window_attention_scratch_bytes(...) bytes, 256-byte aligned; it holds the per-split partial
+ * results and is cleared as needed by the call. */
+size_t fc_op_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
+                                            int32_t head_dim, int32_t max_len, int32_t dtype);
+int fc_op_window_attention(const void *q, const void *kcache, const void *vcache, const int32_t *kv_len,
+                           float *out, int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
+                           int32_t head_dim, int32_t max_seq, int32_t max_len, int32_t dtype,
+                           void *scratch, size_t scratch_bytes, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

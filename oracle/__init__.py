@@ -52,6 +52,7 @@ def _load():
         lib.orc_kv_len.argtypes = [C.c_void_p]
         lib.orc_n_gen.argtypes = [C.c_void_p]
         lib.orc_set_kv.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
+        lib.orc_get_kv.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
         lib.orc_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         lib.orc_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int]
         lib.orc_jacobi_step.argtypes = [C.c_void_p] + [C.c_void_p] * 5
@@ -160,6 +161,13 @@ class Oracle:
         v = np.ascontiguousarray(v, dtype=np.float32)
         rc = self._lib.orc_set_kv(self._h, layer, k.ctypes.data, v.ctypes.data, k.shape[0])
         assert rc == 0, rc
+
+    def get_kv(self, layer: int, length: int):
+        kvd = self.cfg.n_kv_heads * self.cfg.head_dim
+        k, v = np.empty((length, kvd), np.float32), np.empty((length, kvd), np.float32)
+        rc = self._lib.orc_get_kv(self._h, layer, k.ctypes.data, v.ctypes.data, length)
+        assert rc == 0, rc
+        return k, v
 
     def forward(self, tokens, want_logits: bool = True, trace: bool = False):
         """Forward rows at positions kv_len.. without committing.  Returns (argmax, logits[, trace])."""

@@ -412,3 +412,13 @@ int orc_ar_generate(orc *o, const int32_t *prompt, int P, int max_tokens, int eo
   free(lg);
   return n;
 }
+
+/* Copy out the first `len` cached tokens of one layer ([len, n_kv_heads*head_dim] each). */
+int orc_get_kv(const orc *o, int layer, float *k, float *v, int len) {
+  const orc_shape *s = &o->s;
+  size_t kvd = (size_t)s->n_kv_heads * s->head_dim;
+  if (layer < 0 || layer >= s->n_layers || len < 0 || len > s->max_seq) return -1;
+  memcpy(k, o->kcache + (size_t)layer * s->max_seq * kvd, sizeof(float) * len * kvd);
+  memcpy(v, o->vcache + (size_t)layer * s->max_seq * kvd, sizeof(float) * len * kvd);
+  return 0;
+}

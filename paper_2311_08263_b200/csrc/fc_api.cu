@@ -696,3 +696,58 @@ extern "C" int fc_op_accept(int32_t *window, const int32_t *argmax, int32_t *kv_
   if (launch_accept(ac, st) != cudaSuccess) return FC_ERR_CUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------------------------ window attention op
+namespace fc {
+static bool attn_shape_ok(int batch, int c, int hq, int hkv, int hd, int max_len, int dtype) {
+  return batch >= 1 && c >= 1 && hq >= 1 && hkv >= 1 && hq % hkv == 0 && (hd == 32 || hd == 64 || hd == 128) &&
+         max_len >= 0 && (dtype == FC_F32 || dtype == FC_BF16);
+}
+
+size_t window_attention_scratch_bytes(int batch, int c, int hq, int hkv, int hd, int max_len, int dtype) {
+  if (!attn_shape_ok(batch, c, hq, hkv, hd, max_len, dtype)) return 0;
+  const size_t nsplit = (size_t)(max_len + c + attn_tile_keys(dtype, hd) - 1) / attn_tile_keys(dtype, hd);
+  const size_t rows = (size_t)batch * c * hq;
+  return align_up(rows * nsplit * hd * sizeof(float)) + align_up(rows * nsplit * 2 * sizeof(float)) +
+         align_up((size_t)batch * hkv * sizeof(unsigned int));
+}
+
+int run_window_attention(const void *q, const void *kcache, const void *vcache, const int32_t *kv_len, float *out,
+                         int batch, int c, int hq, int hkv, int hd, int max_seq, int max_len, int dtype,
+                         void *scratch, size_t scratch_bytes, cudaStream_t st) {
+  if (!q || !kcache || !vcache || !kv_len || !out || !scratch) return FC_ERR_ARG;
+  if (!attn_shape_ok(batch, c, hq, hkv, hd, max_len, dtype)) return FC_ERR_ARG;
+  if (max_len + c > max_seq) return FC_ERR_CAPACITY;
+  if ((uintptr_t)scratch % kAlign) return FC_ERR_ARG;
+  if (scratch_bytes < window_attention_scratch_bytes(batch, c, hq, hkv, hd, max_len, dtype)) return FC_ERR_CAPACITY;
+  const int tk = attn_tile_keys(dtype, hd);
+  const size_t nsplit = (size_t)(max_len + c + tk - 1) / tk;
+  const size_t rows = (size_t)batch * c * hq;
+  char *p = (char *)scratch;
+  AttnArgs aa; memset(&aa, 0, sizeof aa);
+  aa.part_o = (float *)p; p += align_up(rows * nsplit * hd * sizeof(float));
+  aa.part_ml = (float *)p; p += align_up(rows * nsplit * 2 * sizeof(float));
+  aa.counters = (unsigned int *)p;
+  // the arrival counters must start at zero; the partial results are fully overwritten
+  if (cudaMemsetAsync(aa.counters, 0, (size_t)batch * hkv * sizeof(unsigned int), st) != cudaSuccess) return FC_ERR_CUDA;
+  aa.q = q; aa.kcache = kcache; aa.vcache = vcache;
+  aa.stride_h = (long long)max_seq * hd; aa.stride_b = (long long)hkv * aa.stride_h;
+  aa.kv_len = kv_len; aa.b0 = 0; aa.nb = batch; aa.c = c; aa.hq = hq; aa.hkv = hkv;
+  aa.nsplit = (int)nsplit; aa.out = out;
+  if (launch_attn(aa, dtype, hd, st) != cudaSuccess) return FC_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+}
+}  // namespace fc
+
+extern "C" size_t fc_op_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
+                                                       int32_t head_dim, int32_t max_len, int32_t dtype) {
+  return window_attention_scratch_bytes(batch, c, n_heads, n_kv_heads, head_dim, max_len, dtype);
+}
+
+extern "C" int fc_op_window_attention(const void *q, const void *kcache, const void *vcache, const int32_t *kv_len,
+                                      float *out, int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
+                                      int32_t head_dim, int32_t max_seq, int32_t max_len, int32_t dtype,
+                                      void *scratch, size_t scratch_bytes, void *cuda_stream) {
+  return run_window_attention(q, kcache, vcache, kv_len, out, batch, c, n_heads, n_kv_heads, head_dim, max_seq,
+                              max_len, dtype, scratch, scratch_bytes, (cudaStream_t)cuda_stream);
+}

@@ -113,6 +113,12 @@ cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st);
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 int attn_tile_keys(int dtype, int hd);   // keys per split tile
 
+// Standalone window attention on caller-supplied scratch (shared by the op-level entry points).
+size_t window_attention_scratch_bytes(int batch, int c, int hq, int hkv, int hd, int max_len, int dtype);
+int run_window_attention(const void *q, const void *kcache, const void *vcache, const int32_t *kv_len, float *out,
+                         int batch, int c, int hq, int hkv, int hd, int max_seq, int max_len, int dtype,
+                         void *scratch, size_t scratch_bytes, cudaStream_t st);
+
 // tcgen05 path (bf16 only).  `maps` points at prebuilt tensor maps for the weight matrices.
 struct UmmaPlan;
 UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsigned int *err_word,

@@ -187,3 +187,21 @@ def fc_op_accept(window, argmax, kv_len, n_gen, prompt, prompt_lens, refill: int
     if rc != _l.FC_OK:
         raise FcError(rc, "fc_op_accept")
     return cnt, tok
+
+
+def fc_op_window_attention(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.Tensor, kv_len: torch.Tensor,
+                           c: int, n_heads: int, max_len: int) -> torch.Tensor:
+    """Window attention of one layer.  q [B*c, n_heads*hd]; kcache/vcache [B, n_kv_heads, max_seq, hd];
+    kv_len int32 [B] on the device.  Returns fp32 [B*c, n_heads*hd]."""
+    lib = _l.load()
+    B, hkv, max_seq, hd = kcache.shape
+    dt = _l.FC_F32 if q.dtype == torch.float32 else _l.FC_BF16
+    nbytes = lib.fc_op_window_attention_scratch_bytes(B, c, n_heads, hkv, hd, max_len, dt)
+    scratch = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=q.device)
+    out = torch.empty(B * c, n_heads * hd, dtype=torch.float32, device=q.device)
+    rc = lib.fc_op_window_attention(q.data_ptr(), kcache.data_ptr(), vcache.data_ptr(), kv_len.data_ptr(),
+                                    out.data_ptr(), B, c, n_heads, hkv, hd, max_seq, max_len, dt,
+                                    scratch.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
+    if rc != _l.FC_OK:
+        raise FcError(rc, "fc_op_window_attention")
+    return out

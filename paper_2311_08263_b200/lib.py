@@ -22,7 +22,8 @@ FC_ERR_STATE, FC_ERR_BAD_WINDOW, FC_ERR_DEVICE_TIMEOUT, FC_ERR_CUDA = -5, -6, -7
 EXPORTS = ["fc_kv_bytes", "fc_workspace_bytes", "fc_init", "fc_prefill", "fc_jacobi_step", "fc_generate",
            "fc_debug_set_state", "fc_debug_logits", "fc_get_state", "fc_bench_steps", "fc_profile_step",
            "fc_last_launch_count", "fc_destroy", "fc_strerror", "fc_last_cuda_error",
-           "fc_op_linear", "fc_op_accept"]
+           "fc_op_linear", "fc_op_accept", "fc_op_window_attention",
+           "fc_op_window_attention_scratch_bytes"]
 
 
 class fc_model_shape(C.Structure):
@@ -84,5 +85,8 @@ def load() -> C.CDLL:
     lib.fc_last_cuda_error.argtypes = [vp]
     lib.fc_op_linear.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
     lib.fc_op_accept.argtypes = [vp] * 8 + [i32] * 5 + [vp]
+    lib.fc_op_window_attention_scratch_bytes.restype = C.c_size_t
+    lib.fc_op_window_attention_scratch_bytes.argtypes = [i32] * 7
+    lib.fc_op_window_attention.argtypes = [vp] * 5 + [i32] * 8 + [vp, C.c_size_t, vp]
     _lib = lib
     return lib

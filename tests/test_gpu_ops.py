@@ -94,3 +94,46 @@ def test_accept_kernel_bit_exact(c, refill):
         assert tok[b, :k].tolist() == acc.tolist()
         assert wnew[b].tolist() == w2.tolist()
         assert kd[b].item() == kv_len[b] + k and nd[b].item() == n_gen[b] + k
+
+
+def _oracle_attention_case(cfg, lens, c):
+    """Per sequence: prefill `len` tokens on the oracle, forward a random window with tracing, and
+    return the layer-0 rotated queries, the layer-0 K/V cache (committed + window rows) and the
+    oracle's attention output."""
+    w = wl.make_weights(cfg)
+    qs, wants, ks, vs = [], [], [], []
+    for b, L in enumerate(lens):
+        ids = wl.hash_uniform_int(cfg.seed + b, 5, L + 1, cfg.vocab).numpy()
+        o = oracle.Oracle(cfg, w, L + c + 4)
+        o.prefill(ids, c)
+        win = wl.hash_uniform_int(cfg.seed + 100 + b, 7, c, cfg.vocab).numpy()
+        _, _, tr = o.forward(win, want_logits=True, trace=True)
+        k, v = o.get_kv(0, L + c)
+        qs.append(tr["q"]); wants.append(tr["attn"]); ks.append(k); vs.append(v)
+    return qs, wants, ks, vs
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("hq,hkv,hd,c,lens", [
+    (4, 4, 32, 8, [300, 129, 0, 517]),       # MHA, several key tiles, an empty cache, ragged lengths
+    (8, 2, 64, 5, [260, 1]),                 # GQA, odd window size
+    (2, 2, 128, 16, [200]),                  # head_dim 128
+    (4, 1, 64, 1, [77, 130]),                # c = 1: plain autoregressive attention
+])
+def test_window_attention_vs_oracle(dtype, hq, hkv, hd, c, lens):
+    cfg = wl.small_config(dtype="f32", n_layers=1, d_model=128, n_heads=hq, n_kv_heads=hkv, head_dim=hd,
+                          d_ffn=128, vocab=300, seed=91)
+    qs, wants, ks, vs = _oracle_attention_case(cfg, lens, c)
+    B, max_seq = len(lens), max(lens) + c + 3
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    kc = torch.zeros(B, hkv, max_seq, hd)
+    vc = torch.zeros(B, hkv, max_seq, hd)
+    for b, L in enumerate(lens):
+        kc[b, :, :L + c] = torch.from_numpy(ks[b]).view(L + c, hkv, hd).transpose(0, 1)
+        vc[b, :, :L + c] = torch.from_numpy(vs[b]).view(L + c, hkv, hd).transpose(0, 1)
+    q = torch.from_numpy(np.concatenate(qs)).to(tdt).cuda()
+    out = engine.fc_op_window_attention(q, kc.to(tdt).cuda().contiguous(), vc.to(tdt).cuda().contiguous(),
+                                        torch.tensor(lens, dtype=torch.int32).cuda(), c, hq, max(lens))
+    want = np.concatenate(wants)
+    tol = 2e-5 if dtype == "f32" else 2e-2 * max(1.0, float(np.abs(want).max()))
+    assert np.abs(out.cpu().numpy() - want).max() < tol
