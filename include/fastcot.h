@@ -171,6 +171,24 @@ int fc_op_window_attention(const void *q, const void *kcache, const void *vcache
                            int32_t head_dim, int32_t max_seq, int32_t max_len, int32_t dtype,
                            void *scratch, size_t scratch_bytes, void *cuda_stream);
 
+/* The same window attention for callers that may not allocate device memory (the paper has no
+ * counterpart; this exists for hosts whose device memory is owned by someone else, e.g. a serving
+ * process with a fixed arena, or code that must stay out of the CUDA allocator after start-up).
+ * Scratch is a fixed FC_NOALLOC_SCRATCH_BYTES array built into the library - every GPU that loads the
+ * library holds it until the process exits - so only inputs and outputs are passed; arguments are
+ * those of fc_op_window_attention.  Problems whose scratch need (fc_op_window_attention_scratch_bytes)
+ * exceeds the array are refused with FC_ERR_CAPACITY and a message on stderr.  The call makes no
+ * cudaMalloc/cudaFree and uses no allocating library routine.  The first call on each device looks up
+ * the array's device address (cudaGetSymbolAddress) with that device current; make that first call
+ * before starting any stream capture.  All calls on a device share the one array, which keeps
+ * whatever the previous call left in it (the call clears the part that must start at zero): two calls
+ * that overlap on the GPU - different streams or threads - race on it; serialise them. */
+#define FC_NOALLOC_SCRATCH_BYTES (8u << 20)
+int fc_op_window_attention_noalloc(const void *q, const void *kcache, const void *vcache,
+                                   const int32_t *kv_len, float *out, int32_t batch, int32_t c,
+                                   int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_seq,
+                                   int32_t max_len, int32_t dtype, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -15,6 +15,7 @@ FC_F32, FC_BF16 = 0, 1
 FC_REFILL_PROMPT_CYCLE, FC_REFILL_PAD = 0, 1
 FC_FLAG_SIMT_GEMM, FC_FLAG_NO_GRAPH = 1, 2
 FC_OK = 0
+FC_NOALLOC_SCRATCH_BYTES = 8 << 20
 FC_CLASSES = ["embed", "qkv", "rope", "attn", "oproj", "gateup", "down", "head", "accept"]
 FC_ERR_ARG, FC_ERR_SHAPE, FC_ERR_CAPACITY, FC_ERR_TOKEN_RANGE = -1, -2, -3, -4
 FC_ERR_STATE, FC_ERR_BAD_WINDOW, FC_ERR_DEVICE_TIMEOUT, FC_ERR_CUDA = -5, -6, -7, -8
@@ -23,7 +24,7 @@ EXPORTS = ["fc_kv_bytes", "fc_workspace_bytes", "fc_init", "fc_prefill", "fc_jac
            "fc_debug_set_state", "fc_debug_logits", "fc_get_state", "fc_bench_steps", "fc_profile_step",
            "fc_last_launch_count", "fc_destroy", "fc_strerror", "fc_last_cuda_error",
            "fc_op_linear", "fc_op_accept", "fc_op_window_attention",
-           "fc_op_window_attention_scratch_bytes"]
+           "fc_op_window_attention_scratch_bytes", "fc_op_window_attention_noalloc"]
 
 
 class fc_model_shape(C.Structure):
@@ -88,5 +89,6 @@ def load() -> C.CDLL:
     lib.fc_op_window_attention_scratch_bytes.restype = C.c_size_t
     lib.fc_op_window_attention_scratch_bytes.argtypes = [i32] * 7
     lib.fc_op_window_attention.argtypes = [vp] * 5 + [i32] * 8 + [vp, C.c_size_t, vp]
+    lib.fc_op_window_attention_noalloc.argtypes = [vp] * 5 + [i32] * 8 + [vp]
     _lib = lib
     return lib
