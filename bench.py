@@ -226,9 +226,6 @@ def run_ours(args, cfg, rank, world, local):
     torch.cuda.synchronize()
     barrier(world)
     kv1 = dec.fc_get_state()[0].copy()
-    # keep the GPU under the same load while nvidia-smi catches a few more samples
-    if ms < 1500:
-        dec.fc_bench_steps(max(1, int(steps * 1500 / max(ms, 1))), commit=False)
     clocks = sampler.stop()
     ms_max, tok_sum = reduce_max_sum(world, ms, tokens, device)
 
@@ -306,15 +303,20 @@ def run_ours(args, cfg, rank, world, local):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="7b", choices=sorted(wl.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: keep only the first N layers (same kernel shapes, less device memory)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     cfg = wl.CONFIGS[args.workload]
+    if args.layers > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, n_layers=args.layers, name=f"{cfg.name}-first{args.layers}layers")
     rank, world, local = dist_setup(args.gpus)
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
