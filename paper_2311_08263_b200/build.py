@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libfastcot.so")
-SOURCES = ["fc_api.cu", "k_simt.cu", "k_umma.cu", "fc_noalloc.cu"]
+SOURCES = ["fc_api.cu", "k_simt.cu", "k_umma.cu", "k_attn.cu", "fc_noalloc.cu"]
 
 
 def _stale() -> bool:

@@ -73,7 +73,7 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
   t.ss_ffn = c.take<float>(R);
   t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
   t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
-  t.counters = c.take<unsigned int>((size_t)s->max_batch * s->n_kv_heads);
+  t.counters = c.take<unsigned int>((size_t)s->max_batch * s->n_kv_heads + 1);   // + one grid-wide word
   t.err = c.take<unsigned int>(1);
   t.amax = c.take<unsigned long long>(R);
   t.window = c.take<int32_t>(R);
@@ -104,6 +104,7 @@ struct fc_ctx {
   char *kv; size_t kv_layer_stride, kv_half_stride;   // bytes
   cudaStream_t st;
   bool use_umma;
+  bool fused_attn;   // bf16 with head_dim 64/128: rotary embedding and K/V write happen inside the attention kernel
   int n_sms;
   std::vector<UmmaPlan *> plan_qkv, plan_o, plan_gu, plan_down;
   UmmaPlan *plan_head = nullptr;
@@ -252,6 +253,8 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   ctx->kv_layer_stride = 2 * ctx->kv_half_stride;
   ctx->st = (cudaStream_t)cuda_stream;
   ctx->use_umma = shape->dtype == FC_BF16 && !(shape->flags & FC_FLAG_SIMT_GEMM);
+  ctx->fused_attn = shape->dtype == FC_BF16 && (shape->head_dim == 64 || shape->head_dim == 128) &&
+                    !(shape->flags & FC_FLAG_SIMT_GEMM);
 
   int rc = FC_OK;
   auto fail = [&](int code) { fc_destroy(ctx); return code; };
@@ -328,26 +331,40 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   const long long stride_b = (long long)s.n_kv_heads * stride_h;
   for (int l = 0; l < s.n_layers; ++l) {
     FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV));
-    RopeArgs ra; memset(&ra, 0, sizeof ra);
-    ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
-    ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows;
-    ra.hq = s.n_heads; ra.hkv = s.n_kv_heads; ra.hd = s.head_dim; ra.theta = s.rope_theta;
-    ra.q_out = ctx->b.qb;
-    ra.kcache = ctx->kv + (size_t)l * ctx->kv_layer_stride;
-    ra.vcache = ctx->kv + (size_t)l * ctx->kv_layer_stride + ctx->kv_half_stride;
-    ra.stride_b = stride_b; ra.stride_h = stride_h;
-    ra.z.p[0] = ctx->b.gu; ra.z.n[0] = Rz * 2 * s.d_ffn;
-    ra.z.p[1] = ctx->b.ss_ffn; ra.z.n[1] = Rz;
-    ++ctx->launches;
-    { ProfScope ps(ctx, FC_CLS_ROPE); FC_CK(launch_rope_kv(ra, s.dtype, ctx->st)); }
-    AttnArgs aa; memset(&aa, 0, sizeof aa);
-    aa.q = ctx->b.qb; aa.kcache = ra.kcache; aa.vcache = ra.vcache; aa.stride_b = stride_b; aa.stride_h = stride_h;
-    aa.kv_len = ctx->b.kv_len; aa.b0 = b0; aa.nb = nb; aa.c = rows; aa.hq = s.n_heads; aa.hkv = s.n_kv_heads;
-    aa.nsplit = nsplit; aa.part_o = ctx->b.part_o; aa.part_ml = ctx->b.part_ml; aa.counters = ctx->b.counters;
-    aa.out = ctx->b.attn;
-    aa.z.p[0] = ctx->b.ss_attn; aa.z.n[0] = Rz;
-    ++ctx->launches;
-    { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st)); }
+    void *kc = ctx->kv + (size_t)l * ctx->kv_layer_stride;
+    void *vc = ctx->kv + (size_t)l * ctx->kv_layer_stride + ctx->kv_half_stride;
+    if (ctx->fused_attn) {
+      FusedAttnArgs fa; memset(&fa, 0, sizeof fa);
+      fa.qkv = ctx->b.qkv; fa.ldq = d.ldq; fa.ss = ctx->b.ss_attn; fa.eps = s.rms_eps; fa.dn = s.d_model;
+      fa.theta = s.rope_theta; fa.kcache = kc; fa.vcache = vc; fa.stride_b = stride_b; fa.stride_h = stride_h;
+      fa.kv_len = ctx->b.kv_len; fa.b0 = b0; fa.nb = nb; fa.c = rows; fa.hq = s.n_heads; fa.hkv = s.n_kv_heads;
+      fa.nsplit = nsplit; fa.part_o = ctx->b.part_o; fa.part_ml = ctx->b.part_ml; fa.counters = ctx->b.counters;
+      fa.grid_counter = ctx->b.counters + (size_t)s.max_batch * s.n_kv_heads;
+      fa.out = ctx->b.attn;
+      fa.z.p[0] = ctx->b.gu; fa.z.n[0] = Rz * 2 * s.d_ffn;
+      fa.z.p[1] = ctx->b.ss_ffn; fa.z.n[1] = Rz;
+      ++ctx->launches;
+      { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn_fused(fa, s.head_dim, ctx->st)); }
+    } else {
+      RopeArgs ra; memset(&ra, 0, sizeof ra);
+      ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
+      ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows;
+      ra.hq = s.n_heads; ra.hkv = s.n_kv_heads; ra.hd = s.head_dim; ra.theta = s.rope_theta;
+      ra.q_out = ctx->b.qb; ra.kcache = kc; ra.vcache = vc;
+      ra.stride_b = stride_b; ra.stride_h = stride_h;
+      ra.z.p[0] = ctx->b.gu; ra.z.n[0] = Rz * 2 * s.d_ffn;
+      ra.z.p[1] = ctx->b.ss_ffn; ra.z.n[1] = Rz;
+      ++ctx->launches;
+      { ProfScope ps(ctx, FC_CLS_ROPE); FC_CK(launch_rope_kv(ra, s.dtype, ctx->st)); }
+      AttnArgs aa; memset(&aa, 0, sizeof aa);
+      aa.q = ctx->b.qb; aa.kcache = kc; aa.vcache = vc; aa.stride_b = stride_b; aa.stride_h = stride_h;
+      aa.kv_len = ctx->b.kv_len; aa.b0 = b0; aa.nb = nb; aa.c = rows; aa.hq = s.n_heads; aa.hkv = s.n_kv_heads;
+      aa.nsplit = nsplit; aa.part_o = ctx->b.part_o; aa.part_ml = ctx->b.part_ml; aa.counters = ctx->b.counters;
+      aa.out = ctx->b.attn;
+      aa.z.p[0] = ctx->b.ss_attn; aa.z.n[0] = Rz;
+      ++ctx->launches;
+      { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st)); }
+    }
     FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ));
     FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP));
     FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN));

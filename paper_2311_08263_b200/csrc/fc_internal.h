@@ -82,6 +82,24 @@ struct AttnArgs {
   ZeroList z;
 };
 
+struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attention in one kernel
+  float *qkv;             // [R, ldq] fp32 accumulators (q | k | v) lacking 1/rms; cleared by the kernel
+  int ldq;
+  float *ss;              // [R] sums of squares for 1/rms; cleared by the kernel
+  float eps; int dn;
+  float theta;
+  void *kcache, *vcache;
+  long long stride_b, stride_h;
+  const int32_t *kv_len;
+  int b0, nb, c, hq, hkv;
+  int nsplit;             // 128-key chunks covering max(kv_len) + c
+  float *part_o, *part_ml;
+  unsigned int *counters; // [batch*hkv], zero on entry and on exit
+  unsigned int *grid_counter;   // one word, zero on entry and on exit
+  float *out;             // [R, hq*hd] fp32
+  ZeroList z;
+};
+
 struct AcceptArgs {
   int32_t *window;                 // [batch, c] in/out
   const unsigned long long *amax;  // packed argmax per row, or null
@@ -110,6 +128,7 @@ cudaError_t launch_embed(const EmbedArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_gemm_simt(const GemmArgs &a, int dtype, int pro, int epi, cudaStream_t st);
 cudaError_t launch_rope_kv(const RopeArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st);
+cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st);
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 int attn_tile_keys(int dtype, int hd);   // keys per split tile
 

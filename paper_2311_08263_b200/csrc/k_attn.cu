@@ -1,0 +1,350 @@
+// Fused rotary embedding + in-place K/V write + split-KV window attention for bf16 (head_dim 64/128).
+//
+// grid (splits, kv heads, sequences); one CTA owns one 128-key chunk of one kv head of one sequence.
+// It stages the chunk's K and V in shared memory - cached keys by 16-byte copies; the window's own keys
+// (slots kv_len .. kv_len+c-1) straight from the fp32 QKV accumulators with the deferred 1/rms factor and
+// the rotation applied, writing them to the cache on the way (each window key has exactly one owner CTA).
+// Then, for every 16-row tile of the queries that map to this kv head (group heads x c window rows), the
+// four warps each take 32 keys: S = Q.K^T and P.V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate),
+// softmax statistics by warp shuffles, the four warps are merged through shared memory and one partial
+// (max, sum, out) per (row, head, split) goes to scratch.  The last CTA of a (sequence, kv head) merges the
+// splits and clears the accumulators it owns; the last CTA of the grid clears the per-row sums of squares.
+// Row j of sequence b sees keys 0 .. kv_len[b] + j (cache + causal part of the window).
+#include "fc_internal.h"
+
+namespace fc {
+
+namespace {
+
+constexpr int kChunk = 128;      // keys per CTA
+constexpr int kAttnThreads = 128;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+}  // namespace
+
+template <int HD>
+__global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs a) {
+  constexpr int LD = HD + 8;                 // padded row (elements): ldmatrix rows land in distinct banks
+  constexpr int HALF = HD / 2;
+  constexpr int ND = HD / 8;                 // 8-wide output blocks
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __nv_bfloat16 *Ks = reinterpret_cast<__nv_bfloat16 *>(smem_raw);       // [kChunk][LD]
+  __nv_bfloat16 *Vs = Ks + kChunk * LD;                                  // [kChunk][LD]
+  __nv_bfloat16 *Qs = Vs + kChunk * LD;                                  // [16][LD]
+  float *Om = reinterpret_cast<float *>(Qs + 16 * LD);                   // [4][16][HD]
+  float *mls = Om + 4 * 16 * HD;                                         // [4][16][2]
+  float *inv_freq = mls + 4 * 16 * 2;                                    // [HALF]
+  __shared__ unsigned int s_last, s_last_grid;
+
+  const int split = blockIdx.x, kvh = blockIdx.y, bl = blockIdx.z;
+  const int b = a.b0 + bl;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int L = a.kv_len[b];
+  const int ltot = L + a.c;
+  const int k0 = split * kChunk;
+  const int nk = min(kChunk, ltot - k0);                     // <= 0 for surplus splits
+  const int group = a.hq / a.hkv;
+  const int nq = group * a.c;
+  const int qd = a.hq * HD, kvd = a.hkv * HD;
+  __nv_bfloat16 *kbase = (__nv_bfloat16 *)a.kcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+  __nv_bfloat16 *vbase = (__nv_bfloat16 *)a.vcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+
+  // side clearing of buffers nobody reads during this kernel
+  {
+    const unsigned long long gtid =
+        ((unsigned long long)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * blockDim.x + tid;
+    const unsigned long long nth = (unsigned long long)gridDim.x * gridDim.y * gridDim.z * blockDim.x;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (a.z.p[i]) for (unsigned long long e = gtid; e < a.z.n[i]; e += nth) a.z.p[i][e] = 0.f;
+  }
+
+  for (int i = tid; i < HALF; i += kAttnThreads) inv_freq[i] = powf(a.theta, -2.0f * (float)i / (float)HD);
+  __syncthreads();
+
+  if (nk > 0) {
+    // ---- cached keys: 16-byte copies
+    const int n_cached = min(nk, max(0, L - k0));
+    constexpr int CPR = HD / 8;                              // 16-byte pieces per row
+    for (int e = tid; e < n_cached * CPR; e += kAttnThreads) {
+      const int t = e / CPR, p = e % CPR;
+      cp_async16(smem_addr(Ks + t * LD + p * 8), kbase + (long long)(k0 + t) * HD + p * 8);
+      cp_async16(smem_addr(Vs + t * LD + p * 8), vbase + (long long)(k0 + t) * HD + p * 8);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    // ---- window keys owned by this chunk: from the accumulators, rotated, stored to smem and to the cache
+    for (int e = tid; e < (nk - n_cached) * HALF; e += kAttnThreads) {
+      const int t = n_cached + e / HALF, i = e % HALF;
+      const int pos = k0 + t, j = pos - L;
+      const int r = bl * a.c + j;
+      const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
+      const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
+      const float *vacc = kacc + kvd;
+      float sn, cs;
+      sincosf((float)pos * inv_freq[i], &sn, &cs);
+      const float x0 = kacc[i] * s, x1 = kacc[i + HALF] * s;
+      const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * cs - x1 * sn), o1 = __float2bfloat16_rn(x0 * sn + x1 * cs);
+      const __nv_bfloat16 v0 = __float2bfloat16_rn(vacc[i] * s), v1 = __float2bfloat16_rn(vacc[i + HALF] * s);
+      Ks[t * LD + i] = o0; Ks[t * LD + i + HALF] = o1;
+      Vs[t * LD + i] = v0; Vs[t * LD + i + HALF] = v1;
+      kbase[(long long)pos * HD + i] = o0; kbase[(long long)pos * HD + i + HALF] = o1;
+      vbase[(long long)pos * HD + i] = v0; vbase[(long long)pos * HD + i + HALF] = v1;
+    }
+    // rows beyond nk: zero so that stale shared memory (possibly NaN patterns) never meets a zero weight
+    for (int e = tid; e < (kChunk - nk) * CPR; e += kAttnThreads) {
+      const int t = nk + e / CPR, p = e % CPR;
+      *reinterpret_cast<uint4 *>(Ks + t * LD + p * 8) = make_uint4(0, 0, 0, 0);
+      *reinterpret_cast<uint4 *>(Vs + t * LD + p * 8) = make_uint4(0, 0, 0, 0);
+    }
+  }
+
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  const float scale = rsqrtf((float)HD);
+  const int nqt = (nq + 15) / 16;
+  const int g4 = lane >> 2, t4 = lane & 3;
+  for (int qt = 0; qt < nqt; ++qt) {
+    __syncthreads();                                          // K/V staged; previous tile's Qs/Om/mls free
+    // ---- Q tile: 1/rms, rotation, bf16
+    for (int e = tid; e < 16 * HALF; e += kAttnThreads) {
+      const int row = e / HALF, i = e % HALF;
+      const int qrow = qt * 16 + row;
+      __nv_bfloat16 o0 = __float2bfloat16_rn(0.f), o1 = o0;
+      if (qrow < nq) {
+        const int g = qrow / a.c, j = qrow % a.c;
+        const int r = bl * a.c + j, h = kvh * group + g;
+        const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
+        const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
+        float sn, cs;
+        sincosf((float)(L + j) * inv_freq[i], &sn, &cs);
+        const float x0 = qacc[i] * s, x1 = qacc[i + HALF] * s;
+        o0 = __float2bfloat16_rn(x0 * cs - x1 * sn); o1 = __float2bfloat16_rn(x0 * sn + x1 * cs);
+      }
+      Qs[row * LD + i] = o0; Qs[row * LD + i + HALF] = o1;
+    }
+    __syncthreads();
+
+    // ---- S = Q.K^T for this warp's 32 keys
+    float sacc[4][4];
+#pragma unroll
+    for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) sacc[nb][i] = 0.f;
+    if (nk > 0) {
+#pragma unroll
+      for (int ks = 0; ks < HD / 16; ++ks) {
+        uint32_t af[4];
+        ldsm_x4(smem_addr(Qs + (lane & 15) * LD + ks * 16 + (lane >> 4) * 8), af[0], af[1], af[2], af[3]);
+#pragma unroll
+        for (int nb = 0; nb < 4; nb += 2) {
+          // two key blocks (8 keys each) x one 16-wide k step
+          uint32_t b0, b1, b2, b3;
+          const int key = warp * 32 + nb * 8 + (lane & 7) + ((lane >> 4) & 1) * 8;
+          ldsm_x4(smem_addr(Ks + key * LD + ks * 16 + ((lane >> 3) & 1) * 8), b0, b1, b2, b3);
+          mma_bf16(sacc[nb], af, b0, b1);
+          mma_bf16(sacc[nb + 1], af, b2, b3);
+        }
+      }
+    }
+    // ---- mask, scale, softmax statistics over this warp's keys (rows g4 and g4 + 8)
+    float mrow[2] = {-INFINITY, -INFINITY};
+    int jrow[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int qrow = qt * 16 + g4 + hh * 8;
+      jrow[hh] = (qrow < nq) ? (qrow % a.c) : -1;
+    }
+#pragma unroll
+    for (int nb = 0; nb < 4; ++nb)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int hh = i >> 1;
+        const int key = k0 + warp * 32 + nb * 8 + t4 * 2 + (i & 1);
+        const bool ok = jrow[hh] >= 0 && key < ltot && key <= L + jrow[hh];
+        const float s = ok ? sacc[nb][i] * scale : -INFINITY;
+        sacc[nb][i] = s;
+        mrow[hh] = fmaxf(mrow[hh], s);
+      }
+    float lrow[2] = {0.f, 0.f};
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      mrow[hh] = fmaxf(mrow[hh], __shfl_xor_sync(0xffffffffu, mrow[hh], 1));
+      mrow[hh] = fmaxf(mrow[hh], __shfl_xor_sync(0xffffffffu, mrow[hh], 2));
+    }
+    uint32_t pf[2][4];                                        // P as A fragments: two 16-key steps
+#pragma unroll
+    for (int nb = 0; nb < 4; ++nb) {
+      float p[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int hh = i >> 1;
+        p[i] = (sacc[nb][i] == -INFINITY) ? 0.f : __expf(sacc[nb][i] - mrow[hh]);
+        lrow[hh] += p[i];
+      }
+      pf[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+      pf[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+    }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      lrow[hh] += __shfl_xor_sync(0xffffffffu, lrow[hh], 1);
+      lrow[hh] += __shfl_xor_sync(0xffffffffu, lrow[hh], 2);
+    }
+    // ---- O = P.V
+    float oacc[ND][4];
+#pragma unroll
+    for (int d = 0; d < ND; ++d)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) oacc[d][i] = 0.f;
+    if (nk > 0) {
+#pragma unroll
+      for (int kt = 0; kt < 2; ++kt) {
+#pragma unroll
+        for (int d = 0; d < ND; d += 2) {
+          uint32_t b0, b1, b2, b3;
+          const int key = warp * 32 + kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          ldsm_x4_t(smem_addr(Vs + key * LD + d * 8 + (lane >> 4) * 8), b0, b1, b2, b3);
+          mma_bf16(oacc[d], pf[kt], b0, b1);
+          mma_bf16(oacc[d + 1], pf[kt], b2, b3);
+        }
+      }
+    }
+    // ---- merge the four warps
+    if (t4 == 0) {
+      mls[(warp * 16 + g4) * 2] = mrow[0]; mls[(warp * 16 + g4) * 2 + 1] = lrow[0];
+      mls[(warp * 16 + g4 + 8) * 2] = mrow[1]; mls[(warp * 16 + g4 + 8) * 2 + 1] = lrow[1];
+    }
+    __syncthreads();
+    float fac[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const int row = g4 + hh * 8;
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < 4; ++w) M = fmaxf(M, mls[(w * 16 + row) * 2]);
+      fac[hh] = (mrow[hh] == -INFINITY) ? 0.f : __expf(mrow[hh] - M);
+    }
+#pragma unroll
+    for (int d = 0; d < ND; ++d) {
+      float *o0 = Om + (warp * 16 + g4) * HD + d * 8 + t4 * 2;
+      float *o1 = Om + (warp * 16 + g4 + 8) * HD + d * 8 + t4 * 2;
+      *reinterpret_cast<float2 *>(o0) = make_float2(oacc[d][0] * fac[0], oacc[d][1] * fac[0]);
+      *reinterpret_cast<float2 *>(o1) = make_float2(oacc[d][2] * fac[1], oacc[d][3] * fac[1]);
+    }
+    __syncthreads();
+    for (int e = tid; e < 16 * HD; e += kAttnThreads) {
+      const int row = e / HD, dd = e % HD;
+      const int qrow = qt * 16 + row;
+      if (qrow >= nq) continue;
+      const int g = qrow / a.c, j = qrow % a.c;
+      const int r = bl * a.c + j, h = kvh * group + g;
+      const long long pidx = ((long long)r * a.hq + h) * a.nsplit + split;
+      a.part_o[pidx * HD + dd] = Om[row * HD + dd] + Om[(16 + row) * HD + dd] + Om[(32 + row) * HD + dd] + Om[(48 + row) * HD + dd];
+      if (dd == 0) {
+        float M = -INFINITY;
+        for (int w = 0; w < 4; ++w) M = fmaxf(M, mls[(w * 16 + row) * 2]);
+        float lsum = 0.f;
+        for (int w = 0; w < 4; ++w) {
+          const float mw = mls[(w * 16 + row) * 2];
+          if (mw != -INFINITY) lsum += mls[(w * 16 + row) * 2 + 1] * __expf(mw - M);
+        }
+        a.part_ml[pidx * 2] = M; a.part_ml[pidx * 2 + 1] = lsum;
+      }
+    }
+  }
+
+  // ---- last CTA of this (sequence, kv head): merge the splits, clear the accumulators of its heads
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int prev = atomicAdd(&a.counters[b * a.hkv + kvh], 1u);
+    s_last = (prev == (unsigned int)a.nsplit - 1u);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int qi = warp; qi < nq; qi += 4) {
+    const int g = qi / a.c, j = qi % a.c;
+    const int r = bl * a.c + j, h = kvh * group + g;
+    const long long base = ((long long)r * a.hq + h) * a.nsplit;
+    float M = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, __ldcg(&a.part_ml[(base + s) * 2]));
+    float den = 0.f, o[HD / 32];
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) o[i] = 0.f;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const float ls = __ldcg(&a.part_ml[(base + s) * 2 + 1]);
+      if (ls == 0.f) continue;
+      const float wgt = __expf(__ldcg(&a.part_ml[(base + s) * 2]) - M);
+      den = fmaf(ls, wgt, den);
+#pragma unroll
+      for (int i = 0; i < HD / 32; ++i) o[i] = fmaf(wgt, __ldcg(&a.part_o[(base + s) * HD + i * 32 + lane]), o[i]);
+    }
+    const float inv = 1.0f / den;
+#pragma unroll
+    for (int i = 0; i < HD / 32; ++i) a.out[(long long)r * qd + h * HD + i * 32 + lane] = o[i] * inv;
+    // this head's q accumulator (and, once per row, the kv head's k and v) are no longer needed
+    float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
+    for (int i = lane; i < HD; i += 32) qacc[i] = 0.f;
+    if (g == 0) {
+      float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
+      for (int i = lane; i < HD; i += 32) { kacc[i] = 0.f; kacc[kvd + i] = 0.f; }
+    }
+  }
+  if (tid == 0) {
+    a.counters[b * a.hkv + kvh] = 0u;
+    const unsigned int prev = atomicAdd(a.grid_counter, 1u);
+    s_last_grid = (prev == (unsigned int)(gridDim.y * gridDim.z) - 1u);
+  }
+  __syncthreads();
+  if (s_last_grid) {
+    for (int i = tid; i < a.nb * a.c; i += kAttnThreads) a.ss[i] = 0.f;
+    if (tid == 0) *a.grid_counter = 0u;
+  }
+}
+
+template <int HD>
+static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
+  constexpr int LD = HD + 8;
+  const size_t smem = sizeof(__nv_bfloat16) * (size_t)(2 * kChunk * LD + 16 * LD) +
+                      sizeof(float) * (size_t)(4 * 16 * HD + 4 * 16 * 2 + HD / 2);
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  dim3 grid(a.nsplit, a.hkv, a.nb);
+  attn_fused_kernel<HD><<<grid, kAttnThreads, smem, st>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st) {
+  if (hd == 64) return launch_fused_t<64>(a, st);
+  if (hd == 128) return launch_fused_t<128>(a, st);
+  return cudaErrorInvalidValue;
+}
+
+int attn_fused_chunk() { return kChunk; }
+
+}  // namespace fc
