@@ -25,6 +25,7 @@ struct Carver {          // hands out aligned slices of the caller's workspace (
 
 struct Buffers {
   float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *part_o, *part_ml;
+  float2 *rope;
   void *qb;
   unsigned int *counters, *err;
   unsigned long long *amax;
@@ -73,6 +74,7 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
   t.ss_ffn = c.take<float>(R);
   t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
   t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
+  t.rope = c.take<float2>((size_t)s->max_seq * (s->head_dim / 2));
   t.counters = c.take<unsigned int>((size_t)s->max_batch * s->n_kv_heads + 1);   // + one grid-wide word
   t.err = c.take<unsigned int>(1);
   t.amax = c.take<unsigned long long>(R);
@@ -104,6 +106,7 @@ struct fc_ctx {
   char *kv; size_t kv_layer_stride, kv_half_stride;   // bytes
   cudaStream_t st;
   bool use_umma;
+  bool pdl;          // chain the tensor-core kernels by programmatic dependent launch
   bool fused_attn;   // bf16 with head_dim 64/128: rotary embedding and K/V write happen inside the attention kernel
   int n_sms;
   std::vector<UmmaPlan *> plan_qkv, plan_o, plan_gu, plan_down;
@@ -253,6 +256,7 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   ctx->kv_layer_stride = 2 * ctx->kv_half_stride;
   ctx->st = (cudaStream_t)cuda_stream;
   ctx->use_umma = shape->dtype == FC_BF16 && !(shape->flags & FC_FLAG_SIMT_GEMM);
+  ctx->pdl = !(shape->flags & FC_FLAG_NO_PDL);
   ctx->fused_attn = shape->dtype == FC_BF16 && (shape->head_dim == 64 || shape->head_dim == 128) &&
                     !(shape->flags & FC_FLAG_SIMT_GEMM);
 
@@ -280,6 +284,7 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   if (cudaMallocHost((void **)&ctx->pin, pin_ints * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaEventCreate(&ctx->ev0) != cudaSuccess || cudaEventCreate(&ctx->ev1) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaMemsetAsync(ws, 0, fc_workspace_bytes(shape), ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
+  if (launch_rope_table(ctx->b.rope, shape->max_seq, shape->head_dim, shape->rope_theta, ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaStreamSynchronize(ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
   const int B = shape->max_batch;
   ctx->kv_len_h.assign(B, 0); ctx->n_gen_h.assign(B, 0); ctx->pending_h.assign(B, 0); ctx->done_h.assign(B, 0);
@@ -305,7 +310,7 @@ static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R
   ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
-  if (ctx->use_umma) return launch_gemm_umma(plan, a, ctx->st);
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, ctx->pdl && !ctx->prof, ctx->st);
   return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
 }
 
@@ -336,11 +341,12 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     if (ctx->fused_attn) {
       FusedAttnArgs fa; memset(&fa, 0, sizeof fa);
       fa.qkv = ctx->b.qkv; fa.ldq = d.ldq; fa.ss = ctx->b.ss_attn; fa.eps = s.rms_eps; fa.dn = s.d_model;
-      fa.theta = s.rope_theta; fa.kcache = kc; fa.vcache = vc; fa.stride_b = stride_b; fa.stride_h = stride_h;
+      fa.rope = ctx->b.rope; fa.c_magic = (unsigned int)((0x100000000ull + (unsigned)rows - 1) / (unsigned)rows);
+      fa.kcache = kc; fa.vcache = vc; fa.stride_b = stride_b; fa.stride_h = stride_h;
       fa.kv_len = ctx->b.kv_len; fa.b0 = b0; fa.nb = nb; fa.c = rows; fa.hq = s.n_heads; fa.hkv = s.n_kv_heads;
       fa.nsplit = nsplit; fa.part_o = ctx->b.part_o; fa.part_ml = ctx->b.part_ml; fa.counters = ctx->b.counters;
       fa.grid_counter = ctx->b.counters + (size_t)s.max_batch * s.n_kv_heads;
-      fa.out = ctx->b.attn;
+      fa.out = ctx->b.attn; fa.pdl = ctx->pdl && !ctx->prof;
       fa.z.p[0] = ctx->b.gu; fa.z.n[0] = Rz * 2 * s.d_ffn;
       fa.z.p[1] = ctx->b.ss_ffn; fa.z.n[1] = Rz;
       ++ctx->launches;
@@ -689,7 +695,7 @@ extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, 
   char msg[200];
   UmmaPlan *pl = umma_plan_create(a, PRO_NONE, EPI_ATOMIC_ADD, sms, err_word, msg, sizeof msg);
   if (!pl) { fprintf(stderr, "fc_op_linear: %s\n", msg); return FC_ERR_CUDA; }
-  cudaError_t e = launch_gemm_umma(pl, a, st);
+  cudaError_t e = launch_gemm_umma(pl, a, 0, st);
   unsigned int herr = 0;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&herr, err_word, sizeof herr, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);

@@ -87,7 +87,8 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   int ldq;
   float *ss;              // [R] sums of squares for 1/rms; cleared by the kernel
   float eps; int dn;
-  float theta;
+  const float2 *rope;     // [max_seq][hd/2] (cos, sin) of position * theta^(-2i/hd)
+  unsigned int c_magic;   // ceil(2^32 / c): q / c == umulhi(q, c_magic) for the small q used here
   void *kcache, *vcache;
   long long stride_b, stride_h;
   const int32_t *kv_len;
@@ -96,6 +97,7 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   float *part_o, *part_ml;
   unsigned int *counters; // [batch*hkv], zero on entry and on exit
   unsigned int *grid_counter;   // one word, zero on entry and on exit
+  int pdl;                // launched as a programmatic dependent of the previous kernel
   float *out;             // [R, hq*hd] fp32
   ZeroList z;
 };
@@ -128,6 +130,7 @@ cudaError_t launch_embed(const EmbedArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_gemm_simt(const GemmArgs &a, int dtype, int pro, int epi, cudaStream_t st);
 cudaError_t launch_rope_kv(const RopeArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st);
+cudaError_t launch_rope_table(float2 *table, int max_seq, int hd, float theta, cudaStream_t st);
 cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st);
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 int attn_tile_keys(int dtype, int hd);   // keys per split tile
@@ -144,6 +147,6 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
                            char *err, int errlen);
 void umma_plan_destroy(UmmaPlan *p);
 // x/x2/y/ss pointers and R may differ per launch from those the plan was created with.
-cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, cudaStream_t st);
+cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, int pdl, cudaStream_t st);
 
 }  // namespace fc

@@ -10,6 +10,8 @@
 // (max, sum, out) per (row, head, split) goes to scratch.  The last CTA of a (sequence, kv head) merges the
 // splits and clears the accumulators it owns; the last CTA of the grid clears the per-row sums of squares.
 // Row j of sequence b sees keys 0 .. kv_len[b] + j (cache + causal part of the window).
+#include <cstring>
+
 #include "fc_internal.h"
 
 namespace fc {
@@ -55,7 +57,6 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   __nv_bfloat16 *Qs = Vs + kChunk * LD;                                  // [16][LD]
   float *Om = reinterpret_cast<float *>(Qs + 16 * LD);                   // [4][16][HD]
   float *mls = Om + 4 * 16 * HD;                                         // [4][16][2]
-  float *inv_freq = mls + 4 * 16 * 2;                                    // [HALF]
   __shared__ unsigned int s_last, s_last_grid;
 
   const int split = blockIdx.x, kvh = blockIdx.y, bl = blockIdx.z;
@@ -68,8 +69,24 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   const int group = a.hq / a.hkv;
   const int nq = group * a.c;
   const int qd = a.hq * HD, kvd = a.hkv * HD;
+  const unsigned int c_magic = a.c_magic;
+  auto div_c = [&](int q) -> int { return a.c == 1 ? q : (int)__umulhi((unsigned int)q, c_magic); };
   __nv_bfloat16 *kbase = (__nv_bfloat16 *)a.kcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
   __nv_bfloat16 *vbase = (__nv_bfloat16 *)a.vcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+
+  // ---- cached keys of this chunk: 16-byte asynchronous copies, issued before anything else
+  constexpr int CPR = HD / 8;                                // 16-byte pieces per row
+  const int n_cached = nk > 0 ? min(nk, max(0, L - k0)) : 0;
+  for (int e = tid; e < n_cached * CPR; e += kAttnThreads) {
+    const int t = e / CPR, p = e % CPR;
+    cp_async16(smem_addr(Ks + t * LD + p * 8), kbase + (long long)(k0 + t) * HD + p * 8);
+    cp_async16(smem_addr(Vs + t * LD + p * 8), vbase + (long long)(k0 + t) * HD + p * 8);
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  // The cached keys above were written by earlier steps; everything below depends on the previous kernel
+  // (the QKV projection), so let the next kernel start its prefetch and wait for the previous one here.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // side clearing of buffers nobody reads during this kernel
   {
@@ -81,19 +98,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       if (a.z.p[i]) for (unsigned long long e = gtid; e < a.z.n[i]; e += nth) a.z.p[i][e] = 0.f;
   }
 
-  for (int i = tid; i < HALF; i += kAttnThreads) inv_freq[i] = powf(a.theta, -2.0f * (float)i / (float)HD);
-  __syncthreads();
-
   if (nk > 0) {
-    // ---- cached keys: 16-byte copies
-    const int n_cached = min(nk, max(0, L - k0));
-    constexpr int CPR = HD / 8;                              // 16-byte pieces per row
-    for (int e = tid; e < n_cached * CPR; e += kAttnThreads) {
-      const int t = e / CPR, p = e % CPR;
-      cp_async16(smem_addr(Ks + t * LD + p * 8), kbase + (long long)(k0 + t) * HD + p * 8);
-      cp_async16(smem_addr(Vs + t * LD + p * 8), vbase + (long long)(k0 + t) * HD + p * 8);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
     // ---- window keys owned by this chunk: from the accumulators, rotated, stored to smem and to the cache
     for (int e = tid; e < (nk - n_cached) * HALF; e += kAttnThreads) {
       const int t = n_cached + e / HALF, i = e % HALF;
@@ -102,8 +107,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
       const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
       const float *vacc = kacc + kvd;
-      float sn, cs;
-      sincosf((float)pos * inv_freq[i], &sn, &cs);
+      const float2 rot = __ldg(a.rope + (long long)pos * HALF + i);
+      const float cs = rot.x, sn = rot.y;
       const float x0 = kacc[i] * s, x1 = kacc[i + HALF] * s;
       const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * cs - x1 * sn), o1 = __float2bfloat16_rn(x0 * sn + x1 * cs);
       const __nv_bfloat16 v0 = __float2bfloat16_rn(vacc[i] * s), v1 = __float2bfloat16_rn(vacc[i + HALF] * s);
@@ -132,12 +137,12 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       const int qrow = qt * 16 + row;
       __nv_bfloat16 o0 = __float2bfloat16_rn(0.f), o1 = o0;
       if (qrow < nq) {
-        const int g = qrow / a.c, j = qrow % a.c;
+        const int g = div_c(qrow), j = qrow - g * a.c;
         const int r = bl * a.c + j, h = kvh * group + g;
         const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
         const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
-        float sn, cs;
-        sincosf((float)(L + j) * inv_freq[i], &sn, &cs);
+        const float2 rot = __ldg(a.rope + (long long)(L + j) * HALF + i);
+        const float cs = rot.x, sn = rot.y;
         const float x0 = qacc[i] * s, x1 = qacc[i + HALF] * s;
         o0 = __float2bfloat16_rn(x0 * cs - x1 * sn); o1 = __float2bfloat16_rn(x0 * sn + x1 * cs);
       }
@@ -173,7 +178,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
       const int qrow = qt * 16 + g4 + hh * 8;
-      jrow[hh] = (qrow < nq) ? (qrow % a.c) : -1;
+      jrow[hh] = (qrow < nq) ? (qrow - div_c(qrow) * a.c) : -1;
     }
 #pragma unroll
     for (int nb = 0; nb < 4; ++nb)
@@ -256,7 +261,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       const int row = e / HD, dd = e % HD;
       const int qrow = qt * 16 + row;
       if (qrow >= nq) continue;
-      const int g = qrow / a.c, j = qrow % a.c;
+      const int g = div_c(qrow), j = qrow - g * a.c;
       const int r = bl * a.c + j, h = kvh * group + g;
       const long long pidx = ((long long)r * a.hq + h) * a.nsplit + split;
       a.part_o[pidx * HD + dd] = Om[row * HD + dd] + Om[(16 + row) * HD + dd] + Om[(32 + row) * HD + dd] + Om[(48 + row) * HD + dd];
@@ -284,21 +289,39 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   if (!s_last) return;
   __threadfence();
   for (int qi = warp; qi < nq; qi += 4) {
-    const int g = qi / a.c, j = qi % a.c;
+    const int g = div_c(qi), j = qi - g * a.c;
     const int r = bl * a.c + j, h = kvh * group + g;
     const long long base = ((long long)r * a.hq + h) * a.nsplit;
+    // lanes take one split each for the (max, sum) pairs; the output loads below are independent
+    const float2 *ml2 = reinterpret_cast<const float2 *>(a.part_ml) + base;
     float M = -INFINITY;
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, __ldcg(&a.part_ml[(base + s) * 2]));
+    for (int s0 = 0; s0 < a.nsplit; s0 += 32) {
+      const int s = s0 + lane;
+      if (s < a.nsplit) { const float2 ml = __ldcg(ml2 + s); if (ml.y > 0.f) M = fmaxf(M, ml.x); }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float den = 0.f, o[HD / 32];
 #pragma unroll
     for (int i = 0; i < HD / 32; ++i) o[i] = 0.f;
-    for (int s = 0; s < a.nsplit; ++s) {
-      const float ls = __ldcg(&a.part_ml[(base + s) * 2 + 1]);
-      if (ls == 0.f) continue;
-      const float wgt = __expf(__ldcg(&a.part_ml[(base + s) * 2]) - M);
-      den = fmaf(ls, wgt, den);
+    for (int s0 = 0; s0 < a.nsplit; s0 += 32) {
+      const int s = s0 + lane;
+      float wl = 0.f, wgt = 0.f;
+      if (s < a.nsplit) {
+        const float2 ml = __ldcg(ml2 + s);
+        if (ml.y > 0.f) { wgt = __expf(ml.x - M); wl = ml.y * wgt; }
+      }
 #pragma unroll
-      for (int i = 0; i < HD / 32; ++i) o[i] = fmaf(wgt, __ldcg(&a.part_o[(base + s) * HD + i * 32 + lane]), o[i]);
+      for (int sh = 16; sh > 0; sh >>= 1) wl += __shfl_xor_sync(0xffffffffu, wl, sh);
+      den += wl;
+      const int ns = min(32, a.nsplit - s0);
+      const float *po = a.part_o + (base + s0) * HD + lane;
+#pragma unroll 8
+      for (int t = 0; t < ns; ++t) {
+        const float w = __shfl_sync(0xffffffffu, wgt, t);
+#pragma unroll
+        for (int i = 0; i < HD / 32; ++i) o[i] = fmaf(w, __ldcg(po + (long long)t * HD + i * 32), o[i]);
+      }
     }
     const float inv = 1.0f / den;
 #pragma unroll
@@ -327,16 +350,21 @@ template <int HD>
 static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
   constexpr int LD = HD + 8;
   const size_t smem = sizeof(__nv_bfloat16) * (size_t)(2 * kChunk * LD + 16 * LD) +
-                      sizeof(float) * (size_t)(4 * 16 * HD + 4 * 16 * 2 + HD / 2);
+                      sizeof(float) * (size_t)(4 * 16 * HD + 4 * 16 * 2);
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  dim3 grid(a.nsplit, a.hkv, a.nb);
-  attn_fused_kernel<HD><<<grid, kAttnThreads, smem, st>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(a.nsplit, a.hkv, a.nb); cfg.blockDim = dim3(kAttnThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = a.pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, attn_fused_kernel<HD>, a);
 }
 
 cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st) {
@@ -346,5 +374,22 @@ cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st) {
 }
 
 int attn_fused_chunk() { return kChunk; }
+
+// cos/sin of pos * theta^(-2i/hd), computed once per context with the precise library routines.
+__global__ void rope_table_kernel(float2 *table, int max_seq, int half, float theta) {
+  const long long n = (long long)max_seq * half;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
+    const int pos = (int)(e / half), i = (int)(e % half);
+    const float freq = powf(theta, -2.0f * (float)i / (float)(2 * half));
+    float sn, cs;
+    sincosf((float)pos * freq, &sn, &cs);
+    table[e] = make_float2(cs, sn);
+  }
+}
+
+cudaError_t launch_rope_table(float2 *table, int max_seq, int hd, float theta, cudaStream_t st) {
+  rope_table_kernel<<<296, 256, 0, st>>>(table, max_seq, hd / 2, theta);
+  return cudaGetLastError();
+}
 
 }  // namespace fc

@@ -35,6 +35,7 @@ struct UmmaParams {
   int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
   int stages;
   int items_per_cta_mode;         // 0: stream-K ranges, 1: whole tiles round-robin (argmax epilogue)
+  int pdl;                        // launched as a programmatic dependent of the previous kernel
   unsigned int *err;              // device error word (0 = ok)
 };
 
@@ -198,7 +199,6 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
                  const __grid_constant__ CUtensorMap map2, const UmmaParams p) {
   constexpr int kStageBytes = kWBytes + BN * 128;
-  constexpr int kUnits = BN / 16;                 // (row, 16-byte chunk) units per staging thread per stage
   constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
   constexpr uint32_t kIdesc = make_idesc(BN);
 
@@ -206,7 +206,7 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
   __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
-  __shared__ float ss_s[2][BN];
+  __shared__ float ss_part[2][4][BN];   // per accumulator, per staging warp: partial sums of squares
 
   const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -217,7 +217,7 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
 
   if (threadIdx.x == 0) {
     abort_s = 0;
-    for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&full_w[i]), 1); mbar_init(smem_u32(&full_x[i]), 4); mbar_init(smem_u32(&empty_b[i]), 1); }
+    for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&full_w[i]), 1); mbar_init(smem_u32(&full_x[i]), 1); mbar_init(smem_u32(&empty_b[i]), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
     mbar_init(smem_u32(&drain_bar), 1);
     fence_barrier_init();
@@ -227,6 +227,9 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
+  // Let the next kernel of the chain start its own set-up and weight prefetch as soon as every CTA of this
+  // grid has got this far (it still waits for this grid to finish before it touches any activation).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   int issued = 0;   // producer: k-block loads issued (for the drain on abort)
 
@@ -288,7 +291,14 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
     }
   } else if (warp < 6) {
     // ------------------------------------------------------------ activation staging
-    const int tid_s = threadIdx.x - 64;
+    // Each of the four staging warps owns every fourth k-block, so four blocks are in flight at once and
+    // the L2 latency of the activation loads is hidden.  A lane handles kUW (row, 16-byte chunk) units.
+    // Weights never depend on the previous kernel, so the producer warp is already streaming them; the
+    // activations do, so wait here for the previous grid to complete.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int sw = warp - 2;
+    constexpr int kUW = BN / 4;
+    const int chunk = lane & 7;
     int it = 0, seg = 0;
     bool ok = true;
     for (int rb = 0; rb < nrb && ok; ++rb) {
@@ -296,28 +306,30 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
       Segment s;
       while (ok && si.next(s)) {
         const int acc = seg & 1;
-        float ssq[kUnits], srow[kUnits];
-#pragma unroll
-        for (int u = 0; u < kUnits; ++u) {
-          ssq[u] = 0.f; srow[u] = 1.f;
-          if (PRO == PRO_SILU_MUL) {
-            const int r = rb * BN + ((u * 128 + tid_s) >> 3);
-            if (r < g.R) srow[u] = rsqrtf(g.ss_in[r] / (float)g.dn + g.eps);
+        const bool need_ss = PRO == PRO_GAIN && (EPI == EPI_ARGMAX || (g.ss_out != nullptr && s.tile == 0));
+        float *my_ss = &ss_part[acc][sw][0];
+        if (need_ss) {
+          if (EPI == EPI_ARGMAX) {   // the epilogue two segments back must have let go of this buffer
+            if (!mbar_wait_warp(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
           }
+          for (int row = lane; row < BN; row += 32) my_ss[row] = 0.f;
+          __syncwarp();
         }
         for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+          if ((it & 3) != sw) continue;
           const int stage = it % S;
           const uint32_t ph = (uint32_t)(it / S) & 1u;
           if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
-#pragma unroll
-          for (int u = 0; u < kUnits; ++u) {
-            const int unit = u * 128 + tid_s;
-            const int row = unit >> 3, chunk = unit & 7;
-            const int r = rb * BN + row, k = kb * kTileK + chunk * 8;
+          const int k = kb * kTileK + chunk * 8;
+#pragma unroll 4
+          for (int u = 0; u < kUW; ++u) {
+            const int row = u * 4 + (lane >> 3);
+            const int r = rb * BN + row;
             float v[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) v[i] = 0.f;
+            float sq = 0.f;
             if (r < g.R && k < g.K) {
               const float4 a0 = *reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k);
               const float4 a1 = *reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k + 4);
@@ -328,19 +340,26 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                   const float2 gf = __bfloat1622float2(gp[i]);
-                  ssq[u] = fmaf(v[2 * i], v[2 * i], ssq[u]); ssq[u] = fmaf(v[2 * i + 1], v[2 * i + 1], ssq[u]);
+                  sq = fmaf(v[2 * i], v[2 * i], sq); sq = fmaf(v[2 * i + 1], v[2 * i + 1], sq);
                   v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
                 }
               } else if (PRO == PRO_SILU_MUL) {
+                const float sr = rsqrtf(__ldg(g.ss_in + r) / (float)g.dn + g.eps);
                 const float4 u0 = *reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k);
                 const float4 u1 = *reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k + 4);
                 const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                  const float gt = srow[u] * v[i];
-                  v[i] = (gt / (1.0f + __expf(-gt))) * (srow[u] * uu[i]);
+                  const float gt = sr * v[i];
+                  v[i] = (gt / (1.0f + __expf(-gt))) * (sr * uu[i]);
                 }
               }
+            }
+            if (need_ss) {      // uniform across the warp
+              sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+              sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+              sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+              if (chunk == 0) my_ss[row] += sq;
             }
             uint4 pk;
             __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
@@ -354,26 +373,15 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
           if (lane == 0) mbar_arrive(smem_u32(&full_x[stage]));
         }
         if (!ok) break;
-        if (PRO == PRO_GAIN && (EPI == EPI_ARGMAX || (g.ss_out != nullptr && s.tile == 0))) {
-          if (EPI == EPI_ARGMAX) {   // ss_s[acc] is free once the epilogue two segments back has let go of it
-            if (!mbar_wait_warp(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          }
-#pragma unroll
-          for (int u = 0; u < kUnits; ++u) {
-            float t = ssq[u];
-            t += __shfl_xor_sync(0xffffffffu, t, 1);
-            t += __shfl_xor_sync(0xffffffffu, t, 2);
-            t += __shfl_xor_sync(0xffffffffu, t, 4);
-            const int unit = u * 128 + tid_s;
-            const int row = unit >> 3, r = rb * BN + row;
-            if ((unit & 7) == 0) {
-              if (EPI == EPI_ARGMAX) ss_s[acc][row] = t;
-              else if (r < g.R) atomicAdd(&g.ss_out[r], t);
-            }
-          }
+        if (need_ss) {
+          __syncwarp();
           if (EPI == EPI_ARGMAX) {
-            __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ss_ready[acc]));
+          } else {
+            for (int row = lane; row < BN; row += 32) {
+              const int r = rb * BN + row;
+              if (r < g.R) atomicAdd(&g.ss_out[r], my_ss[row]);
+            }
           }
         }
         ++seg;
@@ -381,6 +389,7 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ epilogue
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs may still be read by the previous grid
     const int q = warp & 3;
     const int n_local = q * 32 + lane;
     int seg = 0;
@@ -409,7 +418,8 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
             if (EPI == EPI_ATOMIC_ADD) {
               if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
             } else {
-              float logit = v[j] * rsqrtf(ss_s[acc][c0 + j] / (float)g.dn + g.eps);
+              const float ssum = ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
+              float logit = v[j] * rsqrtf(ssum / (float)g.dn + g.eps);
               unsigned long long key = 0ull;
               if (valid) {
                 if (g.perm && g.perm[g.tokens[r]] == col) logit += g.beta;
@@ -526,8 +536,14 @@ static cudaError_t launch_one(const UmmaPlan *pl, const UmmaParams &p, int grid,
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  gemm_umma_kernel<PRO, EPI, BN><<<grid, kThreads, smem, st>>>(pl->maps[0], pl->maps[1], pl->maps[2], p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = p.pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<PRO, EPI, BN>, pl->maps[0], pl->maps[1], pl->maps[2], p);
 }
 
 template <int PRO, int EPI>
@@ -541,10 +557,11 @@ static cudaError_t launch_bn(const UmmaPlan *pl, const UmmaParams &p, int bn, in
   }
 }
 
-cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, cudaStream_t st) {
+cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, int pdl, cudaStream_t st) {
   UmmaParams p = pl->p;
   // per-launch fields (buffers and row count); weights, K and the matrix split stay as planned
   p.g.x = a.x; p.g.x2 = a.x2; p.g.ldx = a.ldx; p.g.ss_in = a.ss_in; p.g.ss_out = a.ss_out;
+  p.pdl = pdl;
   p.g.y = a.y; p.g.ldy = a.ldy; p.g.R = a.R; p.g.tokens = a.tokens; p.g.amax = a.amax; p.g.logits = a.logits;
   int bn, cps;
   bn_config(a.R, bn, p.stages, cps);
