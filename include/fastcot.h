@@ -51,7 +51,8 @@ typedef enum {
 enum {                        /* fc_model_shape.flags */
   FC_FLAG_SIMT_GEMM = 1,      /* run projections on the plain FMA kernels even for bf16 (debug aid) */
   FC_FLAG_NO_GRAPH = 2,       /* never capture the step into a CUDA graph */
-  FC_FLAG_NO_PDL = 4          /* launch every kernel fully serialised (no programmatic dependent launch) */
+  FC_FLAG_NO_PDL = 4,         /* launch every kernel fully serialised (no programmatic dependent launch) */
+  FC_FLAG_NO_CHAIN = 8        /* one launch per projection instead of one chained launch per layer */
 };
 
 typedef struct {

@@ -27,7 +27,7 @@ struct Buffers {
   float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *part_o, *part_ml;
   float2 *rope;
   void *qb;
-  unsigned int *counters, *err;
+  unsigned int *counters, *err, *chain_bar;
   unsigned long long *amax;
   int32_t *window, *kv_len, *n_gen, *done, *acc_count, *acc_tokens, *prompt, *prompt_lens, *out_tokens;
 };
@@ -72,6 +72,7 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
   t.gu = c.take<float>(R * 2 * (size_t)s->d_ffn);
   t.ss_attn = c.take<float>(R);
   t.ss_ffn = c.take<float>(R);
+  t.chain_bar = c.take<unsigned int>((size_t)s->n_layers * 4);   // directly after the sums of squares: cleared with them
   t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
   t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
   t.rope = c.take<float2>((size_t)s->max_seq * (s->head_dim / 2));
@@ -107,6 +108,7 @@ struct fc_ctx {
   cudaStream_t st;
   bool use_umma;
   bool pdl;          // chain the tensor-core kernels by programmatic dependent launch
+  bool chain;        // run O -> gate/up -> down -> next layer's QKV as one launch with grid barriers
   bool fused_attn;   // bf16 with head_dim 64/128: rotary embedding and K/V write happen inside the attention kernel
   int n_sms;
   std::vector<UmmaPlan *> plan_qkv, plan_o, plan_gu, plan_down;
@@ -257,6 +259,7 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   ctx->st = (cudaStream_t)cuda_stream;
   ctx->use_umma = shape->dtype == FC_BF16 && !(shape->flags & FC_FLAG_SIMT_GEMM);
   ctx->pdl = !(shape->flags & FC_FLAG_NO_PDL);
+  ctx->chain = ctx->use_umma && !(shape->flags & FC_FLAG_NO_CHAIN);
   ctx->fused_attn = shape->dtype == FC_BF16 && (shape->head_dim == 64 || shape->head_dim == 128) &&
                     !(shape->flags & FC_FLAG_SIMT_GEMM);
 
@@ -326,16 +329,19 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   ea.tokens = tokens; ea.emb = ctx->tok_emb; ea.x = ctx->b.x; ea.R = R; ea.d = s.d_model;
   ea.z.p[0] = ctx->b.qkv; ea.z.n[0] = Rz * d.ldq;
   ea.z.p[1] = ctx->b.gu; ea.z.n[1] = Rz * 2 * s.d_ffn;
-  ea.z.p[2] = ctx->b.ss_attn; ea.z.n[2] = Rz;
-  ea.z.p[3] = ctx->b.ss_ffn; ea.z.n[3] = Rz;
+  // sums of squares (both norms) and the grid-barrier words of the chained projections are adjacent
+  ea.z.p[2] = ctx->b.ss_attn;
+  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + (size_t)s.n_layers * 4) - (char *)ctx->b.ss_attn) / sizeof(float);
   ++ctx->launches;
   { ProfScope ps(ctx, FC_CLS_EMBED); FC_CK(launch_embed(ea, s.dtype, ctx->st)); }
 
   const int nsplit = (max_len_host + rows + d.tk - 1) / d.tk;
   const long long stride_h = (long long)s.max_seq * s.head_dim;
   const long long stride_b = (long long)s.n_kv_heads * stride_h;
+  const bool chained = ctx->chain && !ctx->prof;
   for (int l = 0; l < s.n_layers; ++l) {
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV));
+    if (!chained || l == 0)
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV));
     void *kc = ctx->kv + (size_t)l * ctx->kv_layer_stride;
     void *vc = ctx->kv + (size_t)l * ctx->kv_layer_stride + ctx->kv_half_stride;
     if (ctx->fused_attn) {
@@ -371,9 +377,20 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ++ctx->launches;
       { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st)); }
     }
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ));
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP));
-    FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN));
+    if (chained) {
+      // O projection, gate/up, down and the next layer's QKV: one persistent launch, three grid barriers
+      const UmmaPlan *plans[4] = {ctx->plan_o[l], ctx->plan_gu[l], ctx->plan_down[l], nullptr};
+      GemmArgs ga[4] = {args_o(ctx, l), args_gu(ctx, l), args_down(ctx, l), GemmArgs()};
+      int n = 3;
+      if (l + 1 < s.n_layers) { plans[3] = ctx->plan_qkv[l + 1]; ga[3] = args_qkv(ctx, l + 1); n = 4; }
+      for (int i = 0; i < n; ++i) ga[i].R = R;
+      ++ctx->launches;
+      FC_CK(launch_gemm_chain(plans, ga, n, ctx->b.chain_bar + (size_t)l * 4, ctx->pdl, ctx->st));
+    } else {
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN));
+    }
   }
   if (with_head) {
     GemmArgs ha = args_head(ctx);

@@ -26,23 +26,34 @@ constexpr int kTileM = 128;       // weight rows per tile
 constexpr int kTileK = 64;        // k elements per stage (128 bytes of bf16 = one swizzle row)
 constexpr int kWBytes = kTileM * kTileK * 2;
 constexpr int kThreads = 320;
-constexpr unsigned long long kSpinBudget = 4000000000ull;   // clock64 ticks (~2 s)
+constexpr unsigned long long kSpinBudget = 400000000ull;    // clock64 ticks (~0.2 s)
 
-struct UmmaParams {
+constexpr int kMaxPhases = 4;      // projections chained in one launch (O -> gate/up -> down -> next QKV)
+
+struct PhaseDesc {
   GemmArgs g;
+  int pro;                        // ProOp applied while the activations are staged
   int n_tiles, nkb;               // 128-row tiles over all matrices; 64-wide k blocks
   int tiles_m[kMaxMats];
   int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
+};
+
+struct MapPack { CUtensorMap m[kMaxPhases * kMaxMats]; };
+
+struct UmmaParams {
+  PhaseDesc ph[kMaxPhases];
+  int n_phases;
   int stages;
-  int items_per_cta_mode;         // 0: stream-K ranges, 1: whole tiles round-robin (argmax epilogue)
+  int tile_mode;                  // 0: stream-K ranges, 1: whole tiles round-robin (argmax epilogue)
   int pdl;                        // launched as a programmatic dependent of the previous kernel
   unsigned int *err;              // device error word (0 = ok)
+  unsigned int *bar;              // [n_phases - 1] grid-barrier counters, zero when the kernel starts
 };
 
 struct UmmaPlan {
-  UmmaParams p;
+  PhaseDesc d;
   CUtensorMap maps[kMaxMats];
-  int pro, epi, grid, n_sms;
+  int epi, n_sms;
   unsigned int *err;
 };
 
@@ -147,18 +158,50 @@ __device__ __forceinline__ unsigned int ordered_key_u(float v) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Grid barrier between two phases of a chained launch.  Every CTA of the grid is resident (the grid is
+// sized to the SM count times the CTAs that fit per SM), so the wait ends; it is bounded all the same.
+// signal: each participating warp calls it once after its last global write of the phase.
+__device__ __forceinline__ void grid_bar_signal(unsigned int *ctr, int lane) {
+  __threadfence();
+  __syncwarp();
+  if (lane == 0) atomicAdd(ctr, 1u);
+}
+__device__ __forceinline__ bool grid_bar_wait(const unsigned int *ctr, unsigned int target, int lane,
+                                              volatile int *abort_flag) {
+  int ok = 1;
+  if (lane == 0) {
+    const unsigned long long t0 = clock64();
+    unsigned int spins = 0;
+    while (ld_acquire_u32(ctr) < target) {
+      if ((++spins & 0x3Fu) == 0u) {
+        if (*abort_flag) { ok = 0; break; }
+        if ((unsigned long long)(clock64() - t0) > kSpinBudget) { *abort_flag = 1; ok = 0; break; }
+      }
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;     // also orders the other lanes after lane 0's acquire
+}
+
 struct Segment { int tile, kb0, kb1; };
 
-// Work of one CTA: stream-K mode deals contiguous (tile, k-block) ranges; tile mode deals whole tiles.
+// Work of one CTA in one phase: stream-K mode deals contiguous (tile, k-block) ranges; tile mode deals
+// whole tiles round-robin.
 struct SegIter {
-  long long w, w1;      // stream-K cursor
+  long long w, w1;
   int tile, tile_step, n_tiles, nkb, mode;
-  __device__ SegIter(const UmmaParams &p) {
-    mode = p.items_per_cta_mode; nkb = p.nkb; n_tiles = p.n_tiles;
+  __device__ SegIter(const PhaseDesc &d, int tile_mode) {
+    mode = tile_mode; nkb = d.nkb; n_tiles = d.n_tiles;
     if (mode == 0) {
-      const long long W = (long long)p.n_tiles * p.nkb;
+      const long long W = (long long)d.n_tiles * d.nkb;
       w = W * blockIdx.x / gridDim.x;
       w1 = W * (blockIdx.x + 1) / gridDim.x;
+      tile = tile_step = 0;
     } else { tile = blockIdx.x; tile_step = gridDim.x; w = w1 = 0; }
   }
   __device__ bool next(Segment &s) {
@@ -176,13 +219,13 @@ struct SegIter {
   }
 };
 
-__device__ __forceinline__ void tile_info(const UmmaParams &p, int tile, int &m, int &row0, int &rows_valid, int &ycol0) {
+__device__ __forceinline__ void tile_info(const PhaseDesc &d, int tile, int &m, int &row0, int &rows_valid, int &ycol0) {
   m = 0;
   int lt = tile;
-  while (m + 1 < p.g.n_mats && lt >= p.tiles_m[m]) { lt -= p.tiles_m[m]; ++m; }
+  while (m + 1 < d.g.n_mats && lt >= d.tiles_m[m]) { lt -= d.tiles_m[m]; ++m; }
   row0 = lt * kTileM;
-  rows_valid = min(kTileM, p.g.n_rows[m] - row0);
-  ycol0 = p.g.y_off[m] + row0;
+  rows_valid = min(kTileM, d.g.n_rows[m] - row0);
+  ycol0 = d.g.y_off[m] + row0;
 }
 
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
@@ -194,13 +237,14 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
   return v;
 }
 
-template <int PRO, int EPI, int BN>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant__ CUtensorMap map1,
-                 const __grid_constant__ CUtensorMap map2, const UmmaParams p) {
+// Widths up to 64 rows run two CTAs per SM (the grid barrier needs the whole grid resident).
+template <int EPI, int BN>
+__global__ void __launch_bounds__(kThreads, (BN <= 64 ? 2 : 1))
+gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ UmmaParams p) {
   constexpr int kStageBytes = kWBytes + BN * 128;
   constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
   constexpr uint32_t kIdesc = make_idesc(BN);
+  constexpr unsigned int kSignalsPerCta = 8;    // 4 staging + 4 epilogue warps signal each grid barrier
 
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar;
@@ -211,8 +255,8 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
   const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = p.stages;
-  const GemmArgs &g = p.g;
-  const int nrb = (g.R + BN - 1) / BN;
+  const int R = p.ph[0].g.R;                  // every phase of a chain works on the same rows
+  const int nrb = (R + BN - 1) / BN;
   volatile int *abort_flag = &abort_s;
 
   if (threadIdx.x == 0) {
@@ -227,32 +271,37 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  // Let the next kernel of the chain start its own set-up and weight prefetch as soon as every CTA of this
-  // grid has got this far (it still waits for this grid to finish before it touches any activation).
+  // Let the next kernel of the stream start its own set-up and weight prefetch as soon as every CTA of
+  // this grid has got this far (it still waits for this grid to finish before it touches any activation).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   int issued = 0;   // producer: k-block loads issued (for the drain on abort)
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
+    // Weights depend on nothing that runs on the device, so the producer never waits for a grid barrier
+    // or for the previous kernel: it streams phase after phase, limited only by free ring slots.
     if (lane == 0) {
       int it = 0;
       bool ok = true;
-      for (int rb = 0; rb < nrb && ok; ++rb) {
-        SegIter si(p);
-        Segment s;
-        while (ok && si.next(s)) {
-          int m, row0, rows_valid, ycol0;
-          tile_info(p, s.tile, m, row0, rows_valid, ycol0);
-          const CUtensorMap *mp = (m == 0) ? &map0 : (m == 1 ? &map1 : &map2);
-          for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
-            const int stage = it % S;
-            const uint32_t ph = (uint32_t)(it / S) & 1u;
-            if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t bar = smem_u32(&full_w[stage]);
-            mbar_expect_tx(bar, (uint32_t)p.tx_bytes[m]);
-            tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
-            issued = it + 1;
+      for (int pi = 0; pi < p.n_phases && ok; ++pi) {
+        const PhaseDesc &P = p.ph[pi];
+        for (int rb = 0; rb < nrb && ok; ++rb) {
+          SegIter si(P, p.tile_mode);
+          Segment s;
+          while (ok && si.next(s)) {
+            int m, row0, rows_valid, ycol0;
+            tile_info(P, s.tile, m, row0, rows_valid, ycol0);
+            const CUtensorMap *mp = &maps.m[pi * kMaxMats + m];
+            for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+              const int stage = it % S;
+              const uint32_t ph = (uint32_t)(it / S) & 1u;
+              if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+              const uint32_t bar = smem_u32(&full_w[stage]);
+              mbar_expect_tx(bar, (uint32_t)P.tx_bytes[m]);
+              tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
+              issued = it + 1;
+            }
           }
         }
       }
@@ -262,30 +311,33 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
     if (lane == 0) {
       int it = 0, seg = 0;
       bool ok = true;
-      for (int rb = 0; rb < nrb && ok; ++rb) {
-        SegIter si(p);
-        Segment s;
-        while (ok && si.next(s)) {
-          const int acc = seg & 1;
-          if (!mbar_wait(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-          for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
-            const int stage = it % S;
-            const uint32_t ph = (uint32_t)(it / S) & 1u;
-            if (!mbar_wait(smem_u32(&full_w[stage]), ph, abort_flag) ||
-                !mbar_wait(smem_u32(&full_x[stage]), ph, abort_flag)) { ok = false; break; }
+      for (int pi = 0; pi < p.n_phases && ok; ++pi) {
+        const PhaseDesc &P = p.ph[pi];
+        for (int rb = 0; rb < nrb && ok; ++rb) {
+          SegIter si(P, p.tile_mode);
+          Segment s;
+          while (ok && si.next(s)) {
+            const int acc = seg & 1;
+            if (!mbar_wait(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t a_base = smem_base + stage * kStageBytes;
-            const uint32_t b_base = a_base + kWBytes;
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+            for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+              const int stage = it % S;
+              const uint32_t ph = (uint32_t)(it / S) & 1u;
+              if (!mbar_wait(smem_u32(&full_w[stage]), ph, abort_flag) ||
+                  !mbar_wait(smem_u32(&full_x[stage]), ph, abort_flag)) { ok = false; break; }
+              tc_fence_after();
+              const uint32_t a_base = smem_base + stage * kStageBytes;
+              const uint32_t b_base = a_base + kWBytes;
 #pragma unroll
-            for (int kk = 0; kk < kTileK / 16; ++kk)
-              umma_bf16(d_tmem, smem_desc_sw128(a_base + kk * 32), smem_desc_sw128(b_base + kk * 32), kIdesc,
-                        (kb > s.kb0 || kk > 0) ? 1u : 0u);
-            umma_commit(smem_u32(&empty_b[stage]));
+              for (int kk = 0; kk < kTileK / 16; ++kk)
+                umma_bf16(d_tmem, smem_desc_sw128(a_base + kk * 32), smem_desc_sw128(b_base + kk * 32), kIdesc,
+                          (kb > s.kb0 || kk > 0) ? 1u : 0u);
+              umma_commit(smem_u32(&empty_b[stage]));
+            }
+            if (ok) umma_commit(smem_u32(&accum_full[acc]));
+            ++seg;
           }
-          if (ok) umma_commit(smem_u32(&accum_full[acc]));
-          ++seg;
         }
       }
     }
@@ -301,91 +353,100 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
     const int chunk = lane & 7;
     int it = 0, seg = 0;
     bool ok = true;
-    for (int rb = 0; rb < nrb && ok; ++rb) {
-      SegIter si(p);
-      Segment s;
-      while (ok && si.next(s)) {
-        const int acc = seg & 1;
-        const bool need_ss = PRO == PRO_GAIN && (EPI == EPI_ARGMAX || (g.ss_out != nullptr && s.tile == 0));
-        float *my_ss = &ss_part[acc][sw][0];
-        if (need_ss) {
-          if (EPI == EPI_ARGMAX) {   // the epilogue two segments back must have let go of this buffer
-            if (!mbar_wait_warp(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+    for (int pi = 0; pi < p.n_phases && ok; ++pi) {
+      const PhaseDesc &P = p.ph[pi];
+      const GemmArgs &g = P.g;
+      const int pro = P.pro;
+      // the activations of this phase are the previous phase's outputs, reduced by every CTA of the grid
+      if (pi > 0 && !grid_bar_wait(p.bar + (pi - 1), gridDim.x * kSignalsPerCta, lane, abort_flag)) { ok = false; break; }
+      for (int rb = 0; rb < nrb && ok; ++rb) {
+        SegIter si(P, p.tile_mode);
+        Segment s;
+        while (ok && si.next(s)) {
+          const int acc = seg & 1;
+          const bool need_ss = pro == PRO_GAIN && (EPI == EPI_ARGMAX || (g.ss_out != nullptr && s.tile == 0));
+          float *my_ss = &ss_part[acc][sw][0];
+          if (need_ss) {
+            if (EPI == EPI_ARGMAX) {   // the epilogue two segments back must have let go of this buffer
+              if (!mbar_wait_warp(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+            }
+            for (int row = lane; row < BN; row += 32) my_ss[row] = 0.f;
+            __syncwarp();
           }
-          for (int row = lane; row < BN; row += 32) my_ss[row] = 0.f;
-          __syncwarp();
-        }
-        for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
-          if ((it & 3) != sw) continue;
-          const int stage = it % S;
-          const uint32_t ph = (uint32_t)(it / S) & 1u;
-          if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
-          unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
-          const int k = kb * kTileK + chunk * 8;
+          for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+            if ((it & 3) != sw) continue;
+            const int stage = it % S;
+            const uint32_t ph = (uint32_t)(it / S) & 1u;
+            if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+            unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
+            const int k = kb * kTileK + chunk * 8;
 #pragma unroll 4
-          for (int u = 0; u < kUW; ++u) {
-            const int row = u * 4 + (lane >> 3);
-            const int r = rb * BN + row;
-            float v[8];
+            for (int u = 0; u < kUW; ++u) {
+              const int row = u * 4 + (lane >> 3);
+              const int r = rb * BN + row;
+              float v[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = 0.f;
-            float sq = 0.f;
-            if (r < g.R && k < g.K) {
-              const float4 a0 = *reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k);
-              const float4 a1 = *reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k + 4);
-              v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
-              if (PRO == PRO_GAIN) {
-                const uint4 gq = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
-                const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq);
+              for (int i = 0; i < 8; ++i) v[i] = 0.f;
+              float sq = 0.f;
+              if (r < g.R && k < g.K) {
+                const float4 a0 = __ldcg(reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k));   // L2 only: other CTAs wrote these
+                const float4 a1 = __ldcg(reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k + 4));
+                v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+                if (pro == PRO_GAIN) {
+                  const uint4 gq = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
+                  const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float2 gf = __bfloat1622float2(gp[i]);
-                  sq = fmaf(v[2 * i], v[2 * i], sq); sq = fmaf(v[2 * i + 1], v[2 * i + 1], sq);
-                  v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
-                }
-              } else if (PRO == PRO_SILU_MUL) {
-                const float sr = rsqrtf(__ldg(g.ss_in + r) / (float)g.dn + g.eps);
-                const float4 u0 = *reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k);
-                const float4 u1 = *reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k + 4);
-                const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+                  for (int i = 0; i < 4; ++i) {
+                    const float2 gf = __bfloat1622float2(gp[i]);
+                    sq = fmaf(v[2 * i], v[2 * i], sq); sq = fmaf(v[2 * i + 1], v[2 * i + 1], sq);
+                    v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
+                  }
+                } else if (pro == PRO_SILU_MUL) {
+                  const float sr = rsqrtf(__ldcg(g.ss_in + r) / (float)g.dn + g.eps);
+                  const float4 u0 = __ldcg(reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k));
+                  const float4 u1 = __ldcg(reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k + 4));
+                  const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  const float gt = sr * v[i];
-                  v[i] = (gt / (1.0f + __expf(-gt))) * (sr * uu[i]);
+                  for (int i = 0; i < 8; ++i) {
+                    const float gt = sr * v[i];
+                    v[i] = (gt / (1.0f + __expf(-gt))) * (sr * uu[i]);
+                  }
                 }
               }
+              if (need_ss) {      // uniform across the warp
+                sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+                sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+                sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+                if (chunk == 0) my_ss[row] += sq;
+              }
+              uint4 pk;
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
+              pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+              pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+              *reinterpret_cast<uint4 *>(xs + (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
             }
-            if (need_ss) {      // uniform across the warp
-              sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-              sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-              sq += __shfl_xor_sync(0xffffffffu, sq, 4);
-              if (chunk == 0) my_ss[row] += sq;
-            }
-            uint4 pk;
-            __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
-            pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
-            pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
-            *reinterpret_cast<uint4 *>(xs + (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&full_x[stage]));
           }
-          fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&full_x[stage]));
-        }
-        if (!ok) break;
-        if (need_ss) {
-          __syncwarp();
-          if (EPI == EPI_ARGMAX) {
-            if (lane == 0) mbar_arrive(smem_u32(&ss_ready[acc]));
-          } else {
-            for (int row = lane; row < BN; row += 32) {
-              const int r = rb * BN + row;
-              if (r < g.R) atomicAdd(&g.ss_out[r], my_ss[row]);
+          if (!ok) break;
+          if (need_ss) {
+            __syncwarp();
+            if (EPI == EPI_ARGMAX) {
+              if (lane == 0) mbar_arrive(smem_u32(&ss_ready[acc]));
+            } else {
+              for (int row = lane; row < BN; row += 32) {
+                const int r = rb * BN + row;
+                if (r < g.R) atomicAdd(&g.ss_out[r], my_ss[row]);
+              }
             }
           }
+          ++seg;
         }
-        ++seg;
       }
+      // this warp has finished reading the phase's inputs and adding its sums of squares
+      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, lane);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -394,48 +455,54 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map0, const __grid_constant
     const int n_local = q * 32 + lane;
     int seg = 0;
     bool ok = true;
-    for (int rb = 0; rb < nrb && ok; ++rb) {
-      SegIter si(p);
-      Segment s;
-      while (ok && si.next(s)) {
-        int m, row0, rows_valid, ycol0;
-        tile_info(p, s.tile, m, row0, rows_valid, ycol0);
-        const int acc = seg & 1;
-        const uint32_t ph = ((uint32_t)seg >> 1) & 1u;
-        if (!mbar_wait_warp(smem_u32(&accum_full[acc]), ph, abort_flag)) { ok = false; break; }
-        if (EPI == EPI_ARGMAX && !mbar_wait_warp(smem_u32(&ss_ready[acc]), ph, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const bool valid = n_local < rows_valid;
-        const int col = ycol0 + n_local;
-        for (int c0 = 0; c0 < BN; c0 += 16) {
-          if (rb * BN + c0 >= g.R) break;
-          float v[16];
-          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
+    for (int pi = 0; pi < p.n_phases && ok; ++pi) {
+      const PhaseDesc &P = p.ph[pi];
+      const GemmArgs &g = P.g;
+      for (int rb = 0; rb < nrb && ok; ++rb) {
+        SegIter si(P, p.tile_mode);
+        Segment s;
+        while (ok && si.next(s)) {
+          int m, row0, rows_valid, ycol0;
+          tile_info(P, s.tile, m, row0, rows_valid, ycol0);
+          const int acc = seg & 1;
+          const uint32_t ph = ((uint32_t)seg >> 1) & 1u;
+          if (!mbar_wait_warp(smem_u32(&accum_full[acc]), ph, abort_flag)) { ok = false; break; }
+          if (EPI == EPI_ARGMAX && !mbar_wait_warp(smem_u32(&ss_ready[acc]), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const bool valid = n_local < rows_valid;
+          const int col = ycol0 + n_local;
+          for (int c0 = 0; c0 < BN; c0 += 16) {
+            if (rb * BN + c0 >= g.R) break;
+            float v[16];
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int r = rb * BN + c0 + j;
-            if (r >= g.R) break;
-            if (EPI == EPI_ATOMIC_ADD) {
-              if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
-            } else {
-              const float ssum = ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
-              float logit = v[j] * rsqrtf(ssum / (float)g.dn + g.eps);
-              unsigned long long key = 0ull;
-              if (valid) {
-                if (g.perm && g.perm[g.tokens[r]] == col) logit += g.beta;
-                if (g.logits) g.logits[(long long)r * g.vocab + col] = logit;
-                key = ((unsigned long long)ordered_key_u(logit) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned int)col);
+            for (int j = 0; j < 16; ++j) {
+              const int r = rb * BN + c0 + j;
+              if (r >= g.R) break;
+              if (EPI == EPI_ATOMIC_ADD) {
+                if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
+              } else {
+                const float ssum = ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
+                float logit = v[j] * rsqrtf(ssum / (float)g.dn + g.eps);
+                unsigned long long key = 0ull;
+                if (valid) {
+                  if (g.perm && g.perm[g.tokens[r]] == col) logit += g.beta;
+                  if (g.logits) g.logits[(long long)r * g.vocab + col] = logit;
+                  key = ((unsigned long long)ordered_key_u(logit) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned int)col);
+                }
+                key = warp_max_u64(key);
+                if (lane == 0) atomicMax(&g.amax[r], key);
               }
-              key = warp_max_u64(key);
-              if (lane == 0) atomicMax(&g.amax[r], key);
             }
           }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[acc]));
+          ++seg;
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[acc]));
-        ++seg;
       }
+      // all partial sums of this phase that this warp owns are on their way to L2
+      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, lane);
     }
   }
 
@@ -483,6 +550,7 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
+// accumulator width, ring depth and resident CTAs per SM for a row count
 static void bn_config(int R, int &bn, int &stages, int &ctas_per_sm) {
   if (R <= 16) { bn = 16; stages = 6; ctas_per_sm = 2; }
   else if (R <= 32) { bn = 32; stages = 5; ctas_per_sm = 2; }
@@ -500,17 +568,17 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
   if (a.n_mats < 1 || a.n_mats > kMaxMats) return fail("bad matrix count");
   UmmaPlan *pl = new UmmaPlan();
   memset(pl, 0, sizeof(*pl));
-  pl->p.g = a;
-  pl->pro = pro; pl->epi = epi; pl->n_sms = n_sms; pl->err = err_word;
-  pl->p.err = err_word;
-  pl->p.nkb = (a.K + kTileK - 1) / kTileK;
-  pl->p.n_tiles = 0;
+  pl->d.g = a;
+  pl->d.pro = pro;
+  pl->epi = epi; pl->n_sms = n_sms; pl->err = err_word;
+  pl->d.nkb = (a.K + kTileK - 1) / kTileK;
+  pl->d.n_tiles = 0;
   for (int m = 0; m < a.n_mats; ++m) {
     if (a.n_rows[m] < 1) { delete pl; return fail("empty weight matrix"); }
-    pl->p.tiles_m[m] = (a.n_rows[m] + kTileM - 1) / kTileM;
-    pl->p.n_tiles += pl->p.tiles_m[m];
+    pl->d.tiles_m[m] = (a.n_rows[m] + kTileM - 1) / kTileM;
+    pl->d.n_tiles += pl->d.tiles_m[m];
     const cuuint32_t box_rows = (cuuint32_t)(a.n_rows[m] < kTileM ? a.n_rows[m] : kTileM);
-    pl->p.tx_bytes[m] = (int)(box_rows * kTileK * 2);
+    pl->d.tx_bytes[m] = (int)(box_rows * kTileK * 2);
     cuuint64_t gdim[2] = {(cuuint64_t)a.K, (cuuint64_t)a.n_rows[m]};
     cuuint64_t gstr[1] = {(cuuint64_t)a.K * 2};
     cuuint32_t box[2] = {(cuuint32_t)kTileK, box_rows};
@@ -521,20 +589,19 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
     if (r != CUDA_SUCCESS) { delete pl; return fail("cuTensorMapEncodeTiled failed (weight pointer must be 16-byte aligned)"); }
   }
   for (int m = a.n_mats; m < kMaxMats; ++m) pl->maps[m] = pl->maps[0];
-  pl->p.items_per_cta_mode = (epi == EPI_ARGMAX) ? 1 : 0;
   return pl;
 }
 
 void umma_plan_destroy(UmmaPlan *p) { delete p; }
 
-template <int PRO, int EPI, int BN>
-static cudaError_t launch_one(const UmmaPlan *pl, const UmmaParams &p, int grid, cudaStream_t st) {
+template <int EPI, int BN>
+static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid, cudaStream_t st) {
   const size_t smem = (size_t)p.stages * (kWBytes + BN * 128) + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<PRO, EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  static size_t attr_smem = 0;
+  if (smem > attr_smem) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_smem = smem;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -543,40 +610,65 @@ static cudaError_t launch_one(const UmmaPlan *pl, const UmmaParams &p, int grid,
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = p.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<PRO, EPI, BN>, pl->maps[0], pl->maps[1], pl->maps[2], p);
+  return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<EPI, BN>, maps, p);
 }
 
-template <int PRO, int EPI>
-static cudaError_t launch_bn(const UmmaPlan *pl, const UmmaParams &p, int bn, int grid, cudaStream_t st) {
+template <int EPI>
+static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, int grid, cudaStream_t st) {
   switch (bn) {
-    case 16: return launch_one<PRO, EPI, 16>(pl, p, grid, st);
-    case 32: return launch_one<PRO, EPI, 32>(pl, p, grid, st);
-    case 64: return launch_one<PRO, EPI, 64>(pl, p, grid, st);
-    case 128: return launch_one<PRO, EPI, 128>(pl, p, grid, st);
-    default: return launch_one<PRO, EPI, 256>(pl, p, grid, st);
+    case 16: return launch_one<EPI, 16>(maps, p, grid, st);
+    case 32: return launch_one<EPI, 32>(maps, p, grid, st);
+    case 64: return launch_one<EPI, 64>(maps, p, grid, st);
+    case 128: return launch_one<EPI, 128>(maps, p, grid, st);
+    default: return launch_one<EPI, 256>(maps, p, grid, st);
   }
+}
+
+// One launch that runs plans[0..n-1] back to back on the same rows; plan i+1 consumes what plan i reduced
+// into its output, separated by a grid barrier on bar[i] (zero at launch).  args[i] carries the per-launch
+// buffers and the row count; weights, K and the matrix split stay as planned.
+cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar, int pdl,
+                              cudaStream_t st) {
+  if (n < 1 || n > kMaxPhases) return cudaErrorInvalidValue;
+  if (n > 1 && !bar) return cudaErrorInvalidValue;
+  MapPack maps;
+  UmmaParams p;
+  memset(&p, 0, sizeof p);
+  const int epi = plans[0]->epi;
+  long long max_items = 1;
+  int max_tiles = 1;
+  for (int i = 0; i < n; ++i) {
+    const UmmaPlan *pl = plans[i];
+    const GemmArgs &a = args[i];
+    if (pl->epi != epi || (epi == EPI_ARGMAX && n != 1) || a.R != args[0].R) return cudaErrorInvalidValue;
+    PhaseDesc &d = p.ph[i];
+    d = pl->d;
+    d.g.x = a.x; d.g.x2 = a.x2; d.g.ldx = a.ldx; d.g.ss_in = a.ss_in; d.g.ss_out = a.ss_out;
+    d.g.y = a.y; d.g.ldy = a.ldy; d.g.R = a.R; d.g.tokens = a.tokens; d.g.amax = a.amax; d.g.logits = a.logits;
+    for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = pl->maps[m];
+    const long long W = (long long)d.n_tiles * d.nkb;
+    if (W > max_items) max_items = W;
+    if (d.n_tiles > max_tiles) max_tiles = d.n_tiles;
+  }
+  for (int i = n; i < kMaxPhases; ++i)
+    for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = plans[0]->maps[0];
+  p.n_phases = n; p.pdl = pdl; p.err = plans[0]->err; p.bar = bar;
+  p.tile_mode = (epi == EPI_ARGMAX) ? 1 : 0;
+  int bn, cps;
+  bn_config(args[0].R, bn, p.stages, cps);
+  // Staging warps own every fourth k-block and run ahead of each other; the parity waits on the ring
+  // are only unambiguous while the ring is at least as deep as the number of staging warps.
+  if (p.stages < 4 || p.stages > 8) return cudaErrorInvalidValue;
+  const long long resident = (long long)plans[0]->n_sms * cps;     // the grid barrier needs every CTA resident
+  int grid;
+  if (p.tile_mode == 0) grid = (int)(resident < max_items ? resident : max_items);
+  else grid = (int)(resident < max_tiles ? resident : max_tiles);
+  if (epi == EPI_ARGMAX) return launch_bn<EPI_ARGMAX>(maps, p, bn, grid, st);
+  return launch_bn<EPI_ATOMIC_ADD>(maps, p, bn, grid, st);
 }
 
 cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, int pdl, cudaStream_t st) {
-  UmmaParams p = pl->p;
-  // per-launch fields (buffers and row count); weights, K and the matrix split stay as planned
-  p.g.x = a.x; p.g.x2 = a.x2; p.g.ldx = a.ldx; p.g.ss_in = a.ss_in; p.g.ss_out = a.ss_out;
-  p.pdl = pdl;
-  p.g.y = a.y; p.g.ldy = a.ldy; p.g.R = a.R; p.g.tokens = a.tokens; p.g.amax = a.amax; p.g.logits = a.logits;
-  int bn, cps;
-  bn_config(a.R, bn, p.stages, cps);
-  int grid;
-  if (p.items_per_cta_mode == 0) {
-    const long long W = (long long)p.n_tiles * p.nkb;
-    long long cap = W / 4 > 0 ? W / 4 : 1;
-    grid = (int)((long long)pl->n_sms * cps < cap ? (long long)pl->n_sms * cps : cap);
-  } else {
-    grid = p.n_tiles < pl->n_sms * cps ? p.n_tiles : pl->n_sms * cps;
-  }
-  if (pl->epi == EPI_ARGMAX) return launch_bn<PRO_GAIN, EPI_ARGMAX>(pl, p, bn, grid, st);
-  if (pl->pro == PRO_NONE) return launch_bn<PRO_NONE, EPI_ATOMIC_ADD>(pl, p, bn, grid, st);
-  if (pl->pro == PRO_GAIN) return launch_bn<PRO_GAIN, EPI_ATOMIC_ADD>(pl, p, bn, grid, st);
-  return launch_bn<PRO_SILU_MUL, EPI_ATOMIC_ADD>(pl, p, bn, grid, st);
+  return launch_gemm_chain(&pl, &a, 1, nullptr, pdl, st);
 }
 
 }  // namespace fc
