@@ -167,10 +167,15 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
 // Grid barrier between two phases of a chained launch.  Every CTA of the grid is resident (the grid is
 // sized to the SM count times the CTAs that fit per SM), so the wait ends; it is bounded all the same.
 // signal: each participating warp calls it once after its last global write of the phase.
-__device__ __forceinline__ void grid_bar_signal(unsigned int *ctr, int lane) {
+// The kWarpsSignalling warps of a CTA count up in shared memory; the last one posts the CTA's single arrival.
+constexpr unsigned int kWarpsSignalling = 8;    // 4 staging + 4 epilogue warps
+__device__ __forceinline__ void grid_bar_signal(unsigned int *ctr, unsigned int *cta_count, int lane) {
   __threadfence();
   __syncwarp();
-  if (lane == 0) atomicAdd(ctr, 1u);
+  if (lane == 0 && atomicAdd(cta_count, 1u) == kWarpsSignalling - 1u) {
+    __threadfence();
+    atomicAdd(ctr, 1u);
+  }
 }
 __device__ __forceinline__ bool grid_bar_wait(const unsigned int *ctr, unsigned int target, int lane,
                                               volatile int *abort_flag) {
@@ -244,10 +249,10 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   constexpr int kStageBytes = kWBytes + BN * 128;
   constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
   constexpr uint32_t kIdesc = make_idesc(BN);
-  constexpr unsigned int kSignalsPerCta = 8;    // 4 staging + 4 epilogue warps signal each grid barrier
 
   extern __shared__ unsigned char smem_dyn[];
-  __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar;
+  __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar, go_bar[kMaxPhases];
+  __shared__ unsigned int bar_cnt_s[kMaxPhases];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   __shared__ float ss_part[2][4][BN];   // per accumulator, per staging warp: partial sums of squares
@@ -264,6 +269,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&full_w[i]), 1); mbar_init(smem_u32(&full_x[i]), 1); mbar_init(smem_u32(&empty_b[i]), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
     mbar_init(smem_u32(&drain_bar), 1);
+    for (int i = 0; i < kMaxPhases; ++i) { mbar_init(smem_u32(&go_bar[i]), 1); bar_cnt_s[i] = 0u; }
     fence_barrier_init();
   }
   if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), kCols);
@@ -358,7 +364,16 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       const GemmArgs &g = P.g;
       const int pro = P.pro;
       // the activations of this phase are the previous phase's outputs, reduced by every CTA of the grid
-      if (pi > 0 && !grid_bar_wait(p.bar + (pi - 1), gridDim.x * kSignalsPerCta, lane, abort_flag)) { ok = false; break; }
+      // (one staging warp polls the grid-wide counter and releases the other three through shared memory)
+      if (pi > 0) {
+        if (sw == 0) {
+          ok = grid_bar_wait(p.bar + (pi - 1), gridDim.x, lane, abort_flag);
+          if (ok && lane == 0) mbar_arrive(smem_u32(&go_bar[pi - 1]));
+        } else {
+          ok = mbar_wait_warp(smem_u32(&go_bar[pi - 1]), 0u, abort_flag);
+        }
+        if (!ok) break;
+      }
       for (int rb = 0; rb < nrb && ok; ++rb) {
         SegIter si(P, p.tile_mode);
         Segment s;
@@ -380,20 +395,37 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
             unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
             const int k = kb * kTileK + chunk * 8;
-#pragma unroll 4
-            for (int u = 0; u < kUW; ++u) {
-              const int row = u * 4 + (lane >> 3);
-              const int r = rb * BN + row;
-              float v[8];
+            // Loads first, arithmetic and shared-memory stores after: a store between two units would keep the
+            // compiler from hoisting the next unit's loads, and every unit would pay its own L2 round trip.
+            const bool k_in = k < g.K;
+            uint4 gq = make_uint4(0, 0, 0, 0);
+            if (pro == PRO_GAIN && k_in) gq = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
+            for (int ub = 0; ub < kUW; ub += 4) {
+              float4 xa[4], xb[4], ua[4], ubv[4];
+              float ssr[4];
 #pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = 0.f;
-              float sq = 0.f;
-              if (r < g.R && k < g.K) {
-                const float4 a0 = __ldcg(reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k));   // L2 only: other CTAs wrote these
-                const float4 a1 = __ldcg(reinterpret_cast<const float4 *>(g.x + (long long)r * g.ldx + k + 4));
-                v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+              for (int j = 0; j < 4; ++j) {
+                const int r = rb * BN + (ub + j) * 4 + (lane >> 3);
+                xa[j] = xb[j] = ua[j] = ubv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                ssr[j] = 0.f;
+                if (r < g.R && k_in) {
+                  const float *px = g.x + (long long)r * g.ldx + k;
+                  xa[j] = __ldcg(reinterpret_cast<const float4 *>(px));        // L2 only: other CTAs wrote these
+                  xb[j] = __ldcg(reinterpret_cast<const float4 *>(px + 4));
+                  if (pro == PRO_SILU_MUL) {
+                    const float *pu = g.x2 + (long long)r * g.ldx + k;
+                    ua[j] = __ldcg(reinterpret_cast<const float4 *>(pu));
+                    ubv[j] = __ldcg(reinterpret_cast<const float4 *>(pu + 4));
+                    ssr[j] = __ldcg(g.ss_in + r);
+                  }
+                }
+              }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int row = (ub + j) * 4 + (lane >> 3);
+                float v[8] = {xa[j].x, xa[j].y, xa[j].z, xa[j].w, xb[j].x, xb[j].y, xb[j].z, xb[j].w};
+                float sq = 0.f;
                 if (pro == PRO_GAIN) {
-                  const uint4 gq = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
                   const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq);
 #pragma unroll
                   for (int i = 0; i < 4; ++i) {
@@ -402,29 +434,27 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
                     v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
                   }
                 } else if (pro == PRO_SILU_MUL) {
-                  const float sr = rsqrtf(__ldcg(g.ss_in + r) / (float)g.dn + g.eps);
-                  const float4 u0 = __ldcg(reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k));
-                  const float4 u1 = __ldcg(reinterpret_cast<const float4 *>(g.x2 + (long long)r * g.ldx + k + 4));
-                  const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+                  const float sr = rsqrtf(ssr[j] / (float)g.dn + g.eps);
+                  const float uu[8] = {ua[j].x, ua[j].y, ua[j].z, ua[j].w, ubv[j].x, ubv[j].y, ubv[j].z, ubv[j].w};
 #pragma unroll
                   for (int i = 0; i < 8; ++i) {
                     const float gt = sr * v[i];
-                    v[i] = (gt / (1.0f + __expf(-gt))) * (sr * uu[i]);
+                    v[i] = __fdividef(gt, 1.0f + __expf(-gt)) * (sr * uu[i]);
                   }
                 }
+                if (need_ss) {      // uniform across the warp
+                  sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+                  sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+                  sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+                  if (chunk == 0) my_ss[row] += sq;
+                }
+                uint4 pk;
+                __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
+                __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
+                pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+                pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+                *reinterpret_cast<uint4 *>(xs + (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
               }
-              if (need_ss) {      // uniform across the warp
-                sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-                sq += __shfl_xor_sync(0xffffffffu, sq, 2);
-                sq += __shfl_xor_sync(0xffffffffu, sq, 4);
-                if (chunk == 0) my_ss[row] += sq;
-              }
-              uint4 pk;
-              __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
-              __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
-              pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
-              pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
-              *reinterpret_cast<uint4 *>(xs + (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
             }
             fence_proxy_async();
             __syncwarp();
@@ -446,7 +476,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
       }
       // this warp has finished reading the phase's inputs and adding its sums of squares
-      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, lane);
+      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -502,7 +532,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
       }
       // all partial sums of this phase that this warp owns are on their way to L2
-      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, lane);
+      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
     }
   }
 
