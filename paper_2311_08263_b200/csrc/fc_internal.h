@@ -98,6 +98,7 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   unsigned int *counters; // [batch*hkv], zero on entry and on exit
   unsigned int *grid_counter;   // one word, zero on entry and on exit
   int pdl;                // launched as a programmatic dependent of the previous kernel
+  int cluster;            // set by the launcher: the nsplit CTAs of one kv head form one thread-block cluster
   float *out;             // [R, hq*hd] fp32
   ZeroList z;
 };

@@ -131,22 +131,35 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   const int g4 = lane >> 2, t4 = lane & 3;
   for (int qt = 0; qt < nqt; ++qt) {
     __syncthreads();                                          // K/V staged; previous tile's Qs/Om/mls free
-    // ---- Q tile: 1/rms, rotation, bf16
-    for (int e = tid; e < 16 * HALF; e += kAttnThreads) {
-      const int row = e / HALF, i = e % HALF;
-      const int qrow = qt * 16 + row;
-      __nv_bfloat16 o0 = __float2bfloat16_rn(0.f), o1 = o0;
-      if (qrow < nq) {
-        const int g = div_c(qrow), j = qrow - g * a.c;
-        const int r = bl * a.c + j, h = kvh * group + g;
-        const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
-        const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
-        const float2 rot = __ldg(a.rope + (long long)(L + j) * HALF + i);
-        const float cs = rot.x, sn = rot.y;
-        const float x0 = qacc[i] * s, x1 = qacc[i + HALF] * s;
-        o0 = __float2bfloat16_rn(x0 * cs - x1 * sn); o1 = __float2bfloat16_rn(x0 * sn + x1 * cs);
+    // ---- Q tile: 1/rms, rotation, bf16.  A thread keeps one pair index i and walks the rows; all of its
+    // loads are issued before the first use so that they share one trip to L2.
+    {
+      constexpr int RPI = kAttnThreads / HALF;               // rows covered per pass
+      constexpr int NIT = 16 / RPI;
+      const int i = tid % HALF, rsub = tid / HALF;
+      float x0[NIT], x1[NIT], ssv[NIT];
+      float2 rot[NIT];
+#pragma unroll
+      for (int it = 0; it < NIT; ++it) {
+        const int qrow = qt * 16 + rsub + it * RPI;
+        x0[it] = x1[it] = 0.f; ssv[it] = 0.f; rot[it] = make_float2(1.f, 0.f);
+        if (qrow < nq) {
+          const int g = div_c(qrow), j = qrow - g * a.c;
+          const int r = bl * a.c + j, h = kvh * group + g;
+          const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
+          ssv[it] = __ldcg(a.ss + r);
+          x0[it] = __ldcg(qacc + i); x1[it] = __ldcg(qacc + i + HALF);
+          rot[it] = __ldg(a.rope + (long long)(L + j) * HALF + i);
+        }
       }
-      Qs[row * LD + i] = o0; Qs[row * LD + i + HALF] = o1;
+#pragma unroll
+      for (int it = 0; it < NIT; ++it) {
+        const int row = rsub + it * RPI;
+        const float sc = rsqrtf(ssv[it] / (float)a.dn + a.eps);
+        const float a0 = x0[it] * sc, a1 = x1[it] * sc;
+        Qs[row * LD + i] = __float2bfloat16_rn(a0 * rot[it].x - a1 * rot[it].y);
+        Qs[row * LD + i + HALF] = __float2bfloat16_rn(a0 * rot[it].y + a1 * rot[it].x);
+      }
     }
     __syncthreads();
 
@@ -257,15 +270,20 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       *reinterpret_cast<float2 *>(o1) = make_float2(oacc[d][2] * fac[1], oacc[d][3] * fac[1]);
     }
     __syncthreads();
-    for (int e = tid; e < 16 * HD; e += kAttnThreads) {
-      const int row = e / HD, dd = e % HD;
+    for (int e = tid; e < 16 * (HD / 4); e += kAttnThreads) {
+      const int row = e / (HD / 4), d4 = e % (HD / 4);
       const int qrow = qt * 16 + row;
       if (qrow >= nq) continue;
       const int g = div_c(qrow), j = qrow - g * a.c;
       const int r = bl * a.c + j, h = kvh * group + g;
       const long long pidx = ((long long)r * a.hq + h) * a.nsplit + split;
-      a.part_o[pidx * HD + dd] = Om[row * HD + dd] + Om[(16 + row) * HD + dd] + Om[(32 + row) * HD + dd] + Om[(48 + row) * HD + dd];
-      if (dd == 0) {
+      const float4 p0 = *reinterpret_cast<const float4 *>(Om + row * HD + d4 * 4);
+      const float4 p1 = *reinterpret_cast<const float4 *>(Om + (16 + row) * HD + d4 * 4);
+      const float4 p2 = *reinterpret_cast<const float4 *>(Om + (32 + row) * HD + d4 * 4);
+      const float4 p3 = *reinterpret_cast<const float4 *>(Om + (48 + row) * HD + d4 * 4);
+      *reinterpret_cast<float4 *>(a.part_o + pidx * HD + d4 * 4) =
+          make_float4(p0.x + p1.x + p2.x + p3.x, p0.y + p1.y + p2.y + p3.y, p0.z + p1.z + p2.z + p3.z, p0.w + p1.w + p2.w + p3.w);
+      if (d4 == 0) {
         float M = -INFINITY;
         for (int w = 0; w < 4; ++w) M = fmaxf(M, mls[(w * 16 + row) * 2]);
         float lsum = 0.f;
@@ -273,22 +291,36 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
           const float mw = mls[(w * 16 + row) * 2];
           if (mw != -INFINITY) lsum += mls[(w * 16 + row) * 2 + 1] * __expf(mw - M);
         }
-        a.part_ml[pidx * 2] = M; a.part_ml[pidx * 2 + 1] = lsum;
+        *reinterpret_cast<float2 *>(a.part_ml + pidx * 2) = make_float2(M, lsum);
       }
     }
   }
 
-  // ---- last CTA of this (sequence, kv head): merge the splits, clear the accumulators of its heads
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned int prev = atomicAdd(&a.counters[b * a.hkv + kvh], 1u);
-    s_last = (prev == (unsigned int)a.nsplit - 1u);
+  // ---- merge the splits of this (sequence, kv head) and clear the accumulators of its heads.
+  // Cluster launch (the splits of one kv head form one thread-block cluster): a hardware cluster barrier, then
+  // every CTA of the cluster merges its share of the queries.  Otherwise the last CTA to arrive merges them all.
+  int q_first, q_step;
+  unsigned int ctas_counted;
+  if (a.cluster) {
+    __threadfence();
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    q_first = split * 4 + warp; q_step = a.nsplit * 4;
+    ctas_counted = gridDim.x * gridDim.y * gridDim.z;
+  } else {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      const unsigned int prev = atomicAdd(&a.counters[b * a.hkv + kvh], 1u);
+      s_last = (prev == (unsigned int)a.nsplit - 1u);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    q_first = warp; q_step = 4;
+    ctas_counted = gridDim.y * gridDim.z;
   }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  for (int qi = warp; qi < nq; qi += 4) {
+  for (int qi = q_first; qi < nq; qi += q_step) {
     const int g = div_c(qi), j = qi - g * a.c;
     const int r = bl * a.c + j, h = kvh * group + g;
     const long long base = ((long long)r * a.hq + h) * a.nsplit;
@@ -334,10 +366,12 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       for (int i = lane; i < HD; i += 32) { kacc[i] = 0.f; kacc[kvd + i] = 0.f; }
     }
   }
+  // the last CTA (of those counted) clears the per-row sums of squares: every reader is done by then
+  __syncthreads();
   if (tid == 0) {
-    a.counters[b * a.hkv + kvh] = 0u;
+    if (!a.cluster) a.counters[b * a.hkv + kvh] = 0u;
     const unsigned int prev = atomicAdd(a.grid_counter, 1u);
-    s_last_grid = (prev == (unsigned int)(gridDim.y * gridDim.z) - 1u);
+    s_last_grid = (prev == ctas_counted - 1u);
   }
   __syncthreads();
   if (s_last_grid) {
@@ -360,11 +394,22 @@ static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3(a.nsplit, a.hkv, a.nb); cfg.blockDim = dim3(kAttnThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = a.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, attn_fused_kernel<HD>, a);
+  cudaLaunchAttribute attr[2];
+  int na = 0;
+  if (a.pdl) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  FusedAttnArgs args = a;
+  args.cluster = (a.nsplit >= 2 && a.nsplit <= 8) ? 1 : 0;     // portable cluster size
+  if (args.cluster) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = (unsigned)a.nsplit; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr; cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, attn_fused_kernel<HD>, args);
 }
 
 cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st) {
