@@ -124,7 +124,8 @@ int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen);
 /* Enqueue `n_steps` iterations back to back with no host round trip in between and return the
  * device time in milliseconds from the first to the last kernel (CUDA events on the context's
  * stream).  commit != 0: every step commits its accepted tokens on the device (needs
- * kv_len + n_steps * c <= max_seq); host mirrors are refreshed afterwards and *tokens_out (nullable)
+ * kv_len + n_steps * c <= max_seq; every eighth step the host re-reads kv_len to size the attention grid);
+ * host mirrors are refreshed afterwards and *tokens_out (nullable)
  * gets the tokens committed over all sequences.  commit == 0: kv_len, n_gen and the window are left
  * untouched, so every step runs at the same K/V length (latency sweeps). */
 int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, int32_t commit, float *ms_total, int64_t *tokens_out);

@@ -635,11 +635,21 @@ extern "C" int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, int32_t commit, floa
   for (int b = 0; b < B; ++b)
     if (ctx->kv_len_h[b] + growth > ctx->s.max_seq) return FC_ERR_CAPACITY;
   ctx->launches = 0;
-  const int maxlen = max_live_len(ctx);
+  int maxlen = max_live_len(ctx);
+  int32_t *p_kv = ctx->pin;
   FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
-  for (int i = 0; i < n_steps; ++i) {
-    // committed steps grow the cache by at most c tokens each: size the split count for that bound
-    int rc = forward(ctx, 0, B, c, ctx->b.window, true, commit ? maxlen + i * c : maxlen, commit ? 1 : 0);
+  for (int i = 0, since = 0; i < n_steps; ++i, ++since) {
+    // Committed steps grow each cache by at most c tokens.  The host needs an upper bound on kv_len to size
+    // the attention grid, so the bound grows by c per enqueued step and is refreshed from the device every
+    // eighth step (one small copy; the steps in between are enqueued without any host round trip).
+    if (commit && since == 8) {
+      FC_CK(cudaMemcpyAsync(p_kv, ctx->b.kv_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, ctx->st));
+      FC_CK(cudaStreamSynchronize(ctx->st));
+      maxlen = 0;
+      for (int b = 0; b < B; ++b) maxlen = p_kv[b] > maxlen ? p_kv[b] : maxlen;
+      since = 0;
+    }
+    int rc = forward(ctx, 0, B, c, ctx->b.window, true, commit ? maxlen + since * c : maxlen, commit ? 1 : 0);
     if (rc != FC_OK) return rc;
   }
   FC_CK(cudaEventRecord(ctx->ev1, ctx->st));
@@ -647,7 +657,7 @@ extern "C" int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, int32_t commit, floa
   FC_CK(cudaEventElapsedTime(ms_total, ctx->ev0, ctx->ev1));
   if (tokens_out) *tokens_out = 0;
   if (commit) {
-    int32_t *p_kv = ctx->pin, *p_ng = p_kv + B, *p_win = p_ng + B;   // pin holds B * (1 + 2c) + 4 ints
+    int32_t *p_ng = p_kv + B, *p_win = p_ng + B;   // pin holds B * (1 + 2c) + 4 ints
     FC_CK(cudaMemcpyAsync(p_kv, ctx->b.kv_len, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, ctx->st));
     FC_CK(cudaMemcpyAsync(p_ng, ctx->b.n_gen, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, ctx->st));
     FC_CK(cudaMemcpyAsync(p_win, ctx->b.window, sizeof(int32_t) * B * c, cudaMemcpyDeviceToHost, ctx->st));
