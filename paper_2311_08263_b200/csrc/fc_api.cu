@@ -72,7 +72,9 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
   t.gu = c.take<float>(R * 2 * (size_t)s->d_ffn);
   t.ss_attn = c.take<float>(R);
   t.ss_ffn = c.take<float>(R);
-  t.chain_bar = c.take<unsigned int>((size_t)s->n_layers * 4);   // directly after the sums of squares: cleared with them
+  // eight words per layer (three grid barriers, four work-claim counters) plus one group for the first QKV
+  // and the LM head; directly after the sums of squares so that one pass clears them all
+  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * 8);
   t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
   t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
   t.rope = c.take<float2>((size_t)s->max_seq * (s->head_dim / 2));
@@ -309,11 +311,22 @@ struct ProfScope {
   ~ProfScope() { prof_mark(c, cls, false); }
 };
 
-static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls) {
+// Work-claim counter of a projection (cleared by the embed kernel at the start of every forward).
+enum { GEMM_QKV = -1, GEMM_O = 0, GEMM_GU = 1, GEMM_DOWN = 2, GEMM_HEAD = 3 };
+static unsigned int *claim_word(fc_ctx *ctx, int l, int which) {
+  const int L = ctx->s.n_layers;
+  unsigned int *w = ctx->b.chain_bar;
+  if (which == GEMM_HEAD) return w + (size_t)L * 8 + 5;
+  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * 8 + 4 : w + (size_t)(l - 1) * 8 + 7;   // chained after down(l-1)
+  return w + (size_t)l * 8 + 4 + which;
+}
+
+static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls,
+                            unsigned int *claim) {
   ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
-  if (ctx->use_umma) return launch_gemm_umma(plan, a, ctx->pdl && !ctx->prof, ctx->st);
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, ctx->pdl && !ctx->prof, ctx->st);
   return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
 }
 
@@ -331,7 +344,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   ea.z.p[1] = ctx->b.gu; ea.z.n[1] = Rz * 2 * s.d_ffn;
   // sums of squares (both norms) and the grid-barrier words of the chained projections are adjacent
   ea.z.p[2] = ctx->b.ss_attn;
-  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + (size_t)s.n_layers * 4) - (char *)ctx->b.ss_attn) / sizeof(float);
+  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + ((size_t)s.n_layers + 1) * 8) - (char *)ctx->b.ss_attn) / sizeof(float);
   ++ctx->launches;
   { ProfScope ps(ctx, FC_CLS_EMBED); FC_CK(launch_embed(ea, s.dtype, ctx->st)); }
 
@@ -341,7 +354,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   const bool chained = ctx->chain && !ctx->prof;
   for (int l = 0; l < s.n_layers; ++l) {
     if (!chained || l == 0)
-      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV, claim_word(ctx, l, GEMM_QKV)));
     void *kc = ctx->kv + (size_t)l * ctx->kv_layer_stride;
     void *vc = ctx->kv + (size_t)l * ctx->kv_layer_stride + ctx->kv_half_stride;
     if (ctx->fused_attn) {
@@ -385,17 +398,19 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       if (l + 1 < s.n_layers) { plans[3] = ctx->plan_qkv[l + 1]; ga[3] = args_qkv(ctx, l + 1); n = 4; }
       for (int i = 0; i < n; ++i) ga[i].R = R;
       ++ctx->launches;
-      FC_CK(launch_gemm_chain(plans, ga, n, ctx->b.chain_bar + (size_t)l * 4, ctx->pdl, ctx->st));
+      // barriers at words 0..2 of the layer's group, claim counters at 4..7 (O, gate/up, down, next QKV)
+      FC_CK(launch_gemm_chain(plans, ga, n, ctx->b.chain_bar + (size_t)l * 8, ctx->b.chain_bar + (size_t)l * 8 + 4,
+                              ctx->pdl, ctx->st));
     } else {
-      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ));
-      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP));
-      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O)));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN, claim_word(ctx, l, GEMM_DOWN)));
     }
   }
   if (with_head) {
     GemmArgs ha = args_head(ctx);
     ha.tokens = tokens;
-    FC_CK(run_gemm(ctx, ctx->plan_head, ha, R, PRO_GAIN, EPI_ARGMAX, FC_CLS_HEAD));
+    FC_CK(run_gemm(ctx, ctx->plan_head, ha, R, PRO_GAIN, EPI_ARGMAX, FC_CLS_HEAD, claim_word(ctx, 0, GEMM_HEAD)));
     AcceptArgs ac; memset(&ac, 0, sizeof ac);
     ac.window = ctx->b.window; ac.amax = ctx->b.amax; ac.amax_clear = ctx->b.amax;
     ac.kv_len = ctx->b.kv_len; ac.n_gen = ctx->b.n_gen; ac.done = ctx->b.done;
@@ -698,7 +713,7 @@ extern "C" int fc_profile_step(fc_ctx *ctx, float *ms_by_class, int32_t *launche
 }
 
 // ------------------------------------------------------------------------------------ single operations
-static __device__ unsigned int g_op_err;
+static __device__ unsigned int g_op_err[2];   // error word, work-claim counter of fc_op_linear
 
 extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, int32_t N, int32_t K, int32_t dtype,
                             int32_t use_tensor_cores, void *cuda_stream) {
@@ -718,11 +733,11 @@ extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, 
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
       cudaGetSymbolAddress((void **)&err_word, g_op_err) != cudaSuccess) return FC_ERR_CUDA;
-  if (cudaMemsetAsync(err_word, 0, sizeof(unsigned int), st) != cudaSuccess) return FC_ERR_CUDA;
+  if (cudaMemsetAsync(err_word, 0, 2 * sizeof(unsigned int), st) != cudaSuccess) return FC_ERR_CUDA;
   char msg[200];
   UmmaPlan *pl = umma_plan_create(a, PRO_NONE, EPI_ATOMIC_ADD, sms, err_word, msg, sizeof msg);
   if (!pl) { fprintf(stderr, "fc_op_linear: %s\n", msg); return FC_ERR_CUDA; }
-  cudaError_t e = launch_gemm_umma(pl, a, 0, st);
+  cudaError_t e = launch_gemm_umma(pl, a, err_word + 1, 0, st);
   unsigned int herr = 0;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&herr, err_word, sizeof herr, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);

@@ -148,9 +148,10 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
                            char *err, int errlen);
 void umma_plan_destroy(UmmaPlan *p);
 // x/x2/y/ss pointers and R may differ per launch from those the plan was created with.
-cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, int pdl, cudaStream_t st);
+// claim: one zeroed word per projection of the launch (the work-claim counters).
+cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int *claim, int pdl, cudaStream_t st);
 // Up to four projections in one launch, each consuming the previous one's reduced output; bar: n-1 zeroed words.
-cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar, int pdl,
-                              cudaStream_t st);
+cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
+                              unsigned int *claim, int pdl, cudaStream_t st);
 
 }  // namespace fc

@@ -36,6 +36,7 @@ struct PhaseDesc {
   int n_tiles, nkb;               // 128-row tiles over all matrices; 64-wide k blocks
   int tiles_m[kMaxMats];
   int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
+  int chunk_kb, cpt, n_chunks;    // work is claimed in chunks of chunk_kb k-blocks of one tile; chunks per tile; total
 };
 
 struct MapPack { CUtensorMap m[kMaxPhases * kMaxMats]; };
@@ -44,10 +45,10 @@ struct UmmaParams {
   PhaseDesc ph[kMaxPhases];
   int n_phases;
   int stages;
-  int tile_mode;                  // 0: stream-K ranges, 1: whole tiles round-robin (argmax epilogue)
   int pdl;                        // launched as a programmatic dependent of the previous kernel
   unsigned int *err;              // device error word (0 = ok)
   unsigned int *bar;              // [n_phases - 1] grid-barrier counters, zero when the kernel starts
+  unsigned int *claim;            // [n_phases] work-claim counters, zero when the kernel starts
 };
 
 struct UmmaPlan {
@@ -195,34 +196,20 @@ __device__ __forceinline__ bool grid_bar_wait(const unsigned int *ctr, unsigned 
 
 struct Segment { int tile, kb0, kb1; };
 
-// Work of one CTA in one phase: stream-K mode deals contiguous (tile, k-block) ranges; tile mode deals
-// whole tiles round-robin.
-struct SegIter {
-  long long w, w1;
-  int tile, tile_step, n_tiles, nkb, mode;
-  __device__ SegIter(const PhaseDesc &d, int tile_mode) {
-    mode = tile_mode; nkb = d.nkb; n_tiles = d.n_tiles;
-    if (mode == 0) {
-      const long long W = (long long)d.n_tiles * d.nkb;
-      w = W * blockIdx.x / gridDim.x;
-      w1 = W * (blockIdx.x + 1) / gridDim.x;
-      tile = tile_step = 0;
-    } else { tile = blockIdx.x; tile_step = gridDim.x; w = w1 = 0; }
-  }
-  __device__ bool next(Segment &s) {
-    if (mode == 0) {
-      if (w >= w1) return false;
-      s.tile = (int)(w / nkb); s.kb0 = (int)(w % nkb);
-      long long rem = w1 - w;
-      s.kb1 = (int)((nkb - s.kb0 < rem) ? nkb : s.kb0 + rem);
-      w += s.kb1 - s.kb0;
-      return true;
-    }
-    if (tile >= n_tiles) return false;
-    s.tile = tile; s.kb0 = 0; s.kb1 = nkb; tile += tile_step;
-    return true;
-  }
-};
+// Work distribution.  SMs do not all see the same memory bandwidth, so equal static shares finish microseconds
+// apart and every grid barrier waits for the slowest.  Instead the producer warp of each CTA claims chunks
+// (chunk_kb consecutive k-blocks of one 128-row tile, for one block of rows) from a per-phase global counter
+// and publishes them to the other warps of its CTA through a small shared-memory queue; fast CTAs simply
+// claim more.  A queue entry with tile < 0 ends the phase.
+constexpr int kSegQ = 8;           // queue slots (power of two)
+__device__ __forceinline__ void chunk_decode(const PhaseDesc &d, unsigned int id, Segment &s, int &rb) {
+  const int per_rb = d.n_tiles * d.cpt;
+  rb = (int)(id / (unsigned)per_rb);
+  const int rem = (int)(id - (unsigned)rb * (unsigned)per_rb);
+  s.tile = rem / d.cpt;
+  s.kb0 = (rem - s.tile * d.cpt) * d.chunk_kb;
+  s.kb1 = min(d.nkb, s.kb0 + d.chunk_kb);
+}
 
 __device__ __forceinline__ void tile_info(const PhaseDesc &d, int tile, int &m, int &row0, int &rows_valid, int &ycol0) {
   m = 0;
@@ -251,7 +238,8 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   constexpr uint32_t kIdesc = make_idesc(BN);
 
   extern __shared__ unsigned char smem_dyn[];
-  __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar, go_bar[kMaxPhases];
+  __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar, go_bar[kMaxPhases], seg_full[kSegQ], seg_empty[kSegQ];
+  __shared__ int4 seg_q[kSegQ];          // (tile, kb0, kb1, row block)
   __shared__ unsigned int bar_cnt_s[kMaxPhases];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
@@ -260,8 +248,6 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = p.stages;
-  const int R = p.ph[0].g.R;                  // every phase of a chain works on the same rows
-  const int nrb = (R + BN - 1) / BN;
   volatile int *abort_flag = &abort_s;
 
   if (threadIdx.x == 0) {
@@ -270,6 +256,8 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
     mbar_init(smem_u32(&drain_bar), 1);
     for (int i = 0; i < kMaxPhases; ++i) { mbar_init(smem_u32(&go_bar[i]), 1); bar_cnt_s[i] = 0u; }
+    // a queue slot is read by the MMA thread, four staging warps and four epilogue warps
+    for (int i = 0; i < kSegQ; ++i) { mbar_init(smem_u32(&seg_full[i]), 1); mbar_init(smem_u32(&seg_empty[i]), 9); }
     fence_barrier_init();
   }
   if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), kCols);
@@ -283,46 +271,83 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
 
   int issued = 0;   // producer: k-block loads issued (for the drain on abort)
 
+  // Next queue entry for a whole warp (take_warp) or for a single thread (take_lane): 1 = a segment,
+  // 0 = end of the phase, -1 = a bounded wait gave up.
+  auto take_warp = [&](int &sq, Segment &s, int &rb) -> int {
+    const int slot = sq & (kSegQ - 1);
+    if (!mbar_wait_warp(smem_u32(&seg_full[slot]), (uint32_t)(sq / kSegQ) & 1u, abort_flag)) return -1;
+    const int4 d = seg_q[slot];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&seg_empty[slot]));
+    ++sq;
+    if (d.x < 0) return 0;
+    s.tile = d.x; s.kb0 = d.y; s.kb1 = d.z; rb = d.w;
+    return 1;
+  };
+  auto take_lane = [&](int &sq, Segment &s, int &rb) -> int {
+    const int slot = sq & (kSegQ - 1);
+    if (!mbar_wait(smem_u32(&seg_full[slot]), (uint32_t)(sq / kSegQ) & 1u, abort_flag)) return -1;
+    const int4 d = seg_q[slot];
+    mbar_arrive(smem_u32(&seg_empty[slot]));
+    ++sq;
+    if (d.x < 0) return 0;
+    s.tile = d.x; s.kb0 = d.y; s.kb1 = d.z; rb = d.w;
+    return 1;
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     // Weights depend on nothing that runs on the device, so the producer never waits for a grid barrier
     // or for the previous kernel: it streams phase after phase, limited only by free ring slots.
     if (lane == 0) {
-      int it = 0;
+      int it = 0, sq = 0;
       bool ok = true;
       for (int pi = 0; pi < p.n_phases && ok; ++pi) {
         const PhaseDesc &P = p.ph[pi];
-        for (int rb = 0; rb < nrb && ok; ++rb) {
-          SegIter si(P, p.tile_mode);
-          Segment s;
-          while (ok && si.next(s)) {
-            int m, row0, rows_valid, ycol0;
-            tile_info(P, s.tile, m, row0, rows_valid, ycol0);
-            const CUtensorMap *mp = &maps.m[pi * kMaxMats + m];
-            for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
-              const int stage = it % S;
-              const uint32_t ph = (uint32_t)(it / S) & 1u;
-              if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
-              const uint32_t bar = smem_u32(&full_w[stage]);
-              mbar_expect_tx(bar, (uint32_t)P.tx_bytes[m]);
-              tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
-              issued = it + 1;
-            }
+        for (;;) {
+          const int slot = sq & (kSegQ - 1);
+          if (!mbar_wait(smem_u32(&seg_empty[slot]), ((uint32_t)(sq / kSegQ) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+          const unsigned int id = atomicAdd(p.claim + pi, 1u);
+          if (id >= (unsigned int)P.n_chunks) {                 // nothing left in this phase
+            seg_q[slot] = make_int4(-1, 0, 0, 0);
+            mbar_arrive(smem_u32(&seg_full[slot]));
+            ++sq;
+            break;
           }
+          Segment s;
+          int rb;
+          chunk_decode(P, id, s, rb);
+          seg_q[slot] = make_int4(s.tile, s.kb0, s.kb1, rb);
+          mbar_arrive(smem_u32(&seg_full[slot]));
+          ++sq;
+          int m, row0, rows_valid, ycol0;
+          tile_info(P, s.tile, m, row0, rows_valid, ycol0);
+          const CUtensorMap *mp = &maps.m[pi * kMaxMats + m];
+          for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+            const int stage = it % S;
+            const uint32_t ph = (uint32_t)(it / S) & 1u;
+            if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t bar = smem_u32(&full_w[stage]);
+            mbar_expect_tx(bar, (uint32_t)P.tx_bytes[m]);
+            tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
+            issued = it + 1;
+          }
+          if (!ok) break;
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      int it = 0, seg = 0;
+      int it = 0, seg = 0, sq = 0;
       bool ok = true;
       for (int pi = 0; pi < p.n_phases && ok; ++pi) {
-        const PhaseDesc &P = p.ph[pi];
-        for (int rb = 0; rb < nrb && ok; ++rb) {
-          SegIter si(P, p.tile_mode);
+        {
           Segment s;
-          while (ok && si.next(s)) {
+          int rb = 0;
+          while (ok) {
+            const int got = take_lane(sq, s, rb);
+            if (got <= 0) { ok = got == 0; break; }
             const int acc = seg & 1;
             if (!mbar_wait(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -357,7 +382,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     const int sw = warp - 2;
     constexpr int kUW = BN / 4;
     const int chunk = lane & 7;
-    int it = 0, seg = 0;
+    int it = 0, seg = 0, sq = 0;
     bool ok = true;
     for (int pi = 0; pi < p.n_phases && ok; ++pi) {
       const PhaseDesc &P = p.ph[pi];
@@ -374,10 +399,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
         if (!ok) break;
       }
-      for (int rb = 0; rb < nrb && ok; ++rb) {
-        SegIter si(P, p.tile_mode);
+      {
         Segment s;
-        while (ok && si.next(s)) {
+        int rb = 0;
+        while (ok) {
+          const int got = take_warp(sq, s, rb);
+          if (got <= 0) { ok = got == 0; break; }
           const int acc = seg & 1;
           const bool need_ss = pro == PRO_GAIN && (EPI == EPI_ARGMAX || (g.ss_out != nullptr && s.tile == 0));
           float *my_ss = &ss_part[acc][sw][0];
@@ -483,15 +510,17 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs may still be read by the previous grid
     const int q = warp & 3;
     const int n_local = q * 32 + lane;
-    int seg = 0;
+    int seg = 0, sq = 0;
     bool ok = true;
     for (int pi = 0; pi < p.n_phases && ok; ++pi) {
       const PhaseDesc &P = p.ph[pi];
       const GemmArgs &g = P.g;
-      for (int rb = 0; rb < nrb && ok; ++rb) {
-        SegIter si(P, p.tile_mode);
+      {
         Segment s;
-        while (ok && si.next(s)) {
+        int rb = 0;
+        while (ok) {
+          const int got = take_warp(sq, s, rb);
+          if (got <= 0) { ok = got == 0; break; }
           int m, row0, rows_valid, ycol0;
           tile_info(P, s.tile, m, row0, rows_valid, ycol0);
           const int acc = seg & 1;
@@ -657,16 +686,19 @@ static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, i
 // One launch that runs plans[0..n-1] back to back on the same rows; plan i+1 consumes what plan i reduced
 // into its output, separated by a grid barrier on bar[i] (zero at launch).  args[i] carries the per-launch
 // buffers and the row count; weights, K and the matrix split stay as planned.
-cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar, int pdl,
-                              cudaStream_t st) {
-  if (n < 1 || n > kMaxPhases) return cudaErrorInvalidValue;
+cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
+                              unsigned int *claim, int pdl, cudaStream_t st) {
+  if (n < 1 || n > kMaxPhases || !claim) return cudaErrorInvalidValue;
   if (n > 1 && !bar) return cudaErrorInvalidValue;
   MapPack maps;
   UmmaParams p;
   memset(&p, 0, sizeof p);
   const int epi = plans[0]->epi;
-  long long max_items = 1;
-  int max_tiles = 1;
+  int bn, cps;
+  bn_config(args[0].R, bn, p.stages, cps);
+  const int nrb = (args[0].R + bn - 1) / bn;
+  const int tile_mode = (epi == EPI_ARGMAX) ? 1 : 0;
+  long long max_chunks = 1;
   for (int i = 0; i < n; ++i) {
     const UmmaPlan *pl = plans[i];
     const GemmArgs &a = args[i];
@@ -676,29 +708,29 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.g.x = a.x; d.g.x2 = a.x2; d.g.ldx = a.ldx; d.g.ss_in = a.ss_in; d.g.ss_out = a.ss_out;
     d.g.y = a.y; d.g.ldy = a.ldy; d.g.R = a.R; d.g.tokens = a.tokens; d.g.amax = a.amax; d.g.logits = a.logits;
     for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = pl->maps[m];
-    const long long W = (long long)d.n_tiles * d.nkb;
-    if (W > max_items) max_items = W;
-    if (d.n_tiles > max_tiles) max_tiles = d.n_tiles;
+    // the argmax epilogue needs whole tiles; partial sums may be split along k into chunks of four k-blocks
+    // (one k-block per staging warp)
+    d.chunk_kb = tile_mode ? d.nkb : 4;
+    d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
+    const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
+    if (chunks > 0x7fffffffLL) return cudaErrorInvalidValue;
+    d.n_chunks = (int)chunks;
+    if (chunks > max_chunks) max_chunks = chunks;
   }
   for (int i = n; i < kMaxPhases; ++i)
     for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = plans[0]->maps[0];
-  p.n_phases = n; p.pdl = pdl; p.err = plans[0]->err; p.bar = bar;
-  p.tile_mode = (epi == EPI_ARGMAX) ? 1 : 0;
-  int bn, cps;
-  bn_config(args[0].R, bn, p.stages, cps);
+  p.n_phases = n; p.pdl = pdl; p.err = plans[0]->err; p.bar = bar; p.claim = claim;
   // Staging warps own every fourth k-block and run ahead of each other; the parity waits on the ring
   // are only unambiguous while the ring is at least as deep as the number of staging warps.
   if (p.stages < 4 || p.stages > 8) return cudaErrorInvalidValue;
   const long long resident = (long long)plans[0]->n_sms * cps;     // the grid barrier needs every CTA resident
-  int grid;
-  if (p.tile_mode == 0) grid = (int)(resident < max_items ? resident : max_items);
-  else grid = (int)(resident < max_tiles ? resident : max_tiles);
+  const int grid = (int)(resident < max_chunks ? resident : max_chunks);
   if (epi == EPI_ARGMAX) return launch_bn<EPI_ARGMAX>(maps, p, bn, grid, st);
   return launch_bn<EPI_ATOMIC_ADD>(maps, p, bn, grid, st);
 }
 
-cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, int pdl, cudaStream_t st) {
-  return launch_gemm_chain(&pl, &a, 1, nullptr, pdl, st);
+cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, int pdl, cudaStream_t st) {
+  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, pdl, st);
 }
 
 }  // namespace fc
