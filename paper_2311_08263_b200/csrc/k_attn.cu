@@ -99,23 +99,47 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   }
 
   if (nk > 0) {
-    // ---- window keys owned by this chunk: from the accumulators, rotated, stored to smem and to the cache
-    for (int e = tid; e < (nk - n_cached) * HALF; e += kAttnThreads) {
-      const int t = n_cached + e / HALF, i = e % HALF;
-      const int pos = k0 + t, j = pos - L;
-      const int r = bl * a.c + j;
-      const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
-      const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
-      const float *vacc = kacc + kvd;
-      const float2 rot = __ldg(a.rope + (long long)pos * HALF + i);
-      const float cs = rot.x, sn = rot.y;
-      const float x0 = kacc[i] * s, x1 = kacc[i + HALF] * s;
-      const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * cs - x1 * sn), o1 = __float2bfloat16_rn(x0 * sn + x1 * cs);
-      const __nv_bfloat16 v0 = __float2bfloat16_rn(vacc[i] * s), v1 = __float2bfloat16_rn(vacc[i + HALF] * s);
-      Ks[t * LD + i] = o0; Ks[t * LD + i + HALF] = o1;
-      Vs[t * LD + i] = v0; Vs[t * LD + i + HALF] = v1;
-      kbase[(long long)pos * HD + i] = o0; kbase[(long long)pos * HD + i + HALF] = o1;
-      vbase[(long long)pos * HD + i] = v0; vbase[(long long)pos * HD + i + HALF] = v1;
+    // ---- window keys owned by this chunk: from the accumulators, rotated, stored to smem and to the cache.
+    // A thread keeps one pair index i and walks the window rows in passes; the loads of a pass are all issued
+    // before the first use so that they share one trip to L2.
+    {
+      constexpr int RPI = kAttnThreads / HALF;               // rows covered per pass
+      constexpr int NB = 4;                                  // passes batched together
+      const int i = tid % HALF, rsub = tid / HALF;
+      const int n_win = nk - n_cached;
+      for (int t0 = 0; t0 < n_win; t0 += RPI * NB) {
+        float k0v[NB], k1v[NB], v0v[NB], v1v[NB], ssv[NB];
+        float2 rot[NB];
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+          const int tw = t0 + u * RPI + rsub;
+          k0v[u] = k1v[u] = v0v[u] = v1v[u] = ssv[u] = 0.f; rot[u] = make_float2(1.f, 0.f);
+          if (tw < n_win) {
+            const int pos = k0 + n_cached + tw, j = pos - L;
+            const int r = bl * a.c + j;
+            const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
+            ssv[u] = __ldcg(a.ss + r);
+            k0v[u] = __ldcg(kacc + i); k1v[u] = __ldcg(kacc + i + HALF);
+            v0v[u] = __ldcg(kacc + kvd + i); v1v[u] = __ldcg(kacc + kvd + i + HALF);
+            rot[u] = __ldg(a.rope + (long long)pos * HALF + i);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < NB; ++u) {
+          const int tw = t0 + u * RPI + rsub;
+          if (tw >= n_win) continue;
+          const int t = n_cached + tw, pos = k0 + t;
+          const float sc = rsqrtf(ssv[u] / (float)a.dn + a.eps);
+          const float x0 = k0v[u] * sc, x1 = k1v[u] * sc;
+          const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * rot[u].x - x1 * rot[u].y);
+          const __nv_bfloat16 o1 = __float2bfloat16_rn(x0 * rot[u].y + x1 * rot[u].x);
+          const __nv_bfloat16 w0 = __float2bfloat16_rn(v0v[u] * sc), w1 = __float2bfloat16_rn(v1v[u] * sc);
+          Ks[t * LD + i] = o0; Ks[t * LD + i + HALF] = o1;
+          Vs[t * LD + i] = w0; Vs[t * LD + i + HALF] = w1;
+          kbase[(long long)pos * HD + i] = o0; kbase[(long long)pos * HD + i + HALF] = o1;
+          vbase[(long long)pos * HD + i] = w0; vbase[(long long)pos * HD + i + HALF] = w1;
+        }
+      }
     }
     // rows beyond nk: zero so that stale shared memory (possibly NaN patterns) never meets a zero weight
     for (int e = tid; e < (kChunk - nk) * CPR; e += kAttnThreads) {
