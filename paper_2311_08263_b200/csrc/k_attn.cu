@@ -88,6 +88,30 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  // Q tile registers: a thread keeps one pair index and walks the 16 rows of a tile; all loads of a tile are
+  // issued together.  The first tile's loads are issued here so that their latency overlaps the prologue.
+  constexpr int QRPI = kAttnThreads / HALF;                  // rows covered per pass
+  constexpr int QNIT = 16 / QRPI;
+  const int qi_pair = tid % HALF, q_rsub = tid / HALF;
+  float qx0[QNIT], qx1[QNIT], qss[QNIT];
+  float2 qrot[QNIT];
+  auto q_load = [&](int qt) {
+#pragma unroll
+    for (int it = 0; it < QNIT; ++it) {
+      const int qrow = qt * 16 + q_rsub + it * QRPI;
+      qx0[it] = qx1[it] = 0.f; qss[it] = 0.f; qrot[it] = make_float2(1.f, 0.f);
+      if (qrow < nq) {
+        const int g = div_c(qrow), j = qrow - g * a.c;
+        const int r = bl * a.c + j, h = kvh * group + g;
+        const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
+        qss[it] = __ldcg(a.ss + r);
+        qx0[it] = __ldcg(qacc + qi_pair); qx1[it] = __ldcg(qacc + qi_pair + HALF);
+        qrot[it] = __ldg(a.rope + (long long)(L + j) * HALF + qi_pair);
+      }
+    }
+  };
+  q_load(0);
+
   // side clearing of buffers nobody reads during this kernel
   {
     const unsigned long long gtid =
@@ -155,35 +179,15 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   const int g4 = lane >> 2, t4 = lane & 3;
   for (int qt = 0; qt < nqt; ++qt) {
     __syncthreads();                                          // K/V staged; previous tile's Qs/Om/mls free
-    // ---- Q tile: 1/rms, rotation, bf16.  A thread keeps one pair index i and walks the rows; all of its
-    // loads are issued before the first use so that they share one trip to L2.
-    {
-      constexpr int RPI = kAttnThreads / HALF;               // rows covered per pass
-      constexpr int NIT = 16 / RPI;
-      const int i = tid % HALF, rsub = tid / HALF;
-      float x0[NIT], x1[NIT], ssv[NIT];
-      float2 rot[NIT];
+    // ---- Q tile: 1/rms, rotation, bf16 (loads were issued earlier for the first tile)
+    if (qt > 0) q_load(qt);
 #pragma unroll
-      for (int it = 0; it < NIT; ++it) {
-        const int qrow = qt * 16 + rsub + it * RPI;
-        x0[it] = x1[it] = 0.f; ssv[it] = 0.f; rot[it] = make_float2(1.f, 0.f);
-        if (qrow < nq) {
-          const int g = div_c(qrow), j = qrow - g * a.c;
-          const int r = bl * a.c + j, h = kvh * group + g;
-          const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
-          ssv[it] = __ldcg(a.ss + r);
-          x0[it] = __ldcg(qacc + i); x1[it] = __ldcg(qacc + i + HALF);
-          rot[it] = __ldg(a.rope + (long long)(L + j) * HALF + i);
-        }
-      }
-#pragma unroll
-      for (int it = 0; it < NIT; ++it) {
-        const int row = rsub + it * RPI;
-        const float sc = rsqrtf(ssv[it] / (float)a.dn + a.eps);
-        const float a0 = x0[it] * sc, a1 = x1[it] * sc;
-        Qs[row * LD + i] = __float2bfloat16_rn(a0 * rot[it].x - a1 * rot[it].y);
-        Qs[row * LD + i + HALF] = __float2bfloat16_rn(a0 * rot[it].y + a1 * rot[it].x);
-      }
+    for (int it = 0; it < QNIT; ++it) {
+      const int row = q_rsub + it * QRPI;
+      const float sc = rsqrtf(qss[it] / (float)a.dn + a.eps);
+      const float a0 = qx0[it] * sc, a1 = qx1[it] * sc;
+      Qs[row * LD + qi_pair] = __float2bfloat16_rn(a0 * qrot[it].x - a1 * qrot[it].y);
+      Qs[row * LD + qi_pair + HALF] = __float2bfloat16_rn(a0 * qrot[it].y + a1 * qrot[it].x);
     }
     __syncthreads();
 
