@@ -118,8 +118,14 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
         ((unsigned long long)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * blockDim.x + tid;
     const unsigned long long nth = (unsigned long long)gridDim.x * gridDim.y * gridDim.z * blockDim.x;
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-      if (a.z.p[i]) for (unsigned long long e = gtid; e < a.z.n[i]; e += nth) a.z.p[i][e] = 0.f;
+    for (int i = 0; i < 4; ++i) {
+      if (!a.z.p[i]) continue;
+      // 16-byte stores over the aligned bulk, scalar stores for the tail (buffers are 256-byte aligned)
+      const unsigned long long n4 = a.z.n[i] >> 2;
+      float4 *p4 = reinterpret_cast<float4 *>(a.z.p[i]);
+      for (unsigned long long e = gtid; e < n4; e += nth) p4[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (unsigned long long e = (n4 << 2) + gtid; e < a.z.n[i]; e += nth) a.z.p[i][e] = 0.f;
+    }
   }
 
   if (nk > 0) {
@@ -128,7 +134,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
     // before the first use so that they share one trip to L2.
     {
       constexpr int RPI = kAttnThreads / HALF;               // rows covered per pass
-      constexpr int NB = 4;                                  // passes batched together
+      constexpr int NB = 16 / RPI;                           // passes batched together: 16 window rows per trip
       const int i = tid % HALF, rsub = tid / HALF;
       const int n_win = nk - n_cached;
       for (int t0 = 0; t0 < n_win; t0 += RPI * NB) {
