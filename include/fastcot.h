@@ -130,10 +130,11 @@ int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen);
  * untouched, so every step runs at the same K/V length (latency sweeps). */
 int fc_bench_steps(fc_ctx *ctx, int32_t n_steps, int32_t commit, float *ms_total, int64_t *tokens_out);
 
-/* One non-committing step with CUDA events around every launch.  ms_by_class / launches_by_class
+/* One non-committing step with CUDA events around every launch (launches are therefore fully serialised:
+ * no programmatic overlap between neighbours).  ms_by_class / launches_by_class
  * (host, FC_N_CLASSES entries each) receive device time and launch count per kernel class. */
 enum { FC_CLS_EMBED = 0, FC_CLS_QKV, FC_CLS_ROPE, FC_CLS_ATTN, FC_CLS_OPROJ, FC_CLS_GATEUP, FC_CLS_DOWN,
-       FC_CLS_HEAD, FC_CLS_ACCEPT, FC_N_CLASSES };
+       FC_CLS_HEAD, FC_CLS_ACCEPT, FC_CLS_CHAIN /* O + gate/up + down + next QKV in one launch */, FC_N_CLASSES };
 int fc_profile_step(fc_ctx *ctx, float *ms_by_class, int32_t *launches_by_class);
 
 /* Number of kernels the most recent step / prefill / bench call launched. */

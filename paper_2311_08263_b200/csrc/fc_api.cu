@@ -351,7 +351,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   const int nsplit = (max_len_host + rows + d.tk - 1) / d.tk;
   const long long stride_h = (long long)s.max_seq * s.head_dim;
   const long long stride_b = (long long)s.n_kv_heads * stride_h;
-  const bool chained = ctx->chain && !ctx->prof;
+  const bool chained = ctx->chain;
   for (int l = 0; l < s.n_layers; ++l) {
     if (!chained || l == 0)
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV, claim_word(ctx, l, GEMM_QKV)));
@@ -398,9 +398,10 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       if (l + 1 < s.n_layers) { plans[3] = ctx->plan_qkv[l + 1]; ga[3] = args_qkv(ctx, l + 1); n = 4; }
       for (int i = 0; i < n; ++i) ga[i].R = R;
       ++ctx->launches;
+      ProfScope ps(ctx, FC_CLS_CHAIN);
       // barriers at words 0..2 of the layer's group, claim counters at 4..7 (O, gate/up, down, next QKV)
       FC_CK(launch_gemm_chain(plans, ga, n, ctx->b.chain_bar + (size_t)l * 8, ctx->b.chain_bar + (size_t)l * 8 + 4,
-                              ctx->pdl, ctx->st));
+                              ctx->pdl && !ctx->prof, ctx->st));
     } else {
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O)));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));

@@ -16,7 +16,7 @@ FC_REFILL_PROMPT_CYCLE, FC_REFILL_PAD = 0, 1
 FC_FLAG_SIMT_GEMM, FC_FLAG_NO_GRAPH, FC_FLAG_NO_PDL, FC_FLAG_NO_CHAIN = 1, 2, 4, 8
 FC_OK = 0
 FC_NOALLOC_SCRATCH_BYTES = 8 << 20
-FC_CLASSES = ["embed", "qkv", "rope", "attn", "oproj", "gateup", "down", "head", "accept"]
+FC_CLASSES = ["embed", "qkv", "rope", "attn", "oproj", "gateup", "down", "head", "accept", "chain"]
 FC_ERR_ARG, FC_ERR_SHAPE, FC_ERR_CAPACITY, FC_ERR_TOKEN_RANGE = -1, -2, -3, -4
 FC_ERR_STATE, FC_ERR_BAD_WINDOW, FC_ERR_DEVICE_TIMEOUT, FC_ERR_CUDA = -5, -6, -7, -8
 
