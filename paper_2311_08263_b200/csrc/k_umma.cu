@@ -28,6 +28,11 @@ constexpr int kWBytes = kTileM * kTileK * 2;
 constexpr int kThreads = 320;
 constexpr unsigned long long kSpinBudget = 400000000ull;    // clock64 ticks (~0.2 s)
 
+// Activations are staged as a bf16 pair hi + lo (lo = bf16(x - hi)) while the accumulator is narrow: two MMAs per
+// k-step against the same weight tile, which removes the bf16 rounding of the activations (the tensor pipe is
+// almost idle on this memory-bound kernel).  Wide accumulators (more than 64 rows) stage plain bf16.
+__host__ __device__ constexpr int x_parts(int bn) { return bn <= 64 ? 2 : 1; }
+
 constexpr int kMaxPhases = 4;      // projections chained in one launch (O -> gate/up -> down -> next QKV)
 
 struct PhaseDesc {
@@ -229,11 +234,13 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
   return v;
 }
 
-// Widths up to 64 rows run two CTAs per SM (the grid barrier needs the whole grid resident).
+// Widths up to 32 rows run two CTAs per SM (the grid barrier needs the whole grid resident).
 template <int EPI, int BN>
-__global__ void __launch_bounds__(kThreads, (BN <= 64 ? 2 : 1))
+__global__ void __launch_bounds__(kThreads, (BN <= 32 ? 2 : 1))
 gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ UmmaParams p) {
-  constexpr int kStageBytes = kWBytes + BN * 128;
+  constexpr int kXParts = x_parts(BN);
+  constexpr int kXBytes = BN * 128;                 // one staged activation tile (bf16, 64 k)
+  constexpr int kStageBytes = kWBytes + kXParts * kXBytes;
   constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
   constexpr uint32_t kIdesc = make_idesc(BN);
 
@@ -361,9 +368,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
               const uint32_t a_base = smem_base + stage * kStageBytes;
               const uint32_t b_base = a_base + kWBytes;
 #pragma unroll
-              for (int kk = 0; kk < kTileK / 16; ++kk)
-                umma_bf16(d_tmem, smem_desc_sw128(a_base + kk * 32), smem_desc_sw128(b_base + kk * 32), kIdesc,
-                          (kb > s.kb0 || kk > 0) ? 1u : 0u);
+              for (int kk = 0; kk < kTileK / 16; ++kk) {
+#pragma unroll
+                for (int part = 0; part < kXParts; ++part)
+                  umma_bf16(d_tmem, smem_desc_sw128(a_base + kk * 32), smem_desc_sw128(b_base + part * kXBytes + kk * 32),
+                            kIdesc, (kb > s.kb0 || kk > 0 || part > 0) ? 1u : 0u);
+              }
               umma_commit(smem_u32(&empty_b[stage]));
             }
             if (ok) umma_commit(smem_u32(&accum_full[acc]));
@@ -475,12 +485,22 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
                   sq += __shfl_xor_sync(0xffffffffu, sq, 4);
                   if (chunk == 0) my_ss[row] += sq;
                 }
+                const int soff = (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4);
                 uint4 pk;
                 __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
                 __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
                 pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
                 pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
-                *reinterpret_cast<uint4 *>(xs + (row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4)) = pk;
+                *reinterpret_cast<uint4 *>(xs + soff) = pk;
+                if (kXParts == 2) {      // low part: what the first rounding lost
+                  const float2 h0 = __bfloat1622float2(b0), h1 = __bfloat1622float2(b1);
+                  const float2 h2 = __bfloat1622float2(b2), h3 = __bfloat1622float2(b3);
+                  __nv_bfloat162 l0 = __floats2bfloat162_rn(v[0] - h0.x, v[1] - h0.y), l1 = __floats2bfloat162_rn(v[2] - h1.x, v[3] - h1.y);
+                  __nv_bfloat162 l2 = __floats2bfloat162_rn(v[4] - h2.x, v[5] - h2.y), l3 = __floats2bfloat162_rn(v[6] - h3.x, v[7] - h3.y);
+                  pk.x = *reinterpret_cast<uint32_t *>(&l0); pk.y = *reinterpret_cast<uint32_t *>(&l1);
+                  pk.z = *reinterpret_cast<uint32_t *>(&l2); pk.w = *reinterpret_cast<uint32_t *>(&l3);
+                  *reinterpret_cast<uint4 *>(xs + kXBytes + soff) = pk;
+                }
               }
             }
             fence_proxy_async();
@@ -611,9 +631,9 @@ static EncodeTiledFn get_encode_fn() {
 
 // accumulator width, ring depth and resident CTAs per SM for a row count
 static void bn_config(int R, int &bn, int &stages, int &ctas_per_sm) {
-  if (R <= 16) { bn = 16; stages = 6; ctas_per_sm = 2; }
-  else if (R <= 32) { bn = 32; stages = 5; ctas_per_sm = 2; }
-  else if (R <= 64) { bn = 64; stages = 4; ctas_per_sm = 2; }
+  if (R <= 16) { bn = 16; stages = 5; ctas_per_sm = 2; }          // 5 x (16 + 2 x 2) KB
+  else if (R <= 32) { bn = 32; stages = 4; ctas_per_sm = 2; }     // 4 x (16 + 2 x 4) KB
+  else if (R <= 64) { bn = 64; stages = 6; ctas_per_sm = 1; }     // 6 x (16 + 2 x 8) KB
   else if (R <= 128) { bn = 128; stages = 6; ctas_per_sm = 1; }
   else { bn = 256; stages = 4; ctas_per_sm = 1; }
 }
@@ -655,7 +675,7 @@ void umma_plan_destroy(UmmaPlan *p) { delete p; }
 
 template <int EPI, int BN>
 static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid, cudaStream_t st) {
-  const size_t smem = (size_t)p.stages * (kWBytes + BN * 128) + 1024;
+  const size_t smem = (size_t)p.stages * (kWBytes + x_parts(BN) * BN * 128) + 1024;
   static size_t attr_smem = 0;
   if (smem > attr_smem) {
     cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
