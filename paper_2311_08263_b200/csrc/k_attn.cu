@@ -54,8 +54,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __nv_bfloat16 *Ks = reinterpret_cast<__nv_bfloat16 *>(smem_raw);       // [kChunk][LD]
   __nv_bfloat16 *Vs = Ks + kChunk * LD;                                  // [kChunk][LD]
-  __nv_bfloat16 *Qs = Vs + kChunk * LD;                                  // [16][LD]
-  float *Om = reinterpret_cast<float *>(Qs + 16 * LD);                   // [4][16][HD]
+  __nv_bfloat16 *Qs = Vs + kChunk * LD;                                  // [16][LD]  high part of q
+  __nv_bfloat16 *Ql = Qs + 16 * LD;                                      // [16][LD]  low part: q - bf16(q)
+  float *Om = reinterpret_cast<float *>(Ql + 16 * LD);                   // [4][16][HD]
   float *mls = Om + 4 * 16 * HD;                                         // [4][16][2]
   __shared__ unsigned int s_last, s_last_grid;
 
@@ -192,8 +193,13 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       const int row = q_rsub + it * QRPI;
       const float sc = rsqrtf(qss[it] / (float)a.dn + a.eps);
       const float a0 = qx0[it] * sc, a1 = qx1[it] * sc;
-      Qs[row * LD + qi_pair] = __float2bfloat16_rn(a0 * qrot[it].x - a1 * qrot[it].y);
-      Qs[row * LD + qi_pair + HALF] = __float2bfloat16_rn(a0 * qrot[it].y + a1 * qrot[it].x);
+      // q and the probabilities go through the tensor cores as a bf16 pair hi + lo, so that only the cached
+      // K and V (stored in the model dtype) carry bf16 rounding
+      const float r0 = a0 * qrot[it].x - a1 * qrot[it].y, r1 = a0 * qrot[it].y + a1 * qrot[it].x;
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(r0), h1 = __float2bfloat16_rn(r1);
+      Qs[row * LD + qi_pair] = h0; Qs[row * LD + qi_pair + HALF] = h1;
+      Ql[row * LD + qi_pair] = __float2bfloat16_rn(r0 - __bfloat162float(h0));
+      Ql[row * LD + qi_pair + HALF] = __float2bfloat16_rn(r1 - __bfloat162float(h1));
     }
     __syncthreads();
 
@@ -206,8 +212,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
     if (nk > 0) {
 #pragma unroll
       for (int ks = 0; ks < HD / 16; ++ks) {
-        uint32_t af[4];
+        uint32_t af[4], al[4];
         ldsm_x4(smem_addr(Qs + (lane & 15) * LD + ks * 16 + (lane >> 4) * 8), af[0], af[1], af[2], af[3]);
+        ldsm_x4(smem_addr(Ql + (lane & 15) * LD + ks * 16 + (lane >> 4) * 8), al[0], al[1], al[2], al[3]);
 #pragma unroll
         for (int nb = 0; nb < 4; nb += 2) {
           // two key blocks (8 keys each) x one 16-wide k step
@@ -216,6 +223,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
           ldsm_x4(smem_addr(Ks + key * LD + ks * 16 + ((lane >> 3) & 1) * 8), b0, b1, b2, b3);
           mma_bf16(sacc[nb], af, b0, b1);
           mma_bf16(sacc[nb + 1], af, b2, b3);
+          mma_bf16(sacc[nb], al, b0, b1);
+          mma_bf16(sacc[nb + 1], al, b2, b3);
         }
       }
     }
@@ -244,7 +253,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       mrow[hh] = fmaxf(mrow[hh], __shfl_xor_sync(0xffffffffu, mrow[hh], 1));
       mrow[hh] = fmaxf(mrow[hh], __shfl_xor_sync(0xffffffffu, mrow[hh], 2));
     }
-    uint32_t pf[2][4];                                        // P as A fragments: two 16-key steps
+    uint32_t pf[2][4], pl[2][4];                              // P (high and low parts) as A fragments: two 16-key steps
 #pragma unroll
     for (int nb = 0; nb < 4; ++nb) {
       float p[4];
@@ -256,6 +265,11 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
       }
       pf[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
       pf[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+      float pr[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pr[i] = p[i] - __bfloat162float(__float2bfloat16_rn(p[i]));
+      pl[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16(pr[0], pr[1]);
+      pl[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(pr[2], pr[3]);
     }
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
@@ -278,6 +292,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
           ldsm_x4_t(smem_addr(Vs + key * LD + d * 8 + (lane >> 4) * 8), b0, b1, b2, b3);
           mma_bf16(oacc[d], pf[kt], b0, b1);
           mma_bf16(oacc[d + 1], pf[kt], b2, b3);
+          mma_bf16(oacc[d], pl[kt], b0, b1);
+          mma_bf16(oacc[d + 1], pl[kt], b2, b3);
         }
       }
     }
@@ -417,7 +433,7 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
 template <int HD>
 static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
   constexpr int LD = HD + 8;
-  const size_t smem = sizeof(__nv_bfloat16) * (size_t)(2 * kChunk * LD + 16 * LD) +
+  const size_t smem = sizeof(__nv_bfloat16) * (size_t)(2 * kChunk * LD + 2 * 16 * LD) +
                       sizeof(float) * (size_t)(4 * 16 * HD + 4 * 16 * 2);
   static bool attr_done = false;
   if (!attr_done) {
