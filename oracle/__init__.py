@@ -29,7 +29,7 @@ class _Shape(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "n_kv_heads", "head_dim",
                                          "d_ffn", "vocab", "wdtype")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("bias_beta", C.c_float),
-                ("max_seq", C.c_int32)]
+                ("max_seq", C.c_int32), ("kv_bf16", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -59,6 +59,8 @@ def _load():
         lib.orc_generate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.orc_ar_generate.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                         C.c_void_p, C.c_void_p]
+        lib.orc_round_bf16.restype = C.c_float
+        lib.orc_round_bf16.argtypes = [C.c_float]
         lib.orc_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int,
                                    C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.orc_linear_add.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p]
@@ -76,6 +78,10 @@ def _host(t: torch.Tensor) -> torch.Tensor:
 
 def _i32(a) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def round_bf16(x: float) -> float:
+    return float(_load().orc_round_bf16(C.c_float(x)))
 
 
 def accept(window, argmax, n_gen: int, prompt, refill: int = 0, pad_id: int = 0):
@@ -103,10 +109,12 @@ class Oracle:
     """One sequence's decoder + Jacobi state on the CPU.
 
     `weights` is the dict produced by the workload generator (torch tensors, fp32 or bf16);
-    bf16 tensors are handed to C as raw bit patterns and up-converted exactly there.
+    bf16 tensors are handed to C as raw bit patterns and up-converted exactly there.  For a bf16 model
+    the K and V rows are rounded to bf16 where they are stored (kv_bf16, default = the weights' dtype):
+    the cache holds the model dtype; the arithmetic stays fp32.
     """
 
-    def __init__(self, cfg, weights: Dict[str, object], max_seq: int):
+    def __init__(self, cfg, weights: Dict[str, object], max_seq: int, kv_bf16: Optional[bool] = None):
         lib = _load()
         self.cfg, self.max_seq = cfg, max_seq
         self._keep: List[object] = []
@@ -124,7 +132,8 @@ class Oracle:
             return C.cast(arr, _PP)
 
         self._shape = _Shape(cfg.n_layers, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim,
-                             cfg.d_ffn, cfg.vocab, wd, cfg.rms_eps, cfg.rope_theta, cfg.bias_beta, max_seq)
+                             cfg.d_ffn, cfg.vocab, wd, cfg.rms_eps, cfg.rope_theta, cfg.bias_beta, max_seq,
+                             int((wd == 1) if kv_bf16 is None else kv_bf16))
         perm = weights.get("bias_perm")
         perm_ptr = None
         if perm is not None:

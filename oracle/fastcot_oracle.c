@@ -8,7 +8,8 @@
  * What it computes
  *   - decoder forward: a Llama-style causal decoder (RMSNorm, rotary embedding with
  *     half-split pairing, grouped-query attention, SwiGLU FFN, untied LM head), the model
- *     family the paper evaluates (Section 5.1).  fp32 arithmetic throughout.
+ *     family the paper evaluates (Section 5.1).  fp32 arithmetic throughout.  For a bf16 model the K and V
+ *     rows are rounded to bfloat16 where they are stored (the model's K/V tensors have the model dtype).
  *   - greedy autoregressive decoding: Eq. 1.
  *   - one Jacobi-window iteration: exact token + approximate tokens in one causal forward
  *     (Eq. 2-4), verification of the previous guesses one by one (Eq. 5), and the buffer /
@@ -39,6 +40,8 @@ typedef struct {
   int32_t wdtype;            /* 0: weights are float32; 1: weights are bfloat16 bit patterns */
   float rms_eps, rope_theta, bias_beta;
   int32_t max_seq;           /* capacity of the K/V cache in tokens (committed + window) */
+  int32_t kv_bf16;           /* 1: K and V are rounded to bfloat16 where they are stored (a bf16 model's K/V
+                              * tensors are bf16); all arithmetic stays fp32.  0: K/V kept in fp32 */
 } orc_shape;
 
 typedef struct {             /* host pointers, row-major [out_features, in_features] */
@@ -66,6 +69,14 @@ typedef struct orc {
 /* ------------------------------------------------------------------ element access */
 static inline float bf16_to_f32(uint16_t b) {
   uint32_t u = ((uint32_t)b) << 16; float f; memcpy(&f, &u, 4); return f;
+}
+/* round to nearest even onto the bfloat16 grid (NaN stays NaN) */
+float orc_round_bf16(float f) {
+  uint32_t u; memcpy(&u, &f, 4);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return f;
+  u += 0x7fffu + ((u >> 16) & 1u);
+  u &= 0xffff0000u;
+  memcpy(&f, &u, 4); return f;
 }
 static inline float wload(const void *p, int wdtype, size_t i) {
   return wdtype ? bf16_to_f32(((const uint16_t *)p)[i]) : ((const float *)p)[i];
@@ -165,6 +176,11 @@ int orc_forward(orc *o, const int32_t *tokens, int n, float *logits_out, int32_t
       int pos = L + r;
       for (int hh = 0; hh < hq; ++hh) rope(q + (size_t)r * qd + hh * hd, hd, pos, s->rope_theta);
       for (int hh = 0; hh < hkv; ++hh) rope(kk + (size_t)r * kvd + hh * hd, hd, pos, s->rope_theta);
+      if (s->kv_bf16)
+        for (int i = 0; i < kvd; ++i) {
+          kk[(size_t)r * kvd + i] = orc_round_bf16(kk[(size_t)r * kvd + i]);
+          vv[(size_t)r * kvd + i] = orc_round_bf16(vv[(size_t)r * kvd + i]);
+        }
       memcpy(kc + (size_t)pos * kvd, kk + (size_t)r * kvd, sizeof(float) * kvd);
       memcpy(vc + (size_t)pos * kvd, vv + (size_t)r * kvd, sizeof(float) * kvd);
     }
