@@ -28,10 +28,10 @@ constexpr int kWBytes = kTileM * kTileK * 2;
 constexpr int kThreads = 320;
 constexpr unsigned long long kSpinBudget = 400000000ull;    // clock64 ticks (~0.2 s)
 
-// Activations are staged as a bf16 pair hi + lo (lo = bf16(x - hi)) while the accumulator is narrow: two MMAs per
-// k-step against the same weight tile, which removes the bf16 rounding of the activations (the tensor pipe is
-// almost idle on this memory-bound kernel).  Wide accumulators (more than 64 rows) stage plain bf16.
-__host__ __device__ constexpr int x_parts(int bn) { return bn <= 64 ? 2 : 1; }
+// Activations are staged as a bf16 pair hi + lo (lo = bf16(x - hi)): two MMAs per k-step against the same weight
+// tile, which removes the bf16 rounding of the activations.  Up to 128 rows the kernel stays memory-bound with the
+// doubled MMA work; more rows run as blocks of 128 on the same weight chunk, back to back.
+__host__ __device__ constexpr int x_parts(int bn) { return 2; }
 
 constexpr int kMaxPhases = 4;      // projections chained in one launch (O -> gate/up -> down -> next QKV)
 
@@ -41,7 +41,8 @@ struct PhaseDesc {
   int n_tiles, nkb;               // 128-row tiles over all matrices; 64-wide k blocks
   int tiles_m[kMaxMats];
   int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
-  int chunk_kb, cpt, n_chunks;    // work is claimed in chunks of chunk_kb k-blocks of one tile; chunks per tile; total
+  int chunk_kb, cpt, nrb, n_chunks;   // work is claimed in chunks of chunk_kb k-blocks of one tile for one block of rows:
+                                      // chunks per tile, row blocks, total
 };
 
 struct MapPack { CUtensorMap m[kMaxPhases * kMaxMats]; };
@@ -208,11 +209,14 @@ struct Segment { int tile, kb0, kb1; };
 // claim more.  A queue entry with tile < 0 ends the phase.
 constexpr int kSegQ = 8;           // queue slots (power of two)
 __device__ __forceinline__ void chunk_decode(const PhaseDesc &d, unsigned int id, Segment &s, int &rb) {
-  const int per_rb = d.n_tiles * d.cpt;
-  rb = (int)(id / (unsigned)per_rb);
-  const int rem = (int)(id - (unsigned)rb * (unsigned)per_rb);
-  s.tile = rem / d.cpt;
-  s.kb0 = (rem - s.tile * d.cpt) * d.chunk_kb;
+  // row blocks vary fastest: the blocks of one weight chunk are claimed one after the other, so the chunk is
+  // streamed from HBM once and found in L2 by the later blocks
+  const int per_tile = d.cpt * d.nrb;
+  s.tile = (int)(id / (unsigned)per_tile);
+  const int rem = (int)(id - (unsigned)s.tile * (unsigned)per_tile);
+  const int kc = rem / d.nrb;
+  rb = rem - kc * d.nrb;
+  s.kb0 = kc * d.chunk_kb;
   s.kb1 = min(d.nkb, s.kb0 + d.chunk_kb);
 }
 
@@ -634,8 +638,7 @@ static void bn_config(int R, int &bn, int &stages, int &ctas_per_sm) {
   if (R <= 16) { bn = 16; stages = 5; ctas_per_sm = 2; }          // 5 x (16 + 2 x 2) KB
   else if (R <= 32) { bn = 32; stages = 4; ctas_per_sm = 2; }     // 4 x (16 + 2 x 4) KB
   else if (R <= 64) { bn = 64; stages = 6; ctas_per_sm = 1; }     // 6 x (16 + 2 x 8) KB
-  else if (R <= 128) { bn = 128; stages = 6; ctas_per_sm = 1; }
-  else { bn = 256; stages = 4; ctas_per_sm = 1; }
+  else { bn = 128; stages = 4; ctas_per_sm = 1; }                 // 4 x (16 + 2 x 16) KB; more rows: blocks of 128
 }
 
 UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsigned int *err_word,
@@ -698,8 +701,7 @@ static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, i
     case 16: return launch_one<EPI, 16>(maps, p, grid, st);
     case 32: return launch_one<EPI, 32>(maps, p, grid, st);
     case 64: return launch_one<EPI, 64>(maps, p, grid, st);
-    case 128: return launch_one<EPI, 128>(maps, p, grid, st);
-    default: return launch_one<EPI, 256>(maps, p, grid, st);
+    default: return launch_one<EPI, 128>(maps, p, grid, st);
   }
 }
 
@@ -735,6 +737,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
     if (chunks > 0x7fffffffLL) return cudaErrorInvalidValue;
     d.n_chunks = (int)chunks;
+    d.nrb = nrb;
     if (chunks > max_chunks) max_chunks = chunks;
   }
   for (int i = n; i < kMaxPhases; ++i)
