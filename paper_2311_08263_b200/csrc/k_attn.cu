@@ -451,8 +451,26 @@ static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
   }
+  // Largest cluster this kernel can be scheduled with: 16 (non-portable size) if the device takes it, else 8.
+  static int max_cluster = 0;
+  if (max_cluster == 0) {
+    max_cluster = 8;
+    if (cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t q;
+      memset(&q, 0, sizeof q);
+      q.gridDim = dim3(16, 1, 1); q.blockDim = dim3(kAttnThreads); q.dynamicSmemBytes = smem;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 16; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+      q.attrs = qa; q.numAttrs = 1;
+      int n_clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&n_clusters, attn_fused_kernel<HD>, &q) == cudaSuccess && n_clusters > 0)
+        max_cluster = 16;
+    }
+    (void)cudaGetLastError();
+  }
   FusedAttnArgs args = a;
-  args.cluster = (a.nsplit >= 2 && a.nsplit <= 8) ? 1 : 0;     // portable cluster size
+  args.cluster = (a.nsplit >= 2 && a.nsplit <= max_cluster) ? 1 : 0;
   if (args.cluster) {
     attr[na].id = cudaLaunchAttributeClusterDimension;
     attr[na].val.clusterDim.x = (unsigned)a.nsplit; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
