@@ -82,28 +82,25 @@ static inline float wload(const void *p, int wdtype, size_t i) {
   return wdtype ? bf16_to_f32(((const uint16_t *)p)[i]) : ((const float *)p)[i];
 }
 
-/* dot(w_row, x) over n terms; 16 interleaved partial sums added in a fixed order.  The products and sums are
- * carried in double (inputs and the result are fp32), so that a projection is the correctly rounded fp32 value
- * of the exact sum to within a few 1e-8: K and V rows that are later rounded to bfloat16 then land on the
- * wrong side of a rounding boundary far less often than with fp32 partial sums. */
+/* dot(w_row, x) over n terms; 16 interleaved partial sums added in a fixed order. */
 static float dot_row(const void *w, int wdtype, size_t row, int n, const float *x) {
-  double acc[16];
-  for (int j = 0; j < 16; ++j) acc[j] = 0.0;
+  float acc[16];
+  for (int j = 0; j < 16; ++j) acc[j] = 0.f;
   int k = 0;
   if (wdtype) {
     const uint16_t *wr = (const uint16_t *)w + row * (size_t)n;
     for (; k + 16 <= n; k += 16)
-      for (int j = 0; j < 16; ++j) acc[j] += (double)bf16_to_f32(wr[k + j]) * (double)x[k + j];
-    for (int j = 0; k < n; ++k, ++j) acc[j] += (double)bf16_to_f32(wr[k]) * (double)x[k];
+      for (int j = 0; j < 16; ++j) acc[j] += bf16_to_f32(wr[k + j]) * x[k + j];
+    for (int j = 0; k < n; ++k, ++j) acc[j] += bf16_to_f32(wr[k]) * x[k];
   } else {
     const float *wr = (const float *)w + row * (size_t)n;
     for (; k + 16 <= n; k += 16)
-      for (int j = 0; j < 16; ++j) acc[j] += (double)wr[k + j] * (double)x[k + j];
-    for (int j = 0; k < n; ++k, ++j) acc[j] += (double)wr[k] * (double)x[k];
+      for (int j = 0; j < 16; ++j) acc[j] += wr[k + j] * x[k + j];
+    for (int j = 0; k < n; ++k, ++j) acc[j] += wr[k] * x[k];
   }
-  double s = 0.0;
+  float s = 0.f;
   for (int j = 0; j < 16; ++j) s += acc[j];
-  return (float)s;
+  return s;
 }
 
 /* Y[r, o] = dot(W[o, :], X[r, :]) for r < rows; parallel over output features only. */

@@ -28,12 +28,10 @@ constexpr int kWBytes = kTileM * kTileK * 2;
 constexpr int kThreads = 320;
 constexpr unsigned long long kSpinBudget = 400000000ull;    // clock64 ticks (~0.2 s)
 
-// Activations are staged as three bf16 terms hi + mid + lo (each the bf16 rounding of what the previous ones left),
-// i.e. to fp32 accuracy: three MMAs per k-step against the same weight tile.  The tensor pipe is nearly idle on
-// this memory-bound kernel, and K/V rows that are later rounded to bf16 then fall on the same side of a rounding
-// boundary as an exact computation far more often.  More than 64 rows run as blocks of 64 on the same weight
-// chunk, back to back.
-constexpr int kXParts = 3;
+// Activations are staged as a bf16 pair hi + lo (lo = bf16(x - hi)): two MMAs per k-step against the same weight
+// tile, which removes the bf16 rounding of the activations.  Up to 128 rows the kernel stays memory-bound with the
+// doubled MMA work; more rows run as blocks of 128 on the same weight chunk, back to back.
+__host__ __device__ constexpr int x_parts(int bn) { return 2; }
 
 constexpr int kMaxPhases = 4;      // projections chained in one launch (O -> gate/up -> down -> next QKV)
 
@@ -240,10 +238,11 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
   return v;
 }
 
-// The 16-row width runs two CTAs per SM (the grid barrier needs the whole grid resident).
+// Widths up to 32 rows run two CTAs per SM (the grid barrier needs the whole grid resident).
 template <int EPI, int BN>
-__global__ void __launch_bounds__(kThreads, (BN <= 16 ? 2 : 1))
+__global__ void __launch_bounds__(kThreads, (BN <= 32 ? 2 : 1))
 gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ UmmaParams p) {
+  constexpr int kXParts = x_parts(BN);
   constexpr int kXBytes = BN * 128;                 // one staged activation tile (bf16, 64 k)
   constexpr int kStageBytes = kWBytes + kXParts * kXBytes;
   constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
@@ -497,17 +496,14 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
                 pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
                 pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
                 *reinterpret_cast<uint4 *>(xs + soff) = pk;
-#pragma unroll
-                for (int part = 1; part < kXParts; ++part) {      // what the earlier roundings lost
+                if (kXParts == 2) {      // low part: what the first rounding lost
                   const float2 h0 = __bfloat1622float2(b0), h1 = __bfloat1622float2(b1);
                   const float2 h2 = __bfloat1622float2(b2), h3 = __bfloat1622float2(b3);
-                  v[0] -= h0.x; v[1] -= h0.y; v[2] -= h1.x; v[3] -= h1.y;
-                  v[4] -= h2.x; v[5] -= h2.y; v[6] -= h3.x; v[7] -= h3.y;
-                  b0 = __floats2bfloat162_rn(v[0], v[1]); b1 = __floats2bfloat162_rn(v[2], v[3]);
-                  b2 = __floats2bfloat162_rn(v[4], v[5]); b3 = __floats2bfloat162_rn(v[6], v[7]);
-                  pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
-                  pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
-                  *reinterpret_cast<uint4 *>(xs + part * kXBytes + soff) = pk;
+                  __nv_bfloat162 l0 = __floats2bfloat162_rn(v[0] - h0.x, v[1] - h0.y), l1 = __floats2bfloat162_rn(v[2] - h1.x, v[3] - h1.y);
+                  __nv_bfloat162 l2 = __floats2bfloat162_rn(v[4] - h2.x, v[5] - h2.y), l3 = __floats2bfloat162_rn(v[6] - h3.x, v[7] - h3.y);
+                  pk.x = *reinterpret_cast<uint32_t *>(&l0); pk.y = *reinterpret_cast<uint32_t *>(&l1);
+                  pk.z = *reinterpret_cast<uint32_t *>(&l2); pk.w = *reinterpret_cast<uint32_t *>(&l3);
+                  *reinterpret_cast<uint4 *>(xs + kXBytes + soff) = pk;
                 }
               }
             }
@@ -639,8 +635,10 @@ static EncodeTiledFn get_encode_fn() {
 
 // accumulator width, ring depth and resident CTAs per SM for a row count
 static void bn_config(int R, int &bn, int &stages, int &ctas_per_sm) {
-  if (R <= 16) { bn = 16; stages = 4; ctas_per_sm = 2; }          // 4 x (16 + 3 x 2) KB, two CTAs per SM
-  else { bn = 64; stages = 5; ctas_per_sm = 1; }                  // 5 x (16 + 3 x 8) KB; more rows: blocks of 64
+  if (R <= 16) { bn = 16; stages = 5; ctas_per_sm = 2; }          // 5 x (16 + 2 x 2) KB
+  else if (R <= 32) { bn = 32; stages = 4; ctas_per_sm = 2; }     // 4 x (16 + 2 x 4) KB
+  else if (R <= 64) { bn = 64; stages = 6; ctas_per_sm = 1; }     // 6 x (16 + 2 x 8) KB
+  else { bn = 128; stages = 4; ctas_per_sm = 1; }                 // 4 x (16 + 2 x 16) KB; more rows: blocks of 128
 }
 
 UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsigned int *err_word,
@@ -680,7 +678,7 @@ void umma_plan_destroy(UmmaPlan *p) { delete p; }
 
 template <int EPI, int BN>
 static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid, cudaStream_t st) {
-  const size_t smem = (size_t)p.stages * (kWBytes + kXParts * BN * 128) + 1024;
+  const size_t smem = (size_t)p.stages * (kWBytes + x_parts(BN) * BN * 128) + 1024;
   static size_t attr_smem = 0;
   if (smem > attr_smem) {
     cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -699,8 +697,12 @@ static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid
 
 template <int EPI>
 static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, int grid, cudaStream_t st) {
-  if (bn == 16) return launch_one<EPI, 16>(maps, p, grid, st);
-  return launch_one<EPI, 64>(maps, p, grid, st);
+  switch (bn) {
+    case 16: return launch_one<EPI, 16>(maps, p, grid, st);
+    case 32: return launch_one<EPI, 32>(maps, p, grid, st);
+    case 64: return launch_one<EPI, 64>(maps, p, grid, st);
+    default: return launch_one<EPI, 128>(maps, p, grid, st);
+  }
 }
 
 // One launch that runs plans[0..n-1] back to back on the same rows; plan i+1 consumes what plan i reduced
