@@ -1,4 +1,5 @@
 // C ABI of the Jacobi-window decode library: context, workspace carving, the per-step kernel chain.
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -289,7 +290,22 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   if (cudaMallocHost((void **)&ctx->pin, pin_ints * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaEventCreate(&ctx->ev0) != cudaSuccess || cudaEventCreate(&ctx->ev1) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaMemsetAsync(ws, 0, fc_workspace_bytes(shape), ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
-  if (launch_rope_table(ctx->b.rope, shape->max_seq, shape->head_dim, shape->rope_theta, ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
+  {
+    // cos/sin of pos * theta^(-2i/hd), evaluated on the host in fp32 (inverse frequency in fp32, angle in fp32):
+    // the device's powf is a few ulp off, and at positions in the thousands an ulp of the frequency is 1e-4 rad
+    // of rotation.
+    const int half = shape->head_dim / 2;
+    std::vector<float2> table((size_t)shape->max_seq * half);
+    std::vector<float> inv_freq(half);
+    for (int i = 0; i < half; ++i) inv_freq[i] = powf(shape->rope_theta, -2.0f * (float)i / (float)shape->head_dim);
+    for (int pos = 0; pos < shape->max_seq; ++pos)
+      for (int i = 0; i < half; ++i) {
+        const float ang = (float)pos * inv_freq[i];
+        table[(size_t)pos * half + i] = make_float2(cosf(ang), sinf(ang));
+      }
+    if (cudaMemcpyAsync(ctx->b.rope, table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice, ctx->st) != cudaSuccess ||
+        cudaStreamSynchronize(ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
+  }
   if (cudaStreamSynchronize(ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
   const int B = shape->max_batch;
   ctx->kv_len_h.assign(B, 0); ctx->n_gen_h.assign(B, 0); ctx->pending_h.assign(B, 0); ctx->done_h.assign(B, 0);

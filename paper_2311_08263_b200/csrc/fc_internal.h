@@ -131,7 +131,6 @@ cudaError_t launch_embed(const EmbedArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_gemm_simt(const GemmArgs &a, int dtype, int pro, int epi, cudaStream_t st);
 cudaError_t launch_rope_kv(const RopeArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st);
-cudaError_t launch_rope_table(float2 *table, int max_seq, int hd, float theta, cudaStream_t st);
 cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st);
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 int attn_tile_keys(int dtype, int hd);   // keys per split tile

@@ -488,21 +488,4 @@ cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st) {
 
 int attn_fused_chunk() { return kChunk; }
 
-// cos/sin of pos * theta^(-2i/hd), computed once per context with the precise library routines.
-__global__ void rope_table_kernel(float2 *table, int max_seq, int half, float theta) {
-  const long long n = (long long)max_seq * half;
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (long long)gridDim.x * blockDim.x) {
-    const int pos = (int)(e / half), i = (int)(e % half);
-    const float freq = powf(theta, -2.0f * (float)i / (float)(2 * half));
-    float sn, cs;
-    sincosf((float)pos * freq, &sn, &cs);
-    table[e] = make_float2(cs, sn);
-  }
-}
-
-cudaError_t launch_rope_table(float2 *table, int max_seq, int hd, float theta, cudaStream_t st) {
-  rope_table_kernel<<<296, 256, 0, st>>>(table, max_seq, hd / 2, theta);
-  return cudaGetLastError();
-}
-
 }  // namespace fc
