@@ -313,6 +313,57 @@ def run_ours(args, cfg, rank, world, local):
         print(json.dumps(line), flush=True)
 
 
+def run_sweep(args, cfg):
+    """Window-step sweep (the paper's Fig. 2 experiment: forward time against window size and prompt length):
+    K/V length x window rows x batch on one model shape, random weights, seeded random K/V ~ N(0,1) written
+    straight into the cache, steps that do not commit so every step runs at the same length.  One JSON line per
+    point: latency, algorithmic bytes and flops, fraction of the HBM roofline."""
+    from paper_2311_08263_b200 import engine
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peaks()
+    w = wl.make_weights(cfg, device="cuda")
+    lens = [int(x) for x in args.sweep_lens.split(",")]
+    cs = [int(x) for x in args.sweep_c.split(",")]
+    bs = [int(x) for x in args.sweep_batch.split(",")]
+    g = torch.Generator(device="cuda")
+    for L in lens:
+        for B in bs:
+            max_c = max(cs)
+            max_seq = L + max_c + 8
+            need = cfg.kv_bytes_per_token() * max_seq * B * 1.02 + 6e9
+            free, _ = torch.cuda.mem_get_info()
+            if need > free:
+                for c in cs:
+                    print(json.dumps({"sweep": cfg.name, "kv_len": L, "c": c, "batch": B, "skipped": "does not fit in device memory"}), flush=True)
+                continue
+            dec = engine.Decoder(cfg, w, B, max_c, max_seq)
+            g.manual_seed(cfg.seed + L + B)
+            kv = dec.kv.view(cfg.torch_dtype)
+            for i in range(0, kv.numel(), 1 << 30):
+                kv[i:i + (1 << 30)].normal_(generator=g)
+            for c in cs:
+                pending = wl.make_random_window(cfg, B, 1, salt=c).numpy()[:, 0]
+                dec.fc_debug_set_state([L] * B, pending, c, pad_id=1)
+                ms1, _ = dec.fc_bench_steps(2)
+                n = int(max(3, min(50, 300.0 / max(ms1 / 2, 0.05))))
+                ms, _ = dec.fc_bench_steps(n)
+                step_ms = ms / n
+                by = step_bytes(cfg, B, c, [L] * B)
+                R = B * c
+                flops = 2.0 * R * cfg.weight_params() + 4.0 * cfg.n_layers * cfg.n_heads * cfg.head_dim * B * c * (L + c / 2)
+                gbs = by / (step_ms * 1e-3) / 1e9
+                print(json.dumps({"sweep": cfg.name, "kv_len": L, "c": c, "batch": B, "rows": R, "ms_per_step": round(step_ms, 4),
+                                  "bytes_per_step": by, "flops_per_step": flops, "achieved_gbs": round(gbs, 1),
+                                  "frac_of_peak": round(gbs / peak, 4), "peak_kind": peak_kind,
+                                  "frac_of_8tbs": round(gbs / 8000.0, 4),
+                                  "achieved_tflops": round(flops / (step_ms * 1e-3) / 1e12, 2), "steps": n}), flush=True)
+            dec.close()
+            del dec, kv
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -323,6 +374,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: keep only the first N layers (same kernel shapes, less device memory)")
+    ap.add_argument("--sweep", action="store_true", help="window-step sweep instead of the benchmark line")
+    ap.add_argument("--sweep-lens", default="512,2048,8192")
+    ap.add_argument("--sweep-c", default="1,4,8,16,32,64")
+    ap.add_argument("--sweep-batch", default="1,4,16,32")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -330,6 +385,9 @@ def main():
     if args.layers > 0:
         import dataclasses
         cfg = dataclasses.replace(cfg, n_layers=args.layers, name=f"{cfg.name}-first{args.layers}layers")
+    if args.sweep:
+        run_sweep(args, cfg)
+        return
     rank, world, local = dist_setup(args.gpus)
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
