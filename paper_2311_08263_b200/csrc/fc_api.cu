@@ -24,8 +24,11 @@ struct Carver {          // hands out aligned slices of the caller's workspace (
   }
 };
 
+constexpr int kSyncWords = 12;
+
 struct Buffers {
-  float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *part_o, *part_ml;
+  float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *ss_final, *part_o, *part_ml;
+  void *pan;
   float2 *rope;
   void *qb;
   unsigned int *counters, *err, *chain_bar;
@@ -34,7 +37,7 @@ struct Buffers {
 };
 
 struct Dims {
-  int rmax, qd, kvd, ldq, nsplit_max, tk;
+  int rmax, qd, kvd, ldq, nsplit_max, tk, pan_rows, pan_k;
   size_t esz;
 };
 
@@ -58,6 +61,10 @@ Dims dims_of(const fc_model_shape *s) {
   d.tk = attn_tile_keys(s->dtype, s->head_dim);
   d.nsplit_max = (s->max_seq + d.tk - 1) / d.tk;
   d.esz = s->dtype == FC_F32 ? 4 : 2;
+  // beyond 16 rows the tensor-core projections read their activations from a bf16 high/low panel
+  d.pan_rows = d.rmax > 16 ? (d.rmax + 127) / 128 * 128 : 0;
+  d.pan_k = s->d_model > s->d_ffn ? s->d_model : s->d_ffn;
+  if (d.qd > d.pan_k) d.pan_k = d.qd;
   return d;
 }
 
@@ -73,9 +80,12 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
   t.gu = c.take<float>(R * 2 * (size_t)s->d_ffn);
   t.ss_attn = c.take<float>(R);
   t.ss_ffn = c.take<float>(R);
-  // eight words per layer (three grid barriers, four work-claim counters) plus one group for the first QKV
-  // and the LM head; directly after the sums of squares so that one pass clears them all
-  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * 8);
+  t.ss_final = c.take<float>(R);
+  // kSyncWords words per layer (grid barriers 0..2, work-claim counters 4..7, panel-ready barriers 8..11) plus
+  // one group for the first QKV and the LM head; directly after the sums of squares so that one pass clears
+  // them all
+  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * kSyncWords);
+  t.pan = c.take<char>((size_t)2 * d.pan_rows * d.pan_k * 2);
   t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
   t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
   t.rope = c.take<float2>((size_t)s->max_seq * (s->head_dim / 2));
@@ -198,6 +208,7 @@ static GemmArgs args_qkv(const fc_ctx *c, int l) {
   a.n_rows[0] = c->d.qd; a.n_rows[1] = c->d.kvd; a.n_rows[2] = c->d.kvd;
   a.y_off[0] = 0; a.y_off[1] = c->d.qd; a.y_off[2] = c->d.qd + c->d.kvd;
   a.n_mats = 3; a.y = c->b.qkv; a.ldy = c->d.ldq; a.K = c->s.d_model;
+  a.pan = c->d.pan_rows ? c->b.pan : nullptr; a.pan_rows = c->d.pan_rows;
   return a;
 }
 static GemmArgs args_o(const fc_ctx *c, int l) {
@@ -205,6 +216,7 @@ static GemmArgs args_o(const fc_ctx *c, int l) {
   a.x = c->b.attn; a.ldx = c->d.qd; a.eps = c->s.rms_eps; a.dn = c->s.d_model;
   a.w[0] = c->wo[l]; a.n_rows[0] = c->s.d_model; a.n_mats = 1;
   a.y = c->b.x; a.ldy = c->s.d_model; a.K = c->d.qd;
+  a.pan = c->d.pan_rows ? c->b.pan : nullptr; a.pan_rows = c->d.pan_rows;
   return a;
 }
 static GemmArgs args_gu(const fc_ctx *c, int l) {
@@ -214,6 +226,7 @@ static GemmArgs args_gu(const fc_ctx *c, int l) {
   a.w[0] = c->w_gate[l]; a.w[1] = c->w_up[l];
   a.n_rows[0] = c->s.d_ffn; a.n_rows[1] = c->s.d_ffn; a.y_off[0] = 0; a.y_off[1] = c->s.d_ffn;
   a.n_mats = 2; a.y = c->b.gu; a.ldy = 2 * c->s.d_ffn; a.K = c->s.d_model;
+  a.pan = c->d.pan_rows ? c->b.pan : nullptr; a.pan_rows = c->d.pan_rows;
   return a;
 }
 static GemmArgs args_down(const fc_ctx *c, int l) {
@@ -222,6 +235,7 @@ static GemmArgs args_down(const fc_ctx *c, int l) {
   a.eps = c->s.rms_eps; a.dn = c->s.d_model;
   a.w[0] = c->w_down[l]; a.n_rows[0] = c->s.d_model; a.n_mats = 1;
   a.y = c->b.x; a.ldy = c->s.d_model; a.K = c->s.d_ffn;
+  a.pan = c->d.pan_rows ? c->b.pan : nullptr; a.pan_rows = c->d.pan_rows;
   return a;
 }
 static GemmArgs args_head(const fc_ctx *c) {
@@ -230,6 +244,8 @@ static GemmArgs args_head(const fc_ctx *c) {
   a.w[0] = c->lm_head; a.n_rows[0] = c->s.vocab; a.n_mats = 1; a.K = c->s.d_model;
   a.tokens = c->b.window; a.perm = c->s.bias_beta != 0.f ? c->bias_perm : nullptr; a.beta = c->s.bias_beta;
   a.amax = c->b.amax; a.logits = c->dbg_logits; a.vocab = c->s.vocab; a.ldy = c->s.vocab;
+  a.ss_out = c->b.ss_final;     // panel mode only: the sums of squares of the final norm
+  a.pan = c->d.pan_rows ? c->b.pan : nullptr; a.pan_rows = c->d.pan_rows;
   return a;
 }
 
@@ -332,9 +348,9 @@ enum { GEMM_QKV = -1, GEMM_O = 0, GEMM_GU = 1, GEMM_DOWN = 2, GEMM_HEAD = 3 };
 static unsigned int *claim_word(fc_ctx *ctx, int l, int which) {
   const int L = ctx->s.n_layers;
   unsigned int *w = ctx->b.chain_bar;
-  if (which == GEMM_HEAD) return w + (size_t)L * 8 + 5;
-  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * 8 + 4 : w + (size_t)(l - 1) * 8 + 7;   // chained after down(l-1)
-  return w + (size_t)l * 8 + 4 + which;
+  if (which == GEMM_HEAD) return w + (size_t)L * kSyncWords + 5;
+  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * kSyncWords + 4 : w + (size_t)(l - 1) * kSyncWords + 7;   // chained after down(l-1)
+  return w + (size_t)l * kSyncWords + 4 + which;
 }
 
 static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls,
@@ -342,7 +358,7 @@ static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R
   ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
-  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, ctx->pdl && !ctx->prof, ctx->st);
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + 4, ctx->pdl && !ctx->prof, ctx->st);   // panel-ready word: four after the claim word
   return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
 }
 
@@ -360,7 +376,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   ea.z.p[1] = ctx->b.gu; ea.z.n[1] = Rz * 2 * s.d_ffn;
   // sums of squares (both norms) and the grid-barrier words of the chained projections are adjacent
   ea.z.p[2] = ctx->b.ss_attn;
-  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + ((size_t)s.n_layers + 1) * 8) - (char *)ctx->b.ss_attn) / sizeof(float);
+  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + ((size_t)s.n_layers + 1) * kSyncWords) - (char *)ctx->b.ss_attn) / sizeof(float);
   ++ctx->launches;
   { ProfScope ps(ctx, FC_CLS_EMBED); FC_CK(launch_embed(ea, s.dtype, ctx->st)); }
 
@@ -415,9 +431,10 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       for (int i = 0; i < n; ++i) ga[i].R = R;
       ++ctx->launches;
       ProfScope ps(ctx, FC_CLS_CHAIN);
-      // barriers at words 0..2 of the layer's group, claim counters at 4..7 (O, gate/up, down, next QKV)
-      FC_CK(launch_gemm_chain(plans, ga, n, ctx->b.chain_bar + (size_t)l * 8, ctx->b.chain_bar + (size_t)l * 8 + 4,
-                              ctx->pdl && !ctx->prof, ctx->st));
+      // barriers at words 0..2 of the layer's group, claim counters at 4..7 (O, gate/up, down, next QKV),
+      // panel-ready barriers at 8..11
+      unsigned int *grp = ctx->b.chain_bar + (size_t)l * kSyncWords;
+      FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + 4, grp + 8, ctx->pdl && !ctx->prof, ctx->st));
     } else {
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O)));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));
@@ -754,7 +771,7 @@ extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, 
   char msg[200];
   UmmaPlan *pl = umma_plan_create(a, PRO_NONE, EPI_ATOMIC_ADD, sms, err_word, msg, sizeof msg);
   if (!pl) { fprintf(stderr, "fc_op_linear: %s\n", msg); return FC_ERR_CUDA; }
-  cudaError_t e = launch_gemm_umma(pl, a, err_word + 1, 0, st);
+  cudaError_t e = launch_gemm_umma(pl, a, err_word + 1, nullptr, 0, st);
   unsigned int herr = 0;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&herr, err_word, sizeof herr, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);

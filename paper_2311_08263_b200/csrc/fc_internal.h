@@ -46,6 +46,10 @@ struct GemmArgs {
   unsigned long long *amax;       // [R] packed (ordered logit << 32 | ~index)
   float *logits;                  // optional dump [R, vocab]
   int vocab;
+  // more than 16 rows: bf16 panel [2][pan_rows][K] (high parts, then low parts) that the launch fills with pro(x) once
+  // and streams by TMA; with the argmax epilogue ss_out then holds the row sums of squares the epilogue reads
+  void *pan;
+  int pan_rows;
 };
 
 struct ZeroList {       // buffers a kernel clears on the side (fp32 words)
@@ -148,9 +152,11 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
 void umma_plan_destroy(UmmaPlan *p);
 // x/x2/y/ss pointers and R may differ per launch from those the plan was created with.
 // claim: one zeroed word per projection of the launch (the work-claim counters).
-cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int *claim, int pdl, cudaStream_t st);
+cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b, int pdl,
+                             cudaStream_t st);
 // Up to four projections in one launch, each consuming the previous one's reduced output; bar: n-1 zeroed words.
+// bar_b: n zeroed words (panel-ready barriers), needed when the rows exceed 16 and the plans have panels.
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
-                              unsigned int *claim, int pdl, cudaStream_t st);
+                              unsigned int *claim, unsigned int *bar_b, int pdl, cudaStream_t st);
 
 }  // namespace fc

@@ -45,7 +45,10 @@ struct PhaseDesc {
                                       // chunks per tile, row blocks, total
 };
 
-struct MapPack { CUtensorMap m[kMaxPhases * kMaxMats]; };
+struct MapPack {
+  CUtensorMap m[kMaxPhases * kMaxMats];   // weights
+  CUtensorMap x[kMaxPhases];              // activation panels (rows beyond 16)
+};
 
 struct UmmaParams {
   PhaseDesc ph[kMaxPhases];
@@ -55,11 +58,14 @@ struct UmmaParams {
   unsigned int *err;              // device error word (0 = ok)
   unsigned int *bar;              // [n_phases - 1] grid-barrier counters, zero when the kernel starts
   unsigned int *claim;            // [n_phases] work-claim counters, zero when the kernel starts
+  unsigned int *bar_b;            // [n_phases] panel-ready barriers (panel mode), zero when the kernel starts
 };
 
 struct UmmaPlan {
   PhaseDesc d;
   CUtensorMap maps[kMaxMats];
+  CUtensorMap xmap[3];            // activation panel [2 * pan_rows, K], boxes of 64 k x 32 / 64 / 128 rows
+  bool has_xmap;
   int epi, n_sms;
   unsigned int *err;
 };
@@ -229,6 +235,12 @@ __device__ __forceinline__ void tile_info(const PhaseDesc &d, int tile, int &m, 
   ycol0 = d.g.y_off[m] + row0;
 }
 
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -239,7 +251,9 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 }
 
 // Widths up to 32 rows run two CTAs per SM (the grid barrier needs the whole grid resident).
-template <int EPI, int BN>
+// PANEL: the activations come from a bf16 hi/lo panel in global memory, converted once per projection by all
+// CTAs together and streamed by TMA, instead of being converted by every CTA for every weight tile.
+template <int EPI, int BN, bool PANEL>
 __global__ void __launch_bounds__(kThreads, (BN <= 32 ? 2 : 1))
 gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ UmmaParams p) {
   constexpr int kXParts = x_parts(BN);
@@ -251,7 +265,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar, go_bar[kMaxPhases], seg_full[kSegQ], seg_empty[kSegQ];
   __shared__ int4 seg_q[kSegQ];          // (tile, kb0, kb1, row block)
-  __shared__ unsigned int bar_cnt_s[kMaxPhases];
+  __shared__ unsigned int bar_cnt_s[kMaxPhases], bar_cnt_b[kMaxPhases];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   __shared__ float ss_part[2][4][BN];   // per accumulator, per staging warp: partial sums of squares
@@ -266,7 +280,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&full_w[i]), 1); mbar_init(smem_u32(&full_x[i]), 1); mbar_init(smem_u32(&empty_b[i]), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
     mbar_init(smem_u32(&drain_bar), 1);
-    for (int i = 0; i < kMaxPhases; ++i) { mbar_init(smem_u32(&go_bar[i]), 1); bar_cnt_s[i] = 0u; }
+    for (int i = 0; i < kMaxPhases; ++i) { mbar_init(smem_u32(&go_bar[i]), 1); bar_cnt_s[i] = 0u; bar_cnt_b[i] = 0u; }
     // a queue slot is read by the MMA thread, four staging warps and four epilogue warps
     for (int i = 0; i < kSegQ; ++i) { mbar_init(smem_u32(&seg_full[i]), 1); mbar_init(smem_u32(&seg_empty[i]), 9); }
     fence_barrier_init();
@@ -413,6 +427,130 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
         if (!ok) break;
       }
+      if constexpr (PANEL) {
+        // ---- (1) all CTAs together convert pro(x) into the bf16 panel [high | low] once; a warp takes 32
+        // consecutive (row, 8-wide chunk) units at a time, four such groups per pass so that the loads overlap
+        {
+          const int kc8 = g.K >> 3;
+          const int units = g.R * kc8;                       // the host keeps R * K / 8 below 2^31
+          const int n_groups = (units + 31) >> 5;
+          const int warps_total = (int)gridDim.x * 4;
+          __nv_bfloat16 *pan_hi = (__nv_bfloat16 *)g.pan;
+          __nv_bfloat16 *pan_lo = pan_hi + (long long)g.pan_rows * g.K;
+          const bool want_ss = pro == PRO_GAIN && g.ss_out != nullptr;
+          for (int g0 = (int)blockIdx.x * 4 + sw; g0 < n_groups; g0 += 4 * warps_total) {
+            float4 xa[4], xb[4], ua[4], ubv[4];
+            float ssr[4];
+            uint4 gq[4];
+            int un[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              un[j] = g0 + j * warps_total < n_groups ? ((g0 + j * warps_total) << 5) + lane : units;
+              xa[j] = xb[j] = ua[j] = ubv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+              ssr[j] = 0.f; gq[j] = make_uint4(0, 0, 0, 0);
+              if (un[j] < units) {
+                const int r = un[j] / kc8, k = (un[j] - r * kc8) << 3;
+                const float *px = g.x + (long long)r * g.ldx + k;
+                xa[j] = __ldcg(reinterpret_cast<const float4 *>(px));
+                xb[j] = __ldcg(reinterpret_cast<const float4 *>(px + 4));
+                if (pro == PRO_GAIN) gq[j] = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
+                if (pro == PRO_SILU_MUL) {
+                  const float *pu = g.x2 + (long long)r * g.ldx + k;
+                  ua[j] = __ldcg(reinterpret_cast<const float4 *>(pu));
+                  ubv[j] = __ldcg(reinterpret_cast<const float4 *>(pu + 4));
+                  ssr[j] = __ldcg(g.ss_in + r);
+                }
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const bool live = un[j] < units;
+              const int r = live ? un[j] / kc8 : -1;
+              float v[8] = {xa[j].x, xa[j].y, xa[j].z, xa[j].w, xb[j].x, xb[j].y, xb[j].z, xb[j].w};
+              float sq = 0.f;
+              if (pro == PRO_GAIN) {
+                const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq[j]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float2 gf = __bfloat1622float2(gp[i]);
+                  sq = fmaf(v[2 * i], v[2 * i], sq); sq = fmaf(v[2 * i + 1], v[2 * i + 1], sq);
+                  v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
+                }
+              } else if (pro == PRO_SILU_MUL) {
+                const float sr = rsqrtf(ssr[j] / (float)g.dn + g.eps);
+                const float uu[8] = {ua[j].x, ua[j].y, ua[j].z, ua[j].w, ubv[j].x, ubv[j].y, ubv[j].z, ubv[j].w};
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float gt = sr * v[i];
+                  v[i] = __fdividef(gt, 1.0f + __expf(-gt)) * (sr * uu[i]);
+                }
+              }
+              if (want_ss) {
+                // lanes of a group usually share the row: one reduction per group, else one per lane
+                const int r0 = __shfl_sync(0xffffffffu, r, 0);
+                if (__all_sync(0xffffffffu, r == r0)) {
+                  const float t = warp_sum_f(sq);
+                  if (lane == 0 && r0 >= 0) atomicAdd(&g.ss_out[r0], t);
+                } else if (live) {
+                  atomicAdd(&g.ss_out[r], sq);
+                }
+              }
+              if (live) {
+                const int k = (un[j] - r * kc8) << 3;
+                uint4 pk;
+                __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
+                __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
+                pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+                pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+                *reinterpret_cast<uint4 *>(pan_hi + (long long)r * g.K + k) = pk;
+                const float2 h0 = __bfloat1622float2(b0), h1 = __bfloat1622float2(b1);
+                const float2 h2 = __bfloat1622float2(b2), h3 = __bfloat1622float2(b3);
+                b0 = __floats2bfloat162_rn(v[0] - h0.x, v[1] - h0.y); b1 = __floats2bfloat162_rn(v[2] - h1.x, v[3] - h1.y);
+                b2 = __floats2bfloat162_rn(v[4] - h2.x, v[5] - h2.y); b3 = __floats2bfloat162_rn(v[6] - h3.x, v[7] - h3.y);
+                pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+                pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+                *reinterpret_cast<uint4 *>(pan_lo + (long long)r * g.K + k) = pk;
+              }
+            }
+          }
+        }
+        // ---- (2) panel-ready barrier: the four staging warps of every CTA have stored their share
+        asm volatile("fence.proxy.async;" ::: "memory");      // generic-proxy stores before the TMA reads that follow the barrier
+        __threadfence();
+        __syncwarp();
+        if (lane == 0 && atomicAdd(&bar_cnt_b[pi], 1u) == 3u) { __threadfence(); atomicAdd(p.bar_b + pi, 1u); }
+        if (sw == 0) {
+          ok = grid_bar_wait(p.bar_b + pi, gridDim.x, lane, abort_flag);
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        // ---- (3) warp 0 streams the activation tiles of every claimed k-block into the ring; the other three
+        // staging warps only follow the queue
+        {
+          Segment s;
+          int rb = 0;
+          while (ok) {
+            const int got = take_warp(sq, s, rb);
+            if (got <= 0) { ok = got == 0; break; }
+            if (sw != 0) { it += s.kb1 - s.kb0; ++seg; continue; }
+            for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
+              const int stage = it % S;
+              const uint32_t ph = (uint32_t)(it / S) & 1u;
+              if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+              if (lane == 0) {
+                const uint32_t bar = smem_u32(&full_x[stage]);
+                const uint32_t xs = smem_base + stage * kStageBytes + kWBytes;
+                mbar_expect_tx(bar, (uint32_t)(kXParts * kXBytes));
+#pragma unroll
+                for (int part = 0; part < kXParts; ++part)
+                  tma_load_2d(xs + part * kXBytes, &maps.x[pi], kb * kTileK, part * g.pan_rows + rb * BN, bar);
+              }
+            }
+            ++seg;
+          }
+        }
+        if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+        continue;
+      }
       {
         Segment s;
         int rb = 0;
@@ -550,7 +688,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           const int acc = seg & 1;
           const uint32_t ph = ((uint32_t)seg >> 1) & 1u;
           if (!mbar_wait_warp(smem_u32(&accum_full[acc]), ph, abort_flag)) { ok = false; break; }
-          if (EPI == EPI_ARGMAX && !mbar_wait_warp(smem_u32(&ss_ready[acc]), ph, abort_flag)) { ok = false; break; }
+          if (EPI == EPI_ARGMAX && !PANEL && !mbar_wait_warp(smem_u32(&ss_ready[acc]), ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const bool valid = n_local < rows_valid;
           const int col = ycol0 + n_local;
@@ -565,7 +703,8 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
               if (EPI == EPI_ATOMIC_ADD) {
                 if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
               } else {
-                const float ssum = ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
+                const float ssum = PANEL ? __ldcg(g.ss_out + r)
+                                         : ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
                 float logit = v[j] * rsqrtf(ssum / (float)g.dn + g.eps);
                 unsigned long long key = 0ull;
                 if (valid) {
@@ -671,17 +810,33 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
     if (r != CUDA_SUCCESS) { delete pl; return fail("cuTensorMapEncodeTiled failed (weight pointer must be 16-byte aligned)"); }
   }
   for (int m = a.n_mats; m < kMaxMats; ++m) pl->maps[m] = pl->maps[0];
+  if (a.pan) {
+    // activation panel [high rows | low rows] x K, one map per accumulator width (the box is bn rows high)
+    if (a.pan_rows < 1 || a.pan_rows % kTileM || (long long)a.pan_rows * (a.K / 8) > 0x7fffffffLL) { delete pl; return fail("bad activation panel"); }
+    const int widths[3] = {32, 64, 128};
+    for (int i = 0; i < 3; ++i) {
+      cuuint64_t gdim[2] = {(cuuint64_t)a.K, (cuuint64_t)2 * a.pan_rows};
+      cuuint64_t gstr[1] = {(cuuint64_t)a.K * 2};
+      cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)widths[i]};
+      cuuint32_t estr[2] = {1, 1};
+      CUresult r = enc(&pl->xmap[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.pan, gdim, gstr, box, estr,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) { delete pl; return fail("cuTensorMapEncodeTiled failed (activation panel)"); }
+    }
+    pl->has_xmap = true;
+  }
   return pl;
 }
 
 void umma_plan_destroy(UmmaPlan *p) { delete p; }
 
-template <int EPI, int BN>
+template <int EPI, int BN, bool PANEL>
 static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid, cudaStream_t st) {
   const size_t smem = (size_t)p.stages * (kWBytes + x_parts(BN) * BN * 128) + 1024;
   static size_t attr_smem = 0;
   if (smem > attr_smem) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<EPI, BN, PANEL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_smem = smem;
   }
@@ -692,24 +847,34 @@ static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = p.pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<EPI, BN>, maps, p);
+  return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<EPI, BN, PANEL>, maps, p);
 }
 
 template <int EPI>
-static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, int grid, cudaStream_t st) {
+static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, bool panel, int grid, cudaStream_t st) {
+  if (panel) {
+    switch (bn) {
+      case 32: return launch_one<EPI, 32, true>(maps, p, grid, st);
+      case 64: return launch_one<EPI, 64, true>(maps, p, grid, st);
+      case 128: return launch_one<EPI, 128, true>(maps, p, grid, st);
+      default: return cudaErrorInvalidValue;
+    }
+  }
   switch (bn) {
-    case 16: return launch_one<EPI, 16>(maps, p, grid, st);
-    case 32: return launch_one<EPI, 32>(maps, p, grid, st);
-    case 64: return launch_one<EPI, 64>(maps, p, grid, st);
-    default: return launch_one<EPI, 128>(maps, p, grid, st);
+    case 16: return launch_one<EPI, 16, false>(maps, p, grid, st);
+    case 32: return launch_one<EPI, 32, false>(maps, p, grid, st);
+    case 64: return launch_one<EPI, 64, false>(maps, p, grid, st);
+    default: return launch_one<EPI, 128, false>(maps, p, grid, st);
   }
 }
 
 // One launch that runs plans[0..n-1] back to back on the same rows; plan i+1 consumes what plan i reduced
 // into its output, separated by a grid barrier on bar[i] (zero at launch).  args[i] carries the per-launch
 // buffers and the row count; weights, K and the matrix split stay as planned.
+// Beyond 16 rows, plans that own an activation panel run in panel mode: bar_b[i] (zero at launch) is the
+// panel-ready barrier of phase i.
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
-                              unsigned int *claim, int pdl, cudaStream_t st) {
+                              unsigned int *claim, unsigned int *bar_b, int pdl, cudaStream_t st) {
   if (n < 1 || n > kMaxPhases || !claim) return cudaErrorInvalidValue;
   if (n > 1 && !bar) return cudaErrorInvalidValue;
   MapPack maps;
@@ -720,6 +885,9 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
   bn_config(args[0].R, bn, p.stages, cps);
   const int nrb = (args[0].R + bn - 1) / bn;
   const int tile_mode = (epi == EPI_ARGMAX) ? 1 : 0;
+  bool panel = bar_b != nullptr && args[0].R > 16;
+  for (int i = 0; i < n; ++i) panel = panel && plans[i]->has_xmap && args[0].R <= plans[i]->d.g.pan_rows;
+  if (panel && epi == EPI_ARGMAX && !args[0].ss_out) return cudaErrorInvalidValue;
   long long max_chunks = 1;
   for (int i = 0; i < n; ++i) {
     const UmmaPlan *pl = plans[i];
@@ -730,6 +898,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.g.x = a.x; d.g.x2 = a.x2; d.g.ldx = a.ldx; d.g.ss_in = a.ss_in; d.g.ss_out = a.ss_out;
     d.g.y = a.y; d.g.ldy = a.ldy; d.g.R = a.R; d.g.tokens = a.tokens; d.g.amax = a.amax; d.g.logits = a.logits;
     for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = pl->maps[m];
+    maps.x[i] = pl->xmap[bn == 32 ? 0 : bn == 64 ? 1 : 2];
     // the argmax epilogue needs whole tiles; partial sums may be split along k into chunks of four k-blocks
     // (one k-block per staging warp)
     d.chunk_kb = tile_mode ? d.nkb : 4;
@@ -740,20 +909,23 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.nrb = nrb;
     if (chunks > max_chunks) max_chunks = chunks;
   }
-  for (int i = n; i < kMaxPhases; ++i)
+  for (int i = n; i < kMaxPhases; ++i) {
     for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = plans[0]->maps[0];
-  p.n_phases = n; p.pdl = pdl; p.err = plans[0]->err; p.bar = bar; p.claim = claim;
+    maps.x[i] = plans[0]->xmap[0];
+  }
+  p.n_phases = n; p.pdl = pdl; p.err = plans[0]->err; p.bar = bar; p.claim = claim; p.bar_b = bar_b;
   // Staging warps own every fourth k-block and run ahead of each other; the parity waits on the ring
   // are only unambiguous while the ring is at least as deep as the number of staging warps.
   if (p.stages < 4 || p.stages > 8) return cudaErrorInvalidValue;
   const long long resident = (long long)plans[0]->n_sms * cps;     // the grid barrier needs every CTA resident
   const int grid = (int)(resident < max_chunks ? resident : max_chunks);
-  if (epi == EPI_ARGMAX) return launch_bn<EPI_ARGMAX>(maps, p, bn, grid, st);
-  return launch_bn<EPI_ATOMIC_ADD>(maps, p, bn, grid, st);
+  if (epi == EPI_ARGMAX) return launch_bn<EPI_ARGMAX>(maps, p, bn, panel, grid, st);
+  return launch_bn<EPI_ATOMIC_ADD>(maps, p, bn, panel, grid, st);
 }
 
-cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, int pdl, cudaStream_t st) {
-  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, pdl, st);
+cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b, int pdl,
+                             cudaStream_t st) {
+  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, pdl, st);
 }
 
 }  // namespace fc

@@ -161,6 +161,43 @@ def test_batch_ragged_prompts_independent_accepts():
     assert st.tokens == B * cfg.gen_tokens
 
 
+@pytest.mark.parametrize("B,c", [(3, 8), (4, 12), (6, 16), (10, 16)], ids=["rows24", "rows48", "rows96", "rows160"])
+@pytest.mark.parametrize("shape", ["gqa64", "gqa32"])
+def test_many_rows_prefill_and_steps(B, c, shape):
+    """More than 16 rows per forward: the projections read their activations from the converted panel, for
+    every accumulator width (32, 64, 128 rows) and for two blocks of rows; the prefill runs through the same path.
+    gqa32 has k extents that are not multiples of 256, so a group of conversion units spans two rows."""
+    kw = {"gqa64": dict(n_heads=4, n_kv_heads=2, head_dim=64, d_model=256, d_ffn=512),
+          "gqa32": dict(n_heads=8, n_kv_heads=2, head_dim=32, d_model=320, d_ffn=328)}[shape]
+    cfg = wl.small_config(vocab=700, n_layers=2, prompt_len=200, c=c, gen_tokens=12, **kw)
+    lens = [200 - 17 * b for b in range(B)]
+    w = wl.make_weights(cfg)
+    max_seq = 200 + 12 + c + 8
+    dec = engine.Decoder(cfg, w, B, c, max_seq)
+    ids, _ = wl.make_prompts(cfg, batch=B, lens=lens)
+    dec.fc_prefill(ids.numpy(), lens, c)
+    logits = dec.fc_debug_logits(True)
+    orcs = []
+    for b in range(B):
+        o = oracle.Oracle(cfg, w, max_seq)
+        o.prefill(ids[b, :lens[b]].numpy(), c)
+        orcs.append(o)
+    in_step = True
+    for _ in range(2):
+        cnt, tok, wg = dec.fc_jacobi_step()
+        got = logits[:B * c].cpu().numpy().reshape(B, c, cfg.vocab)
+        for b in range(B):
+            k, acc, wnew, lg = orcs[b].jacobi_step(want_logits=True)
+            assert np.abs(got[b] - lg).max() < LOGIT_TOL
+            srt = np.sort(lg, axis=1)
+            if (srt[:, -1] - srt[:, -2]).min() > MARGIN_TOL:
+                assert cnt[b] == k and tok[b, :k].tolist() == acc.tolist() and wg[b].tolist() == wnew.tolist()
+            else:
+                in_step = False
+        if not in_step:
+            break
+
+
 def test_directed_accepts_in_a_batch_are_per_sequence():
     cfg = wl.CONFIGS["tiny"]
     B, c = 3, 6
