@@ -43,6 +43,7 @@ struct PhaseDesc {
   int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
   int chunk_kb, cpt, nrb, n_chunks;   // work is claimed in chunks of chunk_kb k-blocks of one tile for one block of rows:
                                       // chunks per tile, row blocks, total
+  int k_major;                        // claim order: all tiles of one k range before the next k range
 };
 
 struct MapPack {
@@ -217,6 +218,18 @@ constexpr int kSegQ = 8;           // queue slots (power of two)
 __device__ __forceinline__ void chunk_decode(const PhaseDesc &d, unsigned int id, Segment &s, int &rb) {
   // row blocks vary fastest: the blocks of one weight chunk are claimed one after the other, so the chunk is
   // streamed from HBM once and found in L2 by the later blocks
+  if (d.k_major) {
+    // with many rows the partial sums of one chunk are a lot of reductions; CTAs that claim one after the other
+    // then work on different tiles, so their reductions do not meet on the same addresses
+    const int per_k = d.n_tiles * d.nrb;
+    const int kc = (int)(id / (unsigned)per_k);
+    const int rem = (int)(id - (unsigned)kc * (unsigned)per_k);
+    s.tile = rem / d.nrb;
+    rb = rem - s.tile * d.nrb;
+    s.kb0 = kc * d.chunk_kb;
+    s.kb1 = min(d.nkb, s.kb0 + d.chunk_kb);
+    return;
+  }
   const int per_tile = d.cpt * d.nrb;
   s.tile = (int)(id / (unsigned)per_tile);
   const int rem = (int)(id - (unsigned)s.tile * (unsigned)per_tile);
@@ -695,6 +708,15 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           for (int c0 = 0; c0 < BN; c0 += 16) {
             if (rb * BN + c0 >= g.R) break;
             float v[16];
+            float ssum[16];
+            if (EPI == EPI_ARGMAX) {      // all sixteen loads before the first use
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int r = rb * BN + c0 + j;
+                ssum[j] = PANEL ? (r < g.R ? __ldcg(g.ss_out + r) : 0.f)
+                                : ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
+              }
+            }
             tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -703,9 +725,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
               if (EPI == EPI_ATOMIC_ADD) {
                 if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
               } else {
-                const float ssum = PANEL ? __ldcg(g.ss_out + r)
-                                         : ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
-                float logit = v[j] * rsqrtf(ssum / (float)g.dn + g.eps);
+                float logit = v[j] * rsqrtf(ssum[j] / (float)g.dn + g.eps);
                 unsigned long long key = 0ull;
                 if (valid) {
                   if (g.perm && g.perm[g.tokens[r]] == col) logit += g.beta;
@@ -899,9 +919,11 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.g.y = a.y; d.g.ldy = a.ldy; d.g.R = a.R; d.g.tokens = a.tokens; d.g.amax = a.amax; d.g.logits = a.logits;
     for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = pl->maps[m];
     maps.x[i] = pl->xmap[bn == 32 ? 0 : bn == 64 ? 1 : 2];
-    // the argmax epilogue needs whole tiles; partial sums may be split along k into chunks of four k-blocks
-    // (one k-block per staging warp)
-    d.chunk_kb = tile_mode ? d.nkb : 4;
+    // the argmax epilogue needs whole tiles; partial sums may be split along k: chunks of four k-blocks (one per
+    // staging warp) up to 16 rows, where fine chunks balance the CTAs best; longer chunks for more rows, where every
+    // chunk ends in 128 x rows reductions (measured on the 7B shape: 8 k-blocks best at 32 rows, 16 at 64 and 128)
+    d.chunk_kb = tile_mode ? d.nkb : !panel ? 4 : bn == 32 ? 8 : 16;
+    d.k_major = panel && !tile_mode;
     d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
     if (chunks > 0x7fffffffLL) return cudaErrorInvalidValue;
