@@ -24,7 +24,6 @@ struct Carver {          // hands out aligned slices of the caller's workspace (
   }
 };
 
-constexpr int kSyncWords = 12;
 
 struct Buffers {
   float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *ss_final, *part_o, *part_ml;
@@ -37,7 +36,7 @@ struct Buffers {
 };
 
 struct Dims {
-  int rmax, qd, kvd, ldq, nsplit_max, tk, pan_rows, pan_k;
+  int rmax, qd, kvd, ldq, nsplit_max, tk, pan_rows, pan_k, sync_words;
   size_t esz;
 };
 
@@ -65,6 +64,10 @@ Dims dims_of(const fc_model_shape *s) {
   d.pan_rows = d.rmax > 16 ? (d.rmax + 127) / 128 * 128 : 0;
   d.pan_k = s->d_model > s->d_ffn ? s->d_model : s->d_ffn;
   if (d.qd > d.pan_k) d.pan_k = d.qd;
+  // per-layer group of synchronisation words: grid barriers 0..2, work-claim counters 4..7, panel-ready barriers
+  // 8..11, then one completion counter per 128-column tile of the O and of the down projection
+  d.sync_words = 12 + 2 * ((s->d_model + 127) / 128);
+  d.sync_words = (d.sync_words + 3) / 4 * 4;
   return d;
 }
 
@@ -81,10 +84,9 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
   t.ss_attn = c.take<float>(R);
   t.ss_ffn = c.take<float>(R);
   t.ss_final = c.take<float>(R);
-  // kSyncWords words per layer (grid barriers 0..2, work-claim counters 4..7, panel-ready barriers 8..11) plus
-  // one group for the first QKV and the LM head; directly after the sums of squares so that one pass clears
-  // them all
-  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * kSyncWords);
+  // one group of synchronisation words per layer plus one for the first QKV and the LM head; directly after the
+  // sums of squares so that one pass clears them all
+  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * d.sync_words);
   t.pan = c.take<char>((size_t)2 * d.pan_rows * d.pan_k * 2);
   t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
   t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
@@ -348,9 +350,10 @@ enum { GEMM_QKV = -1, GEMM_O = 0, GEMM_GU = 1, GEMM_DOWN = 2, GEMM_HEAD = 3 };
 static unsigned int *claim_word(fc_ctx *ctx, int l, int which) {
   const int L = ctx->s.n_layers;
   unsigned int *w = ctx->b.chain_bar;
-  if (which == GEMM_HEAD) return w + (size_t)L * kSyncWords + 5;
-  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * kSyncWords + 4 : w + (size_t)(l - 1) * kSyncWords + 7;   // chained after down(l-1)
-  return w + (size_t)l * kSyncWords + 4 + which;
+  const size_t G = ctx->d.sync_words;
+  if (which == GEMM_HEAD) return w + (size_t)L * G + 5;
+  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * G + 4 : w + (size_t)(l - 1) * G + 7;   // chained after down(l-1)
+  return w + (size_t)l * G + 4 + which;
 }
 
 static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls,
@@ -376,7 +379,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   ea.z.p[1] = ctx->b.gu; ea.z.n[1] = Rz * 2 * s.d_ffn;
   // sums of squares (both norms) and the grid-barrier words of the chained projections are adjacent
   ea.z.p[2] = ctx->b.ss_attn;
-  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + ((size_t)s.n_layers + 1) * kSyncWords) - (char *)ctx->b.ss_attn) / sizeof(float);
+  ea.z.n[2] = (size_t)((char *)(ctx->b.chain_bar + ((size_t)s.n_layers + 1) * d.sync_words) - (char *)ctx->b.ss_attn) / sizeof(float);
   ++ctx->launches;
   { ProfScope ps(ctx, FC_CLS_EMBED); FC_CK(launch_embed(ea, s.dtype, ctx->st)); }
 
@@ -432,9 +435,9 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ++ctx->launches;
       ProfScope ps(ctx, FC_CLS_CHAIN);
       // barriers at words 0..2 of the layer's group, claim counters at 4..7 (O, gate/up, down, next QKV),
-      // panel-ready barriers at 8..11
-      unsigned int *grp = ctx->b.chain_bar + (size_t)l * kSyncWords;
-      FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + 4, grp + 8, ctx->pdl && !ctx->prof, ctx->st));
+      // panel-ready barriers at 8..11, tile completion counters from 12
+      unsigned int *grp = ctx->b.chain_bar + (size_t)l * d.sync_words;
+      FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + 4, grp + 8, grp + 12, ctx->pdl && !ctx->prof, ctx->st));
     } else {
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O)));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));

@@ -156,7 +156,10 @@ cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int 
                              cudaStream_t st);
 // Up to four projections in one launch, each consuming the previous one's reduced output; bar: n-1 zeroed words.
 // bar_b: n zeroed words (panel-ready barriers), needed when the rows exceed 16 and the plans have panels.
+// tile_done: optional zeroed words, one per 128-column output tile of projections 0 and 2 (completion counters that
+// let projections 1 and 3 start on finished tiles without a grid barrier; used up to 16 rows).
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
-                              unsigned int *claim, unsigned int *bar_b, int pdl, cudaStream_t st);
+                              unsigned int *claim, unsigned int *bar_b, unsigned int *tile_done, int pdl,
+                              cudaStream_t st);
 
 }  // namespace fc

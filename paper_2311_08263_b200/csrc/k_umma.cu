@@ -44,6 +44,14 @@ struct PhaseDesc {
   int chunk_kb, cpt, nrb, n_chunks;   // work is claimed in chunks of chunk_kb k-blocks of one tile for one block of rows:
                                       // chunks per tile, row blocks, total
   int k_major;                        // claim order: all tiles of one k range before the next k range
+  // Synchronisation with the neighbouring phases of a chained launch.  Either a grid barrier (wait_bar: this phase
+  // starts after bar[pi - 1]; sig_bar: it arrives on bar[pi]) or, between a tile-major phase and the k-major phase
+  // that consumes it, one completion counter per 128-column output tile: the producer's epilogue warps count each
+  // finished chunk on tile_done[tile]; the consumer stages k-block kb once dep_done[kb / 2] has reached dep_need.
+  int wait_bar, sig_bar;
+  unsigned int *tile_done;
+  const unsigned int *dep_done;
+  unsigned int dep_need;
 };
 
 struct MapPack {
@@ -431,7 +439,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       const int pro = P.pro;
       // the activations of this phase are the previous phase's outputs, reduced by every CTA of the grid
       // (one staging warp polls the grid-wide counter and releases the other three through shared memory)
-      if (pi > 0) {
+      if (P.wait_bar) {
         if (sw == 0) {
           ok = grid_bar_wait(p.bar + (pi - 1), gridDim.x, lane, abort_flag);
           if (ok && lane == 0) mbar_arrive(smem_u32(&go_bar[pi - 1]));
@@ -561,7 +569,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             ++seg;
           }
         }
-        if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+        if (ok && P.sig_bar) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
         continue;
       }
       {
@@ -585,6 +593,9 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             const int stage = it % S;
             const uint32_t ph = (uint32_t)(it / S) & 1u;
             if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
+            // dataflow transition: these 64 columns of the input are final once every chunk of the previous
+            // phase's tile kb / 2 has been reduced into them
+            if (P.dep_done && !grid_bar_wait(P.dep_done + (kb >> 1), P.dep_need, lane, abort_flag)) { ok = false; break; }
             unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
             const int k = kb * kTileK + chunk * 8;
             // Loads first, arithmetic and shared-memory stores after: a store between two units would keep the
@@ -678,7 +689,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
       }
       // this warp has finished reading the phase's inputs and adding its sums of squares
-      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+      if (ok && P.sig_bar) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -740,11 +751,16 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[acc]));
+          if (EPI == EPI_ATOMIC_ADD && P.tile_done) {       // this warp's share of the chunk is reduced into the tile
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(P.tile_done + s.tile, 1u);
+          }
           ++seg;
         }
       }
       // all partial sums of this phase that this warp owns are on their way to L2
-      if (ok && pi + 1 < p.n_phases) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+      if (ok && P.sig_bar) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
     }
   }
 
@@ -893,8 +909,11 @@ static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, b
 // buffers and the row count; weights, K and the matrix split stay as planned.
 // Beyond 16 rows, plans that own an activation panel run in panel mode: bar_b[i] (zero at launch) is the
 // panel-ready barrier of phase i.
+// tile_done (optional): zeroed words, one per 128-column output tile of phases 0 and 2; with them, up to 16 rows,
+// phases 1 and 3 follow their producers tile by tile instead of waiting at a grid barrier.
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
-                              unsigned int *claim, unsigned int *bar_b, int pdl, cudaStream_t st) {
+                              unsigned int *claim, unsigned int *bar_b, unsigned int *tile_done, int pdl,
+                              cudaStream_t st) {
   if (n < 1 || n > kMaxPhases || !claim) return cudaErrorInvalidValue;
   if (n > 1 && !bar) return cudaErrorInvalidValue;
   MapPack maps;
@@ -924,12 +943,30 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     // chunk ends in 128 x rows reductions (measured on the 7B shape: 8 k-blocks best at 32 rows, 16 at 64 and 128)
     d.chunk_kb = tile_mode ? d.nkb : !panel ? 4 : bn == 32 ? 8 : 16;
     d.k_major = panel && !tile_mode;
+    d.wait_bar = i > 0; d.sig_bar = i + 1 < n;
+    d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0;
     d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
     if (chunks > 0x7fffffffLL) return cudaErrorInvalidValue;
     d.n_chunks = (int)chunks;
     d.nrb = nrb;
     if (chunks > max_chunks) max_chunks = chunks;
+  }
+  if (tile_done && !panel && !tile_mode && n >= 2) {
+    // phase 0 -> 1 and phase 2 -> 3 become dataflow transitions: the producer stays tile-major (its tiles complete
+    // one after the other), the consumer goes k-major (its first chunks need only the first tiles)
+    unsigned int *td = tile_done;
+    for (int i = 0; i + 1 < n; i += 2) {
+      PhaseDesc &pr = p.ph[i], &co = p.ph[i + 1];
+      if (pr.g.n_mats != 1 || pr.g.y_off[0] != 0 || pr.g.n_rows[0] != co.g.K || pr.g.y != co.g.x) return cudaErrorInvalidValue;
+      pr.tile_done = td;
+      pr.sig_bar = 0;
+      co.wait_bar = 0;
+      co.k_major = 1;
+      co.dep_done = td;
+      co.dep_need = (unsigned int)(pr.cpt * pr.nrb * 4);      // four epilogue warps count every chunk
+      td += pr.n_tiles;
+    }
   }
   for (int i = n; i < kMaxPhases; ++i) {
     for (int m = 0; m < kMaxMats; ++m) maps.m[i * kMaxMats + m] = plans[0]->maps[0];
@@ -947,7 +984,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
 
 cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b, int pdl,
                              cudaStream_t st) {
-  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, pdl, st);
+  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, pdl, st);
 }
 
 }  // namespace fc
