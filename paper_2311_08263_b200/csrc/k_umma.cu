@@ -52,6 +52,7 @@ struct PhaseDesc {
   unsigned int *tile_done;
   const unsigned int *dep_done;
   unsigned int dep_need;
+  int dep_tiles;                      // number of counters behind dep_done
 };
 
 struct MapPack {
@@ -280,8 +281,13 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   constexpr int kXParts = x_parts(BN);
   constexpr int kXBytes = BN * 128;                 // one staged activation tile (bf16, 64 k)
   constexpr int kStageBytes = kWBytes + kXParts * kXBytes;
-  constexpr uint32_t kCols = (2 * BN < 32) ? 32u : (uint32_t)(2 * BN);
-  constexpr uint32_t kIdesc = make_idesc(BN);
+  // The high and the low activation tiles lie back to back in a stage, which is exactly a K-major tile of 2 * BN
+  // rows: one MMA of N = 2 * BN multiplies both (columns 0..BN-1 of the accumulator take the high part's products,
+  // BN..2BN-1 the low part's; the epilogue adds them).  The issuing thread is the kernel's critical path at small
+  // N - an MMA costs it a fixed ~200 cycles whatever its width - so half as many instructions matter.
+  constexpr int kAccCols = kXParts * BN;                        // TMEM columns of one accumulator
+  constexpr uint32_t kCols = (uint32_t)(2 * kAccCols);          // two accumulators: 64 .. 512, a power of two
+  constexpr uint32_t kIdesc = make_idesc(kAccCols);
 
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar, go_bar[kMaxPhases], seg_full[kSegQ], seg_empty[kSegQ];
@@ -347,6 +353,8 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     // or for the previous kernel: it streams phase after phase, limited only by free ring slots.
     if (lane == 0) {
       int it = 0, sq = 0;
+      int stage = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int pi = 0; pi < p.n_phases && ok; ++pi) {
         const PhaseDesc &P = p.ph[pi];
@@ -370,13 +378,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           tile_info(P, s.tile, m, row0, rows_valid, ycol0);
           const CUtensorMap *mp = &maps.m[pi * kMaxMats + m];
           for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
-            const int stage = it % S;
-            const uint32_t ph = (uint32_t)(it / S) & 1u;
             if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t bar = smem_u32(&full_w[stage]);
             mbar_expect_tx(bar, (uint32_t)P.tx_bytes[m]);
             tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
             issued = it + 1;
+            if (++stage == S) { stage = 0; ph ^= 1u; }
           }
           if (!ok) break;
         }
@@ -384,8 +391,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
+    // This thread is the kernel's critical path up to 16 rows (the weights are usually there before it asks):
+    // the ring position is kept incrementally and the operand descriptors are advanced by plain additions.
     if (lane == 0) {
-      int it = 0, seg = 0, sq = 0;
+      int seg = 0, sq = 0;
+      int stage = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int pi = 0; pi < p.n_phases && ok; ++pi) {
         {
@@ -397,23 +408,18 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             const int acc = seg & 1;
             if (!mbar_wait(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-            for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
-              const int stage = it % S;
-              const uint32_t ph = (uint32_t)(it / S) & 1u;
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
+            for (int kb = s.kb0; kb < s.kb1; ++kb) {
               if (!mbar_wait(smem_u32(&full_w[stage]), ph, abort_flag) ||
                   !mbar_wait(smem_u32(&full_x[stage]), ph, abort_flag)) { ok = false; break; }
               tc_fence_after();
               const uint32_t a_base = smem_base + stage * kStageBytes;
-              const uint32_t b_base = a_base + kWBytes;
+              const uint64_t a_desc = smem_desc_sw128(a_base), b_desc = smem_desc_sw128(a_base + kWBytes);
 #pragma unroll
-              for (int kk = 0; kk < kTileK / 16; ++kk) {
-#pragma unroll
-                for (int part = 0; part < kXParts; ++part)
-                  umma_bf16(d_tmem, smem_desc_sw128(a_base + kk * 32), smem_desc_sw128(b_base + part * kXBytes + kk * 32),
-                            kIdesc, (kb > s.kb0 || kk > 0 || part > 0) ? 1u : 0u);
-              }
+              for (int kk = 0; kk < kTileK / 16; ++kk)      // 32 bytes along k: the start-address field counts 16-byte units
+                umma_bf16(d_tmem, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), kIdesc, (kb > s.kb0 || kk > 0) ? 1u : 0u);
               umma_commit(smem_u32(&empty_b[stage]));
+              if (++stage == S) { stage = 0; ph ^= 1u; }
             }
             if (ok) umma_commit(smem_u32(&accum_full[acc]));
             ++seg;
@@ -437,6 +443,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       const PhaseDesc &P = p.ph[pi];
       const GemmArgs &g = P.g;
       const int pro = P.pro;
+      unsigned long long dep_mask = 0ull;      // producer tiles this warp has seen complete
       // the activations of this phase are the previous phase's outputs, reduced by every CTA of the grid
       // (one staging warp polls the grid-wide counter and releases the other three through shared memory)
       if (P.wait_bar) {
@@ -595,7 +602,34 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
             // dataflow transition: these 64 columns of the input are final once every chunk of the previous
             // phase's tile kb / 2 has been reduced into them
-            if (P.dep_done && !grid_bar_wait(P.dep_done + (kb >> 1), P.dep_need, lane, abort_flag)) { ok = false; break; }
+            if (P.dep_done) {
+              const int need_tile = kb >> 1;
+              if (P.dep_tiles > 64) {
+                if (!grid_bar_wait(P.dep_done + need_tile, P.dep_need, lane, abort_flag)) { ok = false; break; }
+              } else if (!((dep_mask >> need_tile) & 1ull)) {
+                // one look fetches every counter of the phase (lane i reads tiles i and i + 32); finished tiles are
+                // remembered, so in steady state a warp asks L2 once or twice per phase, not once per k-block
+                const unsigned long long t0 = clock64();
+                unsigned int spins = 0;
+                for (;;) {
+                  const unsigned int c0 = lane < P.dep_tiles ? ld_acquire_u32(P.dep_done + lane) : 0u;
+                  const unsigned int c1 = lane + 32 < P.dep_tiles ? ld_acquire_u32(P.dep_done + lane + 32) : 0u;
+                  dep_mask |= (unsigned long long)__ballot_sync(0xffffffffu, c0 >= P.dep_need) |
+                              ((unsigned long long)__ballot_sync(0xffffffffu, c1 >= P.dep_need) << 32);
+                  if ((dep_mask >> need_tile) & 1ull) break;
+                  if ((++spins & 0x3Fu) == 0u) {
+                    int give_up = 0;
+                    if (lane == 0) {
+                      if (*abort_flag) give_up = 1;
+                      else if ((unsigned long long)(clock64() - t0) > kSpinBudget) { *abort_flag = 1; give_up = 1; }
+                    }
+                    if (__shfl_sync(0xffffffffu, give_up, 0)) { ok = false; break; }
+                  }
+                }
+                if (!ok) break;
+                __threadfence();      // every lane's later loads come after the counters the warp has just seen
+              }
+            }
             unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
             const int k = kb * kTileK + chunk * 8;
             // Loads first, arithmetic and shared-memory stores after: a store between two units would keep the
@@ -728,7 +762,13 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
                                 : ss_part[acc][0][c0 + j] + ss_part[acc][1][c0 + j] + ss_part[acc][2][c0 + j] + ss_part[acc][3][c0 + j];
               }
             }
-            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c0), v);
+            tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kAccCols + c0), v);
+            {
+              float vl[16];
+              tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kAccCols + BN + c0), vl);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) v[j] += vl[j];
+            }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int r = rb * BN + c0 + j;
@@ -944,7 +984,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.chunk_kb = tile_mode ? d.nkb : !panel ? 4 : bn == 32 ? 8 : 16;
     d.k_major = panel && !tile_mode;
     d.wait_bar = i > 0; d.sig_bar = i + 1 < n;
-    d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0;
+    d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0; d.dep_tiles = 0;
     d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
     if (chunks > 0x7fffffffLL) return cudaErrorInvalidValue;
@@ -965,6 +1005,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
       co.k_major = 1;
       co.dep_done = td;
       co.dep_need = (unsigned int)(pr.cpt * pr.nrb * 4);      // four epilogue warps count every chunk
+      co.dep_tiles = pr.n_tiles;
       td += pr.n_tiles;
     }
   }
