@@ -602,34 +602,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             if (!mbar_wait_warp(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
             // dataflow transition: these 64 columns of the input are final once every chunk of the previous
             // phase's tile kb / 2 has been reduced into them
-            if (P.dep_done) {
-              const int need_tile = kb >> 1;
-              if (P.dep_tiles > 64) {
-                if (!grid_bar_wait(P.dep_done + need_tile, P.dep_need, lane, abort_flag)) { ok = false; break; }
-              } else if (!((dep_mask >> need_tile) & 1ull)) {
-                // one look fetches every counter of the phase (lane i reads tiles i and i + 32); finished tiles are
-                // remembered, so in steady state a warp asks L2 once or twice per phase, not once per k-block
-                const unsigned long long t0 = clock64();
-                unsigned int spins = 0;
-                for (;;) {
-                  const unsigned int c0 = lane < P.dep_tiles ? ld_acquire_u32(P.dep_done + lane) : 0u;
-                  const unsigned int c1 = lane + 32 < P.dep_tiles ? ld_acquire_u32(P.dep_done + lane + 32) : 0u;
-                  dep_mask |= (unsigned long long)__ballot_sync(0xffffffffu, c0 >= P.dep_need) |
-                              ((unsigned long long)__ballot_sync(0xffffffffu, c1 >= P.dep_need) << 32);
-                  if ((dep_mask >> need_tile) & 1ull) break;
-                  if ((++spins & 0x3Fu) == 0u) {
-                    int give_up = 0;
-                    if (lane == 0) {
-                      if (*abort_flag) give_up = 1;
-                      else if ((unsigned long long)(clock64() - t0) > kSpinBudget) { *abort_flag = 1; give_up = 1; }
-                    }
-                    if (__shfl_sync(0xffffffffu, give_up, 0)) { ok = false; break; }
-                  }
-                }
-                if (!ok) break;
-                __threadfence();      // every lane's later loads come after the counters the warp has just seen
-              }
-            }
+            if (P.dep_done && !grid_bar_wait(P.dep_done + (kb >> 1), P.dep_need, lane, abort_flag)) { ok = false; break; }
             unsigned char *xs = smem_dyn + (smem_base - smem_u32(smem_dyn)) + stage * kStageBytes + kWBytes;
             const int k = kb * kTileK + chunk * 8;
             // Loads first, arithmetic and shared-memory stores after: a store between two units would keep the
