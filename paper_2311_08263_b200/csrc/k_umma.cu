@@ -192,12 +192,18 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p) {
 // signal: each participating warp calls it once after its last global write of the phase.
 // The kWarpsSignalling warps of a CTA count up in shared memory; the last one posts the CTA's single arrival.
 constexpr unsigned int kWarpsSignalling = 8;    // 4 staging + 4 epilogue warps
+// Release increments instead of full fences: the warp barrier orders the other lanes' writes before lane 0's
+// release, the acquire-release count in shared memory chains the warps of the CTA, and the release on the global
+// counter publishes all of it to whoever acquires that counter.
+__device__ __forceinline__ void red_release_gpu(unsigned int *p, unsigned int v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void grid_bar_signal(unsigned int *ctr, unsigned int *cta_count, int lane) {
-  __threadfence();
   __syncwarp();
-  if (lane == 0 && atomicAdd(cta_count, 1u) == kWarpsSignalling - 1u) {
-    __threadfence();
-    atomicAdd(ctr, 1u);
+  if (lane == 0) {
+    unsigned int prev;
+    asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(prev) : "r"(smem_u32(cta_count)) : "memory");
+    if (prev == kWarpsSignalling - 1u) red_release_gpu(ctr, 1u);
   }
 }
 __device__ __forceinline__ bool grid_bar_wait(const unsigned int *ctr, unsigned int target, int lane,
@@ -765,9 +771,8 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[acc]));
           if (EPI == EPI_ATOMIC_ADD && P.tile_done) {       // this warp's share of the chunk is reduced into the tile
-            __threadfence();
             __syncwarp();
-            if (lane == 0) atomicAdd(P.tile_done + s.tile, 1u);
+            if (lane == 0) red_release_gpu(P.tile_done + s.tile, 1u);
           }
           ++seg;
         }
