@@ -1,18 +1,20 @@
-// Weight-streaming skinny GEMM for sm_100a:  y[R, N] (+)= pro(x)[R, K] . W[N, K]^T,  R = batch * c rows.
+// Weight-streaming skinny GEMM for sm_100a:  y[R, N] (+)= pro(x)[R, K] . W[N, K]^T,  R = batch * c rows,
+// for up to four projections of a decoder layer in one persistent launch.
 //
-// The contraction is computed "swapped": a 128-row tile of W is the M operand of tcgen05.mma, the
-// R window rows (padded to BN) are the N operand, and the fp32 accumulator [128 x BN] lives in
-// tensor memory.  W tiles (128 rows x 64 k, 16 KB) arrive by TMA into a 128B-swizzled shared-memory
-// ring; the activation operand is produced on chip: four staging warps read the fp32 activations,
-// apply the fused transform (RMSNorm gain, or SwiGLU of the gate/up accumulators), round to bf16 and
-// store them in the same swizzled K-major layout.  Work is split stream-K style: the (tile, k-block)
-// items are dealt out in equal contiguous ranges to a fixed grid, every partial accumulator is added
-// to y with fp32 reductions in L2, so no second pass is needed and HBM traffic is W exactly once.
+// The contraction is computed "swapped": a 128-row tile of W is the M operand of tcgen05.mma, a block of
+// BN rows is the N operand, and the fp32 accumulator lives in tensor memory.  W tiles (128 rows x 64 k, 16 KB)
+// arrive by TMA into a 128B-swizzled shared-memory ring.  The activation operand is a bf16 pair high + low
+// (low = bf16(x - high)) in the same swizzled K-major layout: up to 16 rows four staging warps read the fp32
+// activations, apply the fused transform (RMSNorm gain, or SwiGLU of the gate/up accumulators) and store both
+// tiles; with more rows all CTAs convert the activations once per projection into a panel in global memory and
+// one thread streams panel tiles by TMA.  Work is claimed dynamically in chunks of a few k-blocks of one tile;
+// every partial accumulator is added to y with fp32 reductions in L2, so no second pass is needed and HBM
+// traffic is W exactly once.
 //
-// Warp roles (320 threads): 0 = TMA producer, 1 = MMA issuer + TMEM owner, 2-5 = activation staging,
-// 6-9 = epilogue (TMEM -> registers -> global).  Two accumulators alternate so the epilogue of one
-// segment overlaps the MMAs of the next.  Every mbarrier wait is bounded; on expiry the CTA records
-// an error word, drains its own copies and MMAs (bounded too), frees TMEM and returns.
+// Warp roles (320 threads): 0 = chunk claims + TMA producer, 1 = MMA issuer + TMEM owner, 2-5 = activation
+// staging, 6-9 = epilogue (TMEM -> registers -> global).  Two accumulators alternate so the epilogue of one
+// segment overlaps the MMAs of the next.  Every wait is bounded; on expiry the CTA records an error word,
+// drains its own copies and MMAs (bounded too), frees TMEM and returns.
 #include <cuda.h>
 
 #include <cstdio>
@@ -28,9 +30,9 @@ constexpr int kWBytes = kTileM * kTileK * 2;
 constexpr int kThreads = 320;
 constexpr unsigned long long kSpinBudget = 400000000ull;    // clock64 ticks (~0.2 s)
 
-// Activations are staged as a bf16 pair hi + lo (lo = bf16(x - hi)): two MMAs per k-step against the same weight
-// tile, which removes the bf16 rounding of the activations.  Up to 128 rows the kernel stays memory-bound with the
-// doubled MMA work; more rows run as blocks of 128 on the same weight chunk, back to back.
+// Activations are staged as a bf16 pair hi + lo (lo = bf16(x - hi)), which removes the bf16 rounding of the
+// activations; the two tiles are multiplied by one MMA of twice the width.  More than 128 rows run as blocks of
+// 128 on the same weight chunk, back to back.
 __host__ __device__ constexpr int x_parts(int bn) { return 2; }
 
 constexpr int kMaxPhases = 4;      // projections chained in one launch (O -> gate/up -> down -> next QKV)
