@@ -147,8 +147,8 @@ const char *fc_last_cuda_error(const fc_ctx *ctx);   /* text of the last CUDA fa
 /* ---- single operations of the step, for unit parity tests (all pointers DEVICE unless noted) ---- */
 
 /* y[R, N] += x[R, K] . w[N, K]^T with fp32 x and y and weights in `dtype`; K % 8 == 0.
- * use_tensor_cores != 0 selects the tcgen05 kernel (bf16 only).  The projections of the step
- * (QKV, O, gate/up, down) are this contraction. */
+ * use_tensor_cores != 0 selects the tcgen05 kernel (bf16 only; K >= 64, N % 4 == 0 and y 16-byte aligned,
+ * else FC_ERR_SHAPE).  The projections of the step (QKV, O, gate/up, down) are this contraction. */
 int fc_op_linear(const float *x, const void *w, float *y, int32_t R, int32_t N, int32_t K,
                  int32_t dtype, int32_t use_tensor_cores, void *cuda_stream);
 

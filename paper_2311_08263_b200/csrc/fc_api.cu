@@ -764,7 +764,7 @@ extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, 
     if (launch_gemm_simt(a, dtype, PRO_NONE, EPI_ATOMIC_ADD, st) != cudaSuccess) return FC_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
   }
-  if (dtype != FC_BF16 || K < 64) return FC_ERR_SHAPE;
+  if (dtype != FC_BF16 || K < 64 || N % 4 || ((uintptr_t)y % 16)) return FC_ERR_SHAPE;   // 16-byte reductions into y
   int dev = 0, sms = 0;
   unsigned int *err_word = nullptr;
   if (cudaGetDevice(&dev) != cudaSuccess ||

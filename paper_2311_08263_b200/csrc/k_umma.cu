@@ -271,6 +271,21 @@ __device__ __forceinline__ float warp_sum_f(float v) {
   return v;
 }
 
+// Four fp32 reductions in one instruction (16-byte aligned address).
+__device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+// 4 x 4 transpose across the four lanes of a quad and four registers: afterwards lane i holds in register j what
+// lane j held in register i.
+__device__ __forceinline__ void quad_transpose(float &r0, float &r1, float &r2, float &r3, int lane) {
+  const bool b0 = lane & 1, b1 = lane & 2;
+  float t;
+  t = b0 ? r0 : r1; t = __shfl_xor_sync(0xffffffffu, t, 1); if (b0) r0 = t; else r1 = t;
+  t = b0 ? r2 : r3; t = __shfl_xor_sync(0xffffffffu, t, 1); if (b0) r2 = t; else r3 = t;
+  t = b1 ? r0 : r2; t = __shfl_xor_sync(0xffffffffu, t, 2); if (b1) r0 = t; else r2 = t;
+  t = b1 ? r1 : r3; t = __shfl_xor_sync(0xffffffffu, t, 2); if (b1) r1 = t; else r3 = t;
+}
+
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -749,6 +764,21 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
               tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kAccCols + BN + c0), vl);
 #pragma unroll
               for (int j = 0; j < 16; ++j) v[j] += vl[j];
+            }
+            if (EPI == EPI_ATOMIC_ADD) {
+              // A lane holds one output column (weight row) for 16 rows.  A reduction instruction costs the warp
+              // ~100 cycles here whatever its width, so the quads are transposed first: lane i of a quad then holds
+              // rows i, i + 4, i + 8, i + 12 for the quad's four adjacent columns - four 16-byte reductions instead
+              // of sixteen scalar ones.  (Columns come in multiples of 8, so a quad is valid or invalid as a whole.)
+              float *ybase = g.y + (ycol0 + q * 32 + (lane & ~3));
+              const bool quad_valid = (q * 32 + (lane & ~3)) < rows_valid;
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4) {
+                quad_transpose(v[4 * k4], v[4 * k4 + 1], v[4 * k4 + 2], v[4 * k4 + 3], lane);
+                const int r = rb * BN + c0 + 4 * k4 + (lane & 3);
+                if (quad_valid && r < g.R) red_add_v4(ybase + (long long)r * g.ldy, v[4 * k4], v[4 * k4 + 1], v[4 * k4 + 2], v[4 * k4 + 3]);
+              }
+              continue;
             }
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
