@@ -139,6 +139,31 @@ def test_small_bf16_logits_and_stream(flags, shape):
     _compare_stream_with_resync(cfg, w, dec, prompt, cfg.c, cfg.gen_tokens, max_seq)
 
 
+@pytest.mark.parametrize("c", [1, 2, 16])
+def test_bf16_window_sizes_one_and_sixteen(c):
+    """c = 1 is plain autoregressive decoding through the tensor-core path (one live row in the 16-row
+    accumulator); c = 16 fills it.  Four layers, so that the chained launch runs with and without a next QKV."""
+    cfg = wl.small_config(vocab=800, n_layers=4, prompt_len=140, c=c, gen_tokens=12,
+                          n_heads=4, n_kv_heads=4, head_dim=128, d_model=512, d_ffn=768)
+    w, dec, max_seq = _setup(cfg)
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    o = oracle.Oracle(cfg, w, max_seq)
+    o.prefill(prompt, c)
+    dec.fc_prefill(prompt, [len(prompt)], c)
+    logits = dec.fc_debug_logits(True)
+    for _ in range(3):
+        k, acc, wnew, lg = o.jacobi_step(want_logits=True)
+        cnt, tok, wg = dec.fc_jacobi_step()
+        assert np.abs(logits[:c].cpu().numpy() - lg).max() < LOGIT_TOL
+        srt = np.sort(lg, axis=1)
+        if (srt[:, -1] - srt[:, -2]).min() > MARGIN_TOL:
+            assert cnt[0] == k and tok[0, :k].tolist() == acc.tolist() and wg[0].tolist() == wnew.tolist()
+        else:
+            break
+    dec.fc_debug_logits(False)
+    _compare_stream_with_resync(cfg, w, dec, prompt, c, cfg.gen_tokens, max_seq)
+
+
 def test_batch_ragged_prompts_independent_accepts():
     cfg = wl.small_config(vocab=600, n_layers=2, n_heads=4, n_kv_heads=2, head_dim=64, d_model=256, d_ffn=512,
                           prompt_len=70, c=6, gen_tokens=20)
