@@ -25,6 +25,8 @@ struct Carver {          // hands out aligned slices of the caller's workspace (
 };
 
 
+constexpr int kSyncClaim = kChainMax, kSyncPanel = 2 * kChainMax, kSyncTd = 3 * kChainMax;   // offsets in a group
+
 struct Buffers {
   float *x, *qkv, *attn, *gu, *ss_attn, *ss_ffn, *ss_final, *part_o, *part_ml;
   void *pan;
@@ -64,9 +66,9 @@ Dims dims_of(const fc_model_shape *s) {
   d.pan_rows = d.rmax > 16 ? (d.rmax + 127) / 128 * 128 : 0;
   d.pan_k = s->d_model > s->d_ffn ? s->d_model : s->d_ffn;
   if (d.qd > d.pan_k) d.pan_k = d.qd;
-  // per-layer group of synchronisation words: grid barriers 0..2, work-claim counters 4..7, panel-ready barriers
-  // 8..11, then one completion counter per 128-column tile of the O and of the down projection
-  d.sync_words = 12 + 2 * ((s->d_model + 127) / 128);
+  // per-layer group of synchronisation words: grid barriers 0..5, work-claim counters 6..11, panel-ready barriers
+  // 12..17, then one completion counter per 128-column tile of the O and of the down projection
+  d.sync_words = kSyncTd + 2 * ((s->d_model + 127) / 128);
   d.sync_words = (d.sync_words + 3) / 4 * 4;
   return d;
 }
@@ -127,6 +129,8 @@ struct fc_ctx {
   bool fused_attn;   // bf16 with head_dim 64/128: rotary embedding and K/V write happen inside the attention kernel
   int n_sms;
   std::vector<UmmaPlan *> plan_qkv, plan_o, plan_gu, plan_down;
+  std::vector<UmmaPlan *> plan_gu_half[2], plan_down_half[2];   // the FFN in two halves of d_ffn (chained launch, <= 16 rows)
+  bool ffn_split = false;
   UmmaPlan *plan_head = nullptr;
   float *dbg_logits = nullptr;
   // sequence state mirrored on the host
@@ -184,7 +188,8 @@ extern "C" const char *fc_last_cuda_error(const fc_ctx *ctx) { return ctx ? ctx-
 extern "C" int64_t fc_last_launch_count(const fc_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 static void destroy_plans(fc_ctx *ctx) {
-  for (auto *v : {&ctx->plan_qkv, &ctx->plan_o, &ctx->plan_gu, &ctx->plan_down}) {
+  for (auto *v : {&ctx->plan_qkv, &ctx->plan_o, &ctx->plan_gu, &ctx->plan_down, &ctx->plan_gu_half[0], &ctx->plan_gu_half[1],
+                  &ctx->plan_down_half[0], &ctx->plan_down_half[1]}) {
     for (UmmaPlan *p : *v) umma_plan_destroy(p);
     v->clear();
   }
@@ -238,6 +243,28 @@ static GemmArgs args_down(const fc_ctx *c, int l) {
   a.w[0] = c->w_down[l]; a.n_rows[0] = c->s.d_model; a.n_mats = 1;
   a.y = c->b.x; a.ldy = c->s.d_model; a.K = c->s.d_ffn;
   a.pan = c->d.pan_rows ? c->b.pan : nullptr; a.pan_rows = c->d.pan_rows;
+  return a;
+}
+// Half h of the feed-forward block: gate/up rows (= down columns) h * F/2 .. (h + 1) * F/2.  The two down halves are
+// partial sums of the same output; only the first gate/up half accumulates the row sums of squares.
+static GemmArgs args_gu_half(const fc_ctx *c, int l, int h) {
+  GemmArgs a = args_gu(c, l);
+  const int F2 = c->s.d_ffn / 2;
+  const size_t off = (size_t)h * F2 * c->s.d_model * c->d.esz;
+  a.w[0] = (const char *)c->w_gate[l] + off; a.w[1] = (const char *)c->w_up[l] + off;
+  a.n_rows[0] = a.n_rows[1] = F2;
+  a.y_off[0] = h * F2; a.y_off[1] = c->s.d_ffn + h * F2;
+  if (h) a.ss_out = nullptr;
+  a.pan = nullptr; a.pan_rows = 0;
+  return a;
+}
+static GemmArgs args_down_half(const fc_ctx *c, int l, int h) {
+  GemmArgs a = args_down(c, l);
+  const int F2 = c->s.d_ffn / 2;
+  a.x = c->b.gu + (size_t)h * F2; a.x2 = c->b.gu + c->s.d_ffn + (size_t)h * F2;
+  a.w[0] = (const char *)c->w_down[l] + (size_t)h * F2 * c->d.esz; a.ldw = c->s.d_ffn;
+  a.K = F2;
+  a.pan = nullptr; a.pan_rows = 0;
   return a;
 }
 static GemmArgs args_head(const fc_ctx *c) {
@@ -294,12 +321,18 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
     if (prop.major != 10) return fail(FC_ERR_SHAPE);
     if (shape->d_model < 64 || shape->d_ffn < 64 || ctx->d.qd < 64) return fail(FC_ERR_SHAPE);
     char msg[200];
+    // halves of d_ffn must be whole 128-row tiles (and so whole 64-wide k-blocks of the down projection)
+    ctx->ffn_split = ctx->chain && shape->d_ffn % 256 == 0 && !(shape->flags & FC_FLAG_NO_FFN_SPLIT);
     for (int l = 0; l < L && rc == FC_OK; ++l) {
       UmmaPlan *p;
       if (!(p = umma_plan_create(args_qkv(ctx, l), PRO_GAIN, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_qkv.push_back(p);
       if (rc == FC_OK) { if (!(p = umma_plan_create(args_o(ctx, l), PRO_NONE, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_o.push_back(p); }
       if (rc == FC_OK) { if (!(p = umma_plan_create(args_gu(ctx, l), PRO_GAIN, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_gu.push_back(p); }
       if (rc == FC_OK) { if (!(p = umma_plan_create(args_down(ctx, l), PRO_SILU_MUL, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_down.push_back(p); }
+      for (int h = 0; h < 2 && rc == FC_OK && ctx->ffn_split; ++h) {
+        if (!(p = umma_plan_create(args_gu_half(ctx, l, h), PRO_GAIN, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_gu_half[h].push_back(p);
+        if (rc == FC_OK) { if (!(p = umma_plan_create(args_down_half(ctx, l, h), PRO_SILU_MUL, EPI_ATOMIC_ADD, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA; else ctx->plan_down_half[h].push_back(p); }
+      }
     }
     if (rc == FC_OK && !(ctx->plan_head = umma_plan_create(args_head(ctx), PRO_GAIN, EPI_ARGMAX, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA;
     if (rc != FC_OK) { fprintf(stderr, "fc_init: %s\n", msg); return fail(rc); }
@@ -351,9 +384,9 @@ static unsigned int *claim_word(fc_ctx *ctx, int l, int which) {
   const int L = ctx->s.n_layers;
   unsigned int *w = ctx->b.chain_bar;
   const size_t G = ctx->d.sync_words;
-  if (which == GEMM_HEAD) return w + (size_t)L * G + 5;
-  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * G + 4 : w + (size_t)(l - 1) * G + 7;   // chained after down(l-1)
-  return w + (size_t)l * G + 4 + which;
+  if (which == GEMM_HEAD) return w + (size_t)L * G + kSyncClaim + 1;
+  if (which == GEMM_QKV) return l == 0 ? w + (size_t)L * G + kSyncClaim : w + (size_t)(l - 1) * G + kSyncClaim + 3;
+  return w + (size_t)l * G + kSyncClaim + which;
 }
 
 static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls,
@@ -361,7 +394,7 @@ static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R
   ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
-  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + 4, ctx->pdl && !ctx->prof, ctx->st);   // panel-ready word: four after the claim word
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + (kSyncPanel - kSyncClaim), ctx->pdl && !ctx->prof, ctx->st);   // panel-ready word
   return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
 }
 
@@ -426,18 +459,33 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st)); }
     }
     if (chained) {
-      // O projection, gate/up, down and the next layer's QKV: one persistent launch, three grid barriers
-      const UmmaPlan *plans[4] = {ctx->plan_o[l], ctx->plan_gu[l], ctx->plan_down[l], nullptr};
-      GemmArgs ga[4] = {args_o(ctx, l), args_gu(ctx, l), args_down(ctx, l), GemmArgs()};
-      int n = 3;
-      if (l + 1 < s.n_layers) { plans[3] = ctx->plan_qkv[l + 1]; ga[3] = args_qkv(ctx, l + 1); n = 4; }
+      // O projection, gate/up, down and the next layer's QKV: one persistent launch.
+      // Up to 16 rows the phases are tied together without a stall where the data allow it (see ChainSync): gate/up
+      // (claimed k range by k range) follows the O projection's finished tiles; the feed-forward block runs in two
+      // halves of d_ffn, so that a down half waits only for a gate/up half that finished a whole phase earlier; the
+      // next layer's QKV follows the finished tiles of the two down halves' sum.
+      const UmmaPlan *plans[kChainMax];
+      GemmArgs ga[kChainMax];
+      ChainSync sy[kChainMax];
+      int n = 0;
+      const bool split = ctx->ffn_split && R <= 16;
+      plans[n] = ctx->plan_o[l]; ga[n] = args_o(ctx, l); sy[n++] = ChainSync{-1, -1, 0, -1};
+      if (split) {
+        plans[n] = ctx->plan_gu_half[0][l]; ga[n] = args_gu_half(ctx, l, 0); sy[n++] = ChainSync{-1, 0, -1, 0};
+        plans[n] = ctx->plan_gu_half[1][l]; ga[n] = args_gu_half(ctx, l, 1); sy[n++] = ChainSync{-1, 1, -1, 0};
+        plans[n] = ctx->plan_down_half[0][l]; ga[n] = args_down_half(ctx, l, 0); sy[n++] = ChainSync{0, -1, 1, -1};
+        plans[n] = ctx->plan_down_half[1][l]; ga[n] = args_down_half(ctx, l, 1); sy[n++] = ChainSync{1, -1, 1, -1};
+      } else {
+        plans[n] = ctx->plan_gu[l]; ga[n] = args_gu(ctx, l); sy[n++] = ChainSync{-1, 0, -1, 0};
+        plans[n] = ctx->plan_down[l]; ga[n] = args_down(ctx, l); sy[n++] = ChainSync{0, -1, 1, -1};
+      }
+      if (l + 1 < s.n_layers) { plans[n] = ctx->plan_qkv[l + 1]; ga[n] = args_qkv(ctx, l + 1); sy[n++] = ChainSync{-1, -1, -1, 1}; }
       for (int i = 0; i < n; ++i) ga[i].R = R;
       ++ctx->launches;
       ProfScope ps(ctx, FC_CLS_CHAIN);
-      // barriers at words 0..2 of the layer's group, claim counters at 4..7 (O, gate/up, down, next QKV),
-      // panel-ready barriers at 8..11, tile completion counters from 12
       unsigned int *grp = ctx->b.chain_bar + (size_t)l * d.sync_words;
-      FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + 4, grp + 8, grp + 12, ctx->pdl && !ctx->prof, ctx->st));
+      FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + kSyncClaim, grp + kSyncPanel, R <= 16 ? sy : nullptr, grp + kSyncTd,
+                              (s.d_model + 127) / 128, ctx->pdl && !ctx->prof, ctx->st));
     } else {
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O)));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));

@@ -33,6 +33,7 @@ struct GemmArgs {
   int dn;                 // width the sums of squares are means over (d_model)
   // weights: up to three matrices [n_rows[m], K], outputs concatenated at column offsets y_off[m]
   const void *w[kMaxMats];
+  int ldw;                // row pitch of the weight matrices in elements (0: K) - a column slice of a wider matrix
   int n_rows[kMaxMats];
   int y_off[kMaxMats];
   int n_mats;
@@ -156,10 +157,16 @@ cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int 
                              cudaStream_t st);
 // Up to four projections in one launch, each consuming the previous one's reduced output; bar: n-1 zeroed words.
 // bar_b: n zeroed words (panel-ready barriers), needed when the rows exceed 16 and the plans have panels.
-// tile_done: optional zeroed words, one per 128-column output tile of projections 0 and 2 (completion counters that
-// let projections 1 and 3 start on finished tiles without a grid barrier; used up to 16 rows).
+// sync (optional, used up to 16 rows): how each projection is tied to the others, instead of a grid barrier
+// after every one.  wait_bar / sig_bar: index of the grid barrier (word of `bar`) the projection waits on before
+// its first activation load / arrives on when done, -1 for none.  td_prod: the projection is claimed tile by tile
+// and counts finished chunks per 128-column output tile in counter set td_prod (several projections may feed one
+// set: partial sums of the same output); td_cons: it is claimed k range by k range and stages a k-block once the
+// tile of set td_cons it reads is complete.  tile_done: zeroed words, td_stride per counter set.
+struct ChainSync { int wait_bar, sig_bar, td_prod, td_cons; };
+constexpr int kChainMax = 6;     // projections in one chained launch
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
-                              unsigned int *claim, unsigned int *bar_b, unsigned int *tile_done, int pdl,
-                              cudaStream_t st);
+                              unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,
+                              int td_stride, int pdl, cudaStream_t st);
 
 }  // namespace fc

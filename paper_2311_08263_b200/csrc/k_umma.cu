@@ -35,7 +35,7 @@ constexpr unsigned long long kSpinBudget = 400000000ull;    // clock64 ticks (~0
 // 128 on the same weight chunk, back to back.
 __host__ __device__ constexpr int x_parts(int bn) { return 2; }
 
-constexpr int kMaxPhases = 4;      // projections chained in one launch (O -> gate/up -> down -> next QKV)
+constexpr int kMaxPhases = kChainMax;   // projections chained in one launch (O -> gate/up halves -> down halves -> next QKV)
 
 struct PhaseDesc {
   GemmArgs g;
@@ -46,10 +46,11 @@ struct PhaseDesc {
   int chunk_kb, cpt, nrb, n_chunks;   // work is claimed in chunks of chunk_kb k-blocks of one tile for one block of rows:
                                       // chunks per tile, row blocks, total
   int k_major;                        // claim order: all tiles of one k range before the next k range
-  // Synchronisation with the neighbouring phases of a chained launch.  Either a grid barrier (wait_bar: this phase
-  // starts after bar[pi - 1]; sig_bar: it arrives on bar[pi]) or, between a tile-major phase and the k-major phase
-  // that consumes it, one completion counter per 128-column output tile: the producer's epilogue warps count each
-  // finished chunk on tile_done[tile]; the consumer stages k-block kb once dep_done[kb / 2] has reached dep_need.
+  // Synchronisation with the other phases of a chained launch.  Either a grid barrier (wait_bar: index of the
+  // barrier this phase waits on before its first activation load; sig_bar: index of the one it arrives on; -1: none)
+  // or, between tile-major phases and the k-major phase that consumes their sum, one completion counter per
+  // 128-column output tile: the producers' epilogue warps count each finished chunk on tile_done[tile]; the consumer
+  // stages k-block kb once dep_done[kb / 2] has reached dep_need.
   int wait_bar, sig_bar;
   unsigned int *tile_done;
   const unsigned int *dep_done;
@@ -466,15 +467,14 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       const PhaseDesc &P = p.ph[pi];
       const GemmArgs &g = P.g;
       const int pro = P.pro;
-      unsigned long long dep_mask = 0ull;      // producer tiles this warp has seen complete
       // the activations of this phase are the previous phase's outputs, reduced by every CTA of the grid
       // (one staging warp polls the grid-wide counter and releases the other three through shared memory)
-      if (P.wait_bar) {
+      if (P.wait_bar >= 0) {
         if (sw == 0) {
-          ok = grid_bar_wait(p.bar + (pi - 1), gridDim.x, lane, abort_flag);
-          if (ok && lane == 0) mbar_arrive(smem_u32(&go_bar[pi - 1]));
+          ok = grid_bar_wait(p.bar + P.wait_bar, gridDim.x, lane, abort_flag);
+          if (ok && lane == 0) mbar_arrive(smem_u32(&go_bar[pi]));
         } else {
-          ok = mbar_wait_warp(smem_u32(&go_bar[pi - 1]), 0u, abort_flag);
+          ok = mbar_wait_warp(smem_u32(&go_bar[pi]), 0u, abort_flag);
         }
         if (!ok) break;
       }
@@ -599,7 +599,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
             ++seg;
           }
         }
-        if (ok && P.sig_bar) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+        if (ok && P.sig_bar >= 0) grid_bar_signal(p.bar + P.sig_bar, &bar_cnt_s[P.sig_bar], lane);
         continue;
       }
       {
@@ -719,7 +719,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
       }
       // this warp has finished reading the phase's inputs and adding its sums of squares
-      if (ok && P.sig_bar) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+      if (ok && P.sig_bar >= 0) grid_bar_signal(p.bar + P.sig_bar, &bar_cnt_s[P.sig_bar], lane);
     }
   } else {
     // ------------------------------------------------------------ epilogue
@@ -778,15 +778,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
                 const int r = rb * BN + c0 + 4 * k4 + (lane & 3);
                 if (quad_valid && r < g.R) red_add_v4(ybase + (long long)r * g.ldy, v[4 * k4], v[4 * k4 + 1], v[4 * k4 + 2], v[4 * k4 + 3]);
               }
-              continue;
-            }
+            } else {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const int r = rb * BN + c0 + j;
               if (r >= g.R) break;
-              if (EPI == EPI_ATOMIC_ADD) {
-                if (valid) atomicAdd(&g.y[(long long)r * g.ldy + col], v[j]);
-              } else {
+              {
                 float logit = v[j] * rsqrtf(ssum[j] / (float)g.dn + g.eps);
                 unsigned long long key = 0ull;
                 if (valid) {
@@ -797,6 +794,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
                 key = warp_max_u64(key);
                 if (lane == 0) atomicMax(&g.amax[r], key);
               }
+            }
             }
           }
           tc_fence_before();
@@ -810,7 +808,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         }
       }
       // all partial sums of this phase that this warp owns are on their way to L2
-      if (ok && P.sig_bar) grid_bar_signal(p.bar + pi, &bar_cnt_s[pi], lane);
+      if (ok && P.sig_bar >= 0) grid_bar_signal(p.bar + P.sig_bar, &bar_cnt_s[P.sig_bar], lane);
     }
   }
 
@@ -887,7 +885,7 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
     const cuuint32_t box_rows = (cuuint32_t)(a.n_rows[m] < kTileM ? a.n_rows[m] : kTileM);
     pl->d.tx_bytes[m] = (int)(box_rows * kTileK * 2);
     cuuint64_t gdim[2] = {(cuuint64_t)a.K, (cuuint64_t)a.n_rows[m]};
-    cuuint64_t gstr[1] = {(cuuint64_t)a.K * 2};
+    cuuint64_t gstr[1] = {(cuuint64_t)(a.ldw ? a.ldw : a.K) * 2};
     cuuint32_t box[2] = {(cuuint32_t)kTileK, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = enc(&pl->maps[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(a.w[m]), gdim, gstr, box,
@@ -958,12 +956,11 @@ static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, b
 // into its output, separated by a grid barrier on bar[i] (zero at launch).  args[i] carries the per-launch
 // buffers and the row count; weights, K and the matrix split stay as planned.
 // Beyond 16 rows, plans that own an activation panel run in panel mode: bar_b[i] (zero at launch) is the
-// panel-ready barrier of phase i.
-// tile_done (optional): zeroed words, one per 128-column output tile of phases 0 and 2; with them, up to 16 rows,
-// phases 1 and 3 follow their producers tile by tile instead of waiting at a grid barrier.
+// panel-ready barrier of phase i.  Without `sync` (and always in panel mode) every phase waits at a grid barrier
+// for the one before it.
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
-                              unsigned int *claim, unsigned int *bar_b, unsigned int *tile_done, int pdl,
-                              cudaStream_t st) {
+                              unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,
+                              int td_stride, int pdl, cudaStream_t st) {
   if (n < 1 || n > kMaxPhases || !claim) return cudaErrorInvalidValue;
   if (n > 1 && !bar) return cudaErrorInvalidValue;
   MapPack maps;
@@ -977,6 +974,8 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
   bool panel = bar_b != nullptr && args[0].R > 16;
   for (int i = 0; i < n; ++i) panel = panel && plans[i]->has_xmap && args[0].R <= plans[i]->d.g.pan_rows;
   if (panel && epi == EPI_ARGMAX && !args[0].ss_out) return cudaErrorInvalidValue;
+  if (args[0].R > 16 && !panel && n > 1 && sync) return cudaErrorInvalidValue;   // the caller plans `sync` for <= 16 rows
+  const bool explicit_sync = sync && tile_done && !panel && !tile_mode && args[0].R <= 16;
   long long max_chunks = 1;
   for (int i = 0; i < n; ++i) {
     const UmmaPlan *pl = plans[i];
@@ -993,7 +992,8 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     // chunk ends in 128 x rows reductions (measured on the 7B shape: 8 k-blocks best at 32 rows, 16 at 64 and 128)
     d.chunk_kb = tile_mode ? d.nkb : !panel ? 4 : bn == 32 ? 8 : 16;
     d.k_major = panel && !tile_mode;
-    d.wait_bar = i > 0; d.sig_bar = i + 1 < n;
+    d.wait_bar = i > 0 ? i - 1 : -1;
+    d.sig_bar = i + 1 < n ? i : -1;
     d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0; d.dep_tiles = 0;
     d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
@@ -1002,21 +1002,31 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.nrb = nrb;
     if (chunks > max_chunks) max_chunks = chunks;
   }
-  if (tile_done && !panel && !tile_mode && n >= 2) {
-    // phase 0 -> 1 and phase 2 -> 3 become dataflow transitions: the producer stays tile-major (its tiles complete
-    // one after the other), the consumer goes k-major (its first chunks need only the first tiles)
-    unsigned int *td = tile_done;
-    for (int i = 0; i + 1 < n; i += 2) {
-      PhaseDesc &pr = p.ph[i], &co = p.ph[i + 1];
-      if (pr.g.n_mats != 1 || pr.g.y_off[0] != 0 || pr.g.n_rows[0] != co.g.K || pr.g.y != co.g.x) return cudaErrorInvalidValue;
-      pr.tile_done = td;
-      pr.sig_bar = 0;
-      co.wait_bar = 0;
-      co.k_major = 1;
-      co.dep_done = td;
-      co.dep_need = (unsigned int)(pr.cpt * pr.nrb * 4);      // four epilogue warps count every chunk
-      co.dep_tiles = pr.n_tiles;
-      td += pr.n_tiles;
+  if (explicit_sync) {
+    for (int i = 0; i < n; ++i) {
+      PhaseDesc &d = p.ph[i];
+      const ChainSync &c = sync[i];
+      if (c.wait_bar >= n || c.sig_bar >= n || c.td_prod > 1 || c.td_cons > 1) return cudaErrorInvalidValue;
+      d.wait_bar = c.wait_bar; d.sig_bar = c.sig_bar;
+      if (c.td_prod >= 0) {          // tile-major producer: its tiles complete one after the other
+        if (d.g.n_mats != 1 || d.g.y_off[0] != 0 || d.n_tiles > td_stride) return cudaErrorInvalidValue;
+        d.tile_done = tile_done + (size_t)c.td_prod * td_stride;
+      }
+      if (c.td_cons >= 0) {          // k-major consumer: its first chunks need only the first tiles
+        unsigned int need = 0;
+        int tiles = 0;
+        for (int j = 0; j < i; ++j)
+          if (sync[j].td_prod == c.td_cons) {
+            if (p.ph[j].g.n_rows[0] != d.g.K || p.ph[j].g.y != d.g.x) return cudaErrorInvalidValue;
+            need += (unsigned int)(p.ph[j].cpt * p.ph[j].nrb * 4);     // four epilogue warps count every chunk
+            tiles = p.ph[j].n_tiles;
+          }
+        if (!need) return cudaErrorInvalidValue;
+        d.k_major = 1;
+        d.dep_done = tile_done + (size_t)c.td_cons * td_stride;
+        d.dep_need = need;
+        d.dep_tiles = tiles;
+      }
     }
   }
   for (int i = n; i < kMaxPhases; ++i) {
@@ -1035,7 +1045,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
 
 cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b, int pdl,
                              cudaStream_t st) {
-  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, pdl, st);
+  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, nullptr, 0, pdl, st);
 }
 
 }  // namespace fc

@@ -111,8 +111,9 @@ def _compare_stream_with_resync(cfg, w, dec, prompt, c, n_tokens, max_seq):
     return tolerated
 
 
-@pytest.mark.parametrize("flags", [lib.FC_FLAG_SIMT_GEMM, 0, lib.FC_FLAG_NO_PDL | lib.FC_FLAG_NO_CHAIN],
-                         ids=["fma", "tensor", "tensor-unchained"])
+@pytest.mark.parametrize("flags", [lib.FC_FLAG_SIMT_GEMM, 0, lib.FC_FLAG_NO_PDL | lib.FC_FLAG_NO_CHAIN,
+                                   lib.FC_FLAG_NO_FFN_SPLIT],
+                         ids=["fma", "tensor", "tensor-unchained", "tensor-ffn-unsplit"])
 @pytest.mark.parametrize("shape", ["gqa64", "mha128", "gqa32"])
 def test_small_bf16_logits_and_stream(flags, shape):
     kw = {"gqa64": dict(n_heads=4, n_kv_heads=2, head_dim=64, d_model=256, d_ffn=512),
