@@ -98,7 +98,9 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   long long stride_b, stride_h;
   const int32_t *kv_len;
   int b0, nb, c, hq, hkv;
-  int nsplit;             // 128-key chunks covering max(kv_len) + c
+  int nsplit;             // CTAs per (sequence, kv head); nsplit * cpc 128-key chunks cover max(kv_len) + c
+  int cpc;                // consecutive chunks per CTA
+  int qsplit;             // 1, or the number of 16-row query tiles per kv head: then every tile has CTAs of its own (needed for cpc > 1)
   float *part_o, *part_ml;
   unsigned int *counters; // [batch*hkv], zero on entry and on exit
   unsigned int *grid_counter;   // one word, zero on entry and on exit

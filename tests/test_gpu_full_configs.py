@@ -128,3 +128,15 @@ def test_13b_batch8_ragged_step():
     _need(45, 40)
     lens = [1024, 700, 1000, 513, 1024, 64, 900, 1]
     _random_kv_case(cfg, lens, cfg.c, [1, 5, 7])
+
+
+@pytest.mark.parametrize("hd,heads,kv_heads", [(64, 8, 8), (128, 4, 4), (64, 8, 2)])
+def test_long_ragged_caches_several_chunks_per_cta(hd, heads, kv_heads):
+    """Long caches in a batch: more 128-key chunks than the GPU holds CTAs, so one CTA walks over several
+    consecutive chunks with running softmax statistics (ragged lengths: CTAs with fewer live chunks, with
+    none, and with the window's own keys in their last chunk; with grouped queries there are two 16-row query
+    tiles per kv head, each with CTAs of its own)."""
+    cfg = wl.small_config(vocab=500, n_layers=2, n_heads=heads, n_kv_heads=kv_heads, head_dim=hd, d_model=512,
+                          d_ffn=512, c=8, prompt_len=64, gen_tokens=8)
+    lens = [6000, 4100, 129, 5000, 1, 3333, 6000, 2047, 640, 5990]
+    _random_kv_case(cfg, lens, cfg.c, [0, 1, 2, 4, 7, 9])
