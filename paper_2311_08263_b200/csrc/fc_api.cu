@@ -431,14 +431,14 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       fa.rope = ctx->b.rope; fa.c_magic = (unsigned int)((0x100000000ull + (unsigned)rows - 1) / (unsigned)rows);
       fa.kcache = kc; fa.vcache = vc; fa.stride_b = stride_b; fa.stride_h = stride_h;
       fa.kv_len = ctx->b.kv_len; fa.b0 = b0; fa.nb = nb; fa.c = rows; fa.hq = s.n_heads; fa.hkv = s.n_kv_heads;
-      // One CTA per 128-key chunk while that fills the GPU at most a few times over; beyond, a CTA walks over
+      // One CTA per 128-key chunk while all of them are resident at once (two per SM); beyond, a CTA walks over
       // several consecutive chunks, so that the queries are staged and the partial result is written once per CTA
       // (every 16-row query tile then has CTAs of its own).
       int cpc = 1, qsplit = 1;
       {
         const int nqt = ((s.n_heads / s.n_kv_heads) * rows + 15) / 16;
         const long long per_split = (long long)s.n_kv_heads * nb;
-        if ((long long)nsplit * per_split > 4ll * ctx->n_sms) {
+        if ((long long)nsplit * per_split > 2ll * ctx->n_sms) {       // more CTAs than are resident at once
           long long groups = (2ll * ctx->n_sms + per_split * nqt - 1) / (per_split * nqt);   // ~2 CTAs per SM in all
           if (groups < 1) groups = 1;
           cpc = (int)((nsplit + groups - 1) / groups);
