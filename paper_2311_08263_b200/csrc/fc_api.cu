@@ -439,7 +439,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
         const int nqt = ((s.n_heads / s.n_kv_heads) * rows + 15) / 16;
         const long long per_split = (long long)s.n_kv_heads * nb;
         if ((long long)nsplit * per_split > 2ll * ctx->n_sms) {       // more CTAs than are resident at once
-          long long groups = (2ll * ctx->n_sms + per_split * nqt - 1) / (per_split * nqt);   // ~2 CTAs per SM in all
+          long long groups = 2ll * ctx->n_sms / (per_split * nqt);      // as many CTAs as are resident at once, not more
           if (groups < 1) groups = 1;
           cpc = (int)((nsplit + groups - 1) / groups);
           if (cpc > 1) qsplit = nqt;
