@@ -187,7 +187,8 @@ def test_batch_ragged_prompts_independent_accepts():
     assert st.tokens == B * cfg.gen_tokens
 
 
-@pytest.mark.parametrize("B,c", [(3, 8), (4, 12), (6, 16), (10, 16)], ids=["rows24", "rows48", "rows96", "rows160"])
+@pytest.mark.parametrize("B,c", [(3, 8), (4, 12), (6, 16), (10, 16), (1, 64), (3, 33)],
+                         ids=["rows24", "rows48", "rows96", "rows160", "c64", "c33x3"])
 @pytest.mark.parametrize("shape", ["gqa64", "gqa32"])
 def test_many_rows_prefill_and_steps(B, c, shape):
     """More than 16 rows per forward: the projections read their activations from the converted panel, for
