@@ -4,17 +4,20 @@
  * One step = one causal decoder forward over (committed prefix held in a K/V cache) + (a window
  * of c tokens: the pending exact token followed by c-1 approximate tokens), greedy argmax at
  * every window row, verification of the previous guesses one by one, K/V commit of the accepted
- * rows and shift + refill of the window (paper Section 3.3: Eq. 4 inference, Eq. 5 verification,
- * "Cache Update"; buffer and index vector: Section 3.2).  With c = 1 the step is plain greedy
- * autoregressive decoding (Eq. 1).
+ * rows and shift + refill of the window (paper, Method, "Approximate Rationale Generation": Eq. 4
+ * inference, Eq. 5 verification, "Cache Update"; buffer and index vector: "Approximate Tokens
+ * Buffer").  With c = 1 the step is plain greedy autoregressive decoding (Eq. 1).
  *
  * Conventions
  *   - "host"/"device" on every pointer says where the memory lives.  The library allocates NO
  *     device memory: weights, K/V slab and workspace are caller-owned device buffers, BORROWED for
  *     the lifetime of the context.  fc_destroy frees host state only.
  *   - All matrices are row-major [out_features, in_features] in the model dtype.
- *   - Every call returns FC_OK (0) or a negative fc_status; nothing aborts or throws, no device
- *     trap is used, and a failed call leaves the committed state (tokens, kv_len) unchanged.
+ *   - Every call returns FC_OK (0) or a negative fc_status; nothing aborts or throws and no device
+ *     trap is used.  A call refused for its arguments (FC_ERR_ARG, _CAPACITY, _TOKEN_RANGE, _BAD_WINDOW,
+ *     _STATE) leaves the committed state (tokens, kv_len) unchanged, with one exception: fc_prefill
+ *     drops the previous sequences as soon as its arguments are accepted.  After FC_ERR_DEVICE_TIMEOUT
+ *     or FC_ERR_CUDA from a call that launched kernels, the sequences are lost: call fc_prefill again.
  *   - Calls are synchronous with respect to their host outputs: they wait on the context's stream.
  *   - A context is bound to one device and one stream and is not re-entrant.
  */
@@ -32,8 +35,8 @@ typedef struct fc_ctx fc_ctx;
 
 typedef enum { FC_F32 = 0, FC_BF16 = 1 } fc_dtype;
 
-/* How window slots that no forward has predicted yet are filled (Section 3.2: the buffer is
- * initialised from the prompt's own token ids; a pad token is the alternative it mentions). */
+/* How window slots that no forward has predicted yet are filled ("Approximate Tokens Buffer": the
+ * buffer is initialised from the prompt's own token ids; a pad token is the alternative it mentions). */
 typedef enum { FC_REFILL_PROMPT_CYCLE = 0, FC_REFILL_PAD = 1 } fc_refill;
 
 typedef enum {
@@ -50,7 +53,6 @@ typedef enum {
 
 enum {                        /* fc_model_shape.flags */
   FC_FLAG_SIMT_GEMM = 1,      /* run projections on the plain FMA kernels even for bf16 (debug aid) */
-  FC_FLAG_NO_GRAPH = 2,       /* never capture the step into a CUDA graph */
   FC_FLAG_NO_PDL = 4,         /* launch every kernel fully serialised (no programmatic dependent launch) */
   FC_FLAG_NO_CHAIN = 8,       /* one launch per projection instead of one chained launch per layer */
   FC_FLAG_NO_FFN_SPLIT = 16   /* chained launch: gate/up and down as one phase each instead of two halves of d_ffn */
@@ -78,7 +80,7 @@ typedef struct {              /* DEVICE pointers, borrowed */
 typedef struct {              /* filled by fc_generate */
   int64_t steps, tokens;      /* forwards run; tokens committed over all sequences */
   int32_t accept_hist[65];    /* accept_hist[k] = (sequence, step) pairs that accepted k tokens; k>64 -> [64] */
-  float ms_prefill, ms_steps; /* device time; ms_prefill is 0 unless prefill ran inside the call */
+  float ms_prefill, ms_steps; /* device time of the most recent fc_prefill and of this call's iterations */
 } fc_stats;
 
 /* Bytes the caller must provide.  K/V slab layout: [layer][K|V][max_batch][n_kv_heads][max_seq][head_dim]
@@ -86,16 +88,19 @@ typedef struct {              /* filled by fc_generate */
 size_t fc_kv_bytes(const fc_model_shape *shape);
 size_t fc_workspace_bytes(const fc_model_shape *shape);
 
-/* Create a context.  shape, weights: host structs (copied).  kv, ws: device, >= the sizes above,
+/* Create a context: the decode state of "Approximate Tokens Buffer" (buffer Y as window + committed tokens,
+ * index vector I as kv_len per sequence) and the K/V cache of the exact prefix, all empty.
+ * shape, weights: host structs (copied).  kv, ws: device, >= the sizes above,
  * 256-byte aligned.  cuda_stream: a cudaStream_t (NULL = default stream).  Shape limits:
  * head_dim in {32, 64, 128}; n_heads % n_kv_heads == 0; d_model, d_ffn, n_heads*head_dim multiples of 8;
  * max_c <= 64.  The bf16 tensor-core path needs an sm_100a device; FC_F32 runs on FMA kernels. */
 int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weights *weights,
             void *kv, size_t kv_bytes, void *ws, size_t ws_bytes, void *cuda_stream);
 
-/* Start `batch` sequences.  prompt_ids: host [batch, p_stride]; prompt_lens: host [batch], each >= 1.
- * Caches K/V of prompt[0 .. P-2]; prompt[P-1] becomes the pending exact token (window slot 0);
- * slots 1..c-1 are filled by the refill rule.  Section 3.1 (prompt + window form the first input). */
+/* Start `batch` sequences (dropping any previous ones).  prompt_ids: host [batch, p_stride]; prompt_lens:
+ * host [batch], each >= 1.  Caches K/V of prompt[0 .. P-2] in blocks of at least 128 rows per forward;
+ * prompt[P-1] becomes the pending exact token (window slot 0); slots 1..c-1 are filled by the refill rule.
+ * "Overview of FastCoT": the prompt and the window taken from the buffer form the first input. */
 int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids, int32_t p_stride,
                const int32_t *prompt_lens, int32_t c, int32_t refill, int32_t pad_id);
 
@@ -106,11 +111,31 @@ int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids, int32_t p_
 int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *accepted_count,
                    int32_t *accepted_tokens, int32_t *window_out);
 
-/* Iterate until every sequence has committed max_tokens tokens or eos_id (eos_id < 0: never).
- * Streams are cut at max_tokens and just after the first EOS (Section 3.4, condition 2).
- * out_tokens: host [batch, max_tokens]; out_lens: host [batch]; stats nullable. */
-int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t eos_id, int32_t *out_tokens,
-                int32_t *out_lens, fc_stats *stats);
+/* Change the number of window rows c between iterations (the paper treats the context-window length as a free
+ * parameter, "Context Window Length"): the pending token and the guesses that still fit are kept, new slots are
+ * filled by the refill rule for their generated index.  1 <= c <= max_c. */
+int fc_set_window(fc_ctx *ctx, int32_t c);
+
+/* Iterate with c rows per forward (c <= 0: keep the current window size; otherwise as fc_set_window) until every
+ * sequence has committed max_tokens tokens since its prefill or eos_id (eos_id < 0: never), or until max_iters
+ * forwards have run (max_iters <= 0: no cap).  "Iteration Stop Condition": condition 1 is an upper bound on the
+ * iterations, condition 2 a verified EOS.  Streams are cut at max_tokens and just after the first EOS.
+ * out_tokens: host [batch, max_tokens], receives the tokens committed by THIS call; out_lens: host [batch];
+ * stats nullable.  A later call with a larger max_tokens goes on where this one stopped (sequences that ended
+ * on eos_id stay finished). */
+int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t c, int32_t eos_id, int32_t max_iters,
+                int32_t *out_tokens, int32_t *out_lens, fc_stats *stats);
+
+/* Hand-off of the approximate rationale ("Overview of FastCoT", last step; "Trigger Answer"): everything generated
+ * so far - the exact tokens and the approximate tokens still in the window, taken as they are - is joined with the
+ * answer trigger, and the answer is decoded greedily (Eq. 1) from there.  Per sequence the context
+ * [window slot 0 .. c-1 | trigger_ids] is appended to the cache (all but its last token, which becomes the pending
+ * token) and up to max_answer_tokens tokens are decoded, cut just after eos_id (eos_id < 0: never).
+ * trigger_ids: host [n_trigger] (n_trigger may be 0); answer_tokens: host [batch, max_answer_tokens];
+ * answer_lens: host [batch].  Needs kv_len + c + n_trigger + max_answer_tokens <= max_seq.  The Jacobi state is
+ * consumed: call fc_prefill before iterating again. */
+int fc_finish_with_trigger(fc_ctx *ctx, const int32_t *trigger_ids, int32_t n_trigger, int32_t max_answer_tokens,
+                           int32_t eos_id, int32_t *answer_tokens, int32_t *answer_lens);
 
 /* Benchmark/debug aids.  fc_debug_set_state: declare `batch` sequences with kv_lens[b] tokens
  * already present in the K/V slab (written by the caller) and pending tokens pending[b]; windows are
@@ -121,6 +146,14 @@ int fc_debug_set_state(fc_ctx *ctx, int32_t batch, const int32_t *kv_lens, const
                        int32_t c, int32_t pad_id);
 int fc_debug_logits(fc_ctx *ctx, float *dev_logits);
 int fc_get_state(fc_ctx *ctx, int32_t *kv_lens, int32_t *n_gen);
+
+/* Robustness aids for tests (no compute-sanitizer is assumed).  fc_debug_inject_timeout: the accept kernel of the
+ * next step raises the device error word exactly as an expired bounded wait would, without any wait; that step
+ * returns FC_ERR_DEVICE_TIMEOUT and the context needs fc_prefill.  fc_debug_check_guards: the workspace slices are
+ * separated by canary bands written at fc_init; *n_damaged (host) receives how many of them no longer hold the
+ * pattern (0 = no kernel wrote outside its slice). */
+int fc_debug_inject_timeout(fc_ctx *ctx);
+int fc_debug_check_guards(fc_ctx *ctx, int32_t *n_damaged);
 
 /* Enqueue `n_steps` iterations back to back with no host round trip in between and return the
  * device time in milliseconds from the first to the last kernel (CUDA events on the context's
@@ -175,6 +208,22 @@ int fc_op_window_attention(const void *q, const void *kcache, const void *vcache
                            float *out, int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
                            int32_t head_dim, int32_t max_seq, int32_t max_len, int32_t dtype,
                            void *scratch, size_t scratch_bytes, void *cuda_stream);
+
+/* The attention kernel of the bf16 step as it runs inside fc_jacobi_step (head_dim 64 or 128): applies the deferred
+ * RMSNorm factor 1/sqrt(sumsq[r] / d_norm + rms_eps) to the q, k and v accumulators of every window row, rotates q and k
+ * at position kv_len[b] + j (pairs i <-> i + head_dim/2, angle pos * rope_theta^(-2i/head_dim)), stores the window's k and v
+ * rows as bf16 at cache slots kv_len[b] .. kv_len[b]+c-1, and computes the window attention of Eq. 4's forward as
+ * fc_op_window_attention does.  qkv_acc: fp32 [batch*c, (n_heads + 2 n_kv_heads) * head_dim] = (q | k | v), cleared by
+ * the call; sumsq: fp32 [batch*c], cleared by the call; kcache/vcache: bf16 [batch][n_kv_heads][max_seq][head_dim],
+ * in/out; out: fp32 [batch*c, n_heads*head_dim].  chunks_per_cta: 0 = the grid fc_jacobi_step would choose, > 0 forces
+ * that many 128-key chunks per CTA.  scratch: device, 256-byte aligned, >= ..._scratch_bytes(...). */
+size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
+                                                  int32_t head_dim, int32_t max_seq, int32_t max_len);
+int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float rms_eps, int32_t d_norm, float rope_theta,
+                                 void *kcache, void *vcache, const int32_t *kv_len, float *out, int32_t batch,
+                                 int32_t c, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_seq,
+                                 int32_t max_len, int32_t chunks_per_cta, void *scratch, size_t scratch_bytes,
+                                 void *cuda_stream);
 
 /* The same window attention for callers that may not allocate device memory (the paper has no
  * counterpart; this exists for hosts whose device memory is owned by someone else, e.g. a serving

@@ -56,7 +56,9 @@ def _load():
         lib.orc_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         lib.orc_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int]
         lib.orc_jacobi_step.argtypes = [C.c_void_p] + [C.c_void_p] * 5
-        lib.orc_generate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.orc_generate.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.orc_set_window.argtypes = [C.c_void_p, C.c_int]
+        lib.orc_finish_with_trigger.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
         lib.orc_ar_generate.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                         C.c_void_p, C.c_void_p]
         lib.orc_round_bf16.restype = C.c_float
@@ -222,16 +224,34 @@ class Oracle:
         res = (int(k.value), acc[:k.value].copy(), wout)
         return res + (logits,) if want_logits else res
 
-    def generate(self, max_tokens: int, eos_id: int = -1):
+    def generate(self, max_tokens: int, eos_id: int = -1, max_iters: int = 0):
         """Returns (tokens, accept_counts per step)."""
         out = np.empty(max_tokens, np.int32)
         counts = np.zeros(max(max_tokens, 1), np.int32)
         steps = C.c_int32(0)
-        n = self._lib.orc_generate(self._h, max_tokens, eos_id, out.ctypes.data, counts.ctypes.data,
+        n = self._lib.orc_generate(self._h, max_tokens, eos_id, max_iters, out.ctypes.data, counts.ctypes.data,
                                    C.addressof(steps))
         if n < 0:
             raise RuntimeError(f"orc_generate rc={n}")
         return out[:n].copy(), counts[:steps.value].copy()
+
+    def set_window(self, c: int):
+        """Change the rows per forward between iterations; returns the resized window."""
+        rc = self._lib.orc_set_window(self._h, c)
+        if rc:
+            raise RuntimeError(f"orc_set_window rc={rc}")
+        self.c = c
+
+    def finish_with_trigger(self, trigger, max_answer: int, eos_id: int = -1):
+        """Exact + approximate tokens + answer trigger, then greedy answer tokens.  Ends the Jacobi state."""
+        t = _i32(trigger)
+        out = np.empty(max(max_answer, 1), np.int32)
+        n = self._lib.orc_finish_with_trigger(self._h, t.ctypes.data if t.shape[0] else None, t.shape[0],
+                                              max_answer, eos_id, out.ctypes.data)
+        if n < 0:
+            raise RuntimeError(f"orc_finish_with_trigger rc={n}")
+        self.c = 0
+        return out[:n].copy()
 
     def ar_generate(self, prompt, max_tokens: int, eos_id: int = -1):
         """Plain greedy decoding.  Returns (tokens, top1-top2 logit margins)."""

@@ -8,16 +8,19 @@
  * What it computes
  *   - decoder forward: a Llama-style causal decoder (RMSNorm, rotary embedding with
  *     half-split pairing, grouped-query attention, SwiGLU FFN, untied LM head), the model
- *     family the paper evaluates (Section 5.1).  fp32 arithmetic throughout.  For a bf16 model the K and V
+ *     family the paper evaluates (Experiment Settings).  fp32 arithmetic throughout.  For a bf16 model the K and V
  *     rows are rounded to bfloat16 where they are stored (the model's K/V tensors have the model dtype).
  *   - greedy autoregressive decoding: Eq. 1.
  *   - one Jacobi-window iteration: exact token + approximate tokens in one causal forward
  *     (Eq. 2-4), verification of the previous guesses one by one (Eq. 5), and the buffer /
- *     index update (Section 3.3 "Cache Update", Section 3.2 buffer initialisation).
+ *     index update (Method, "Cache Update"; "Approximate Tokens Buffer" for its initialisation).
+ *   - the hand-off of the approximate rationale: exact tokens + current approximate tokens +
+ *     answer trigger, then greedy decoding of the answer (Method, "Overview of FastCoT" and
+ *     "Trigger Answer"), and the iteration cap of "Iteration Stop Condition" (condition 1).
  *
  * Every output row is evaluated by the same scalar routine with a fixed summation order,
  * so row j of a window forward is bitwise the autoregressive forward of the same context.
- * That makes the paper's losslessness statement (Section 3.1: each forward yields at least
+ * That makes the paper's losslessness statement ("Overview of FastCoT": each forward yields at least
  * one token identical to autoregressive decoding) checkable exactly.
  *
  * Pins (tests/test_oracle_*.py): stream == greedy AR stream; closed form of the accept
@@ -58,7 +61,7 @@ typedef struct orc {
   orc_weights w;
   float *kcache, *vcache;    /* [layer][max_seq][n_kv_heads*head_dim] */
   int32_t kv_len;            /* tokens whose K/V is committed */
-  /* Jacobi state (Section 3.2): window = pending exact token + guesses */
+  /* Jacobi state ("Approximate Tokens Buffer"): window = pending exact token + guesses */
   int32_t *prompt; int32_t prompt_len;
   int32_t *window; int32_t c;
   int32_t n_gen; int32_t refill; int32_t pad_id;
@@ -138,7 +141,7 @@ static void rope(float *v, int hd, int pos, float theta) {
  * Forward `n` tokens at absolute positions kv_len .. kv_len+n-1 on top of the committed
  * cache.  K/V of the new rows are written at cache slots kv_len .. kv_len+n-1 (scratch until
  * committed).  Row j attends keys 0 .. kv_len+j: the cache plus the causal part of the
- * window (Section 3.3, "FastCoT Inference": lossless and Jacobi decoding share one forward
+ * window (Method, "FastCoT Inference": lossless and Jacobi decoding share one forward
  * through the causal mask).  logits_out: [n, vocab] or NULL.  argmax_out: [n] or NULL;
  * ties go to the lowest token id, NaN never wins.  Returns 0, or -1 on capacity overflow. */
 int orc_forward(orc *o, const int32_t *tokens, int n, float *logits_out, int32_t *argmax_out) {
@@ -292,11 +295,11 @@ int orc_set_kv(orc *o, int layer, const float *k, const float *v, int len) {
 }
 
 /* ------------------------------------------------------------------ Jacobi-window decoding
- * State (Section 3.2): committed tokens T[0..N-1]; K/V cached for T[0..N-2]; window w[0..c-1]
+ * State ("Approximate Tokens Buffer"): committed tokens T[0..N-1]; K/V cached for T[0..N-2]; window w[0..c-1]
  * with w[0] = T[N-1] (exact, K/V not cached yet) and w[j>=1] the guess for token N-1+j. */
 
 /* Initial / replacement guess for generated index g (0-based among generated tokens):
- * the prompt's own ids, cycled (Section 3.2: buffer initialised from the question's token ids),
+ * the prompt's own ids, cycled ("Approximate Tokens Buffer": initialised from the question's token ids),
  * or a pad id (the alternative the paper mentions). */
 static int32_t refill_token(const orc *o, int g) {
   return o->refill == 1 ? o->pad_id : o->prompt[g % o->prompt_len];
@@ -321,7 +324,7 @@ int orc_prefill(orc *o, const int32_t *prompt, int P, int c, int refill, int pad
   return 0;
 }
 
-/* Verification (Eq. 5) and buffer update (Section 3.3 "Cache Update") on plain arrays.
+/* Verification (Eq. 5) and buffer update (Method, "Cache Update") on plain arrays.
  * w[0..c-1]: the window that was fed (w[0] exact); a[j]: greedy token following window slot j;
  * n_gen: tokens generated before this step.  a[0] is always exact; a[j] is exact as long as every
  * guess w[1..j] equalled the exact token before it: check one by one.  Outputs: *k in [1, c],
@@ -378,14 +381,29 @@ int orc_jacobi_step(orc *o, const int32_t *window_in, int32_t *accepted, int32_t
   return 0;
 }
 
-/* Iterate until max_tokens are committed or eos_id is committed (eos_id < 0: never).  The
- * stream is cut at max_tokens and just after the first EOS; accept_counts[i] (optional, up to
- * max_tokens entries) gets the per-step count after that cut.  Returns the stream length. */
-int orc_generate(orc *o, int max_tokens, int eos_id, int32_t *out_tokens, int32_t *accept_counts,
-                 int32_t *n_steps) {
+/* Change the number of rows per forward between iterations (the paper studies the context-window
+ * length as a free parameter, "Context Window Length"; nothing in Eq. 4-5 ties one iteration's c to the
+ * next).  The pending exact token stays in slot 0; guesses that still fit are kept; new slots get the
+ * refill rule's guess for their generated index. */
+int orc_set_window(orc *o, int c_new) {
+  if (!o->window || c_new < 1 || o->kv_len + c_new > o->s.max_seq) return -1;
+  int32_t *w2 = malloc(sizeof(int32_t) * c_new);
+  for (int j = 0; j < c_new; ++j)
+    w2[j] = j < o->c ? o->window[j] : refill_token(o, o->n_gen + j - 1);
+  free(o->window);
+  o->window = w2; o->c = c_new;
+  return 0;
+}
+
+/* Iterate until max_tokens are committed, eos_id is committed (eos_id < 0: never) or max_iters forwards
+ * have run (max_iters <= 0: no cap; "Iteration Stop Condition": an upper bound on the iterations, and a
+ * verified EOS).  The stream is cut at max_tokens and just after the first EOS; accept_counts[i]
+ * (optional, up to max_tokens entries) gets the per-step count after that cut.  Returns the stream length. */
+int orc_generate(orc *o, int max_tokens, int eos_id, int max_iters, int32_t *out_tokens,
+                 int32_t *accept_counts, int32_t *n_steps) {
   int n = 0, steps = 0, done = 0;
   int32_t *acc = malloc(sizeof(int32_t) * o->c);
-  while (n < max_tokens && !done) {
+  while (n < max_tokens && !done && (max_iters <= 0 || steps < max_iters)) {
     int32_t k;
     int rc = orc_jacobi_step(o, NULL, &k, acc, NULL, NULL);
     if (rc) { free(acc); return rc; }
@@ -399,6 +417,45 @@ int orc_generate(orc *o, int max_tokens, int eos_id, int32_t *out_tokens, int32_
   }
   if (n_steps) *n_steps = steps;
   free(acc);
+  return n;
+}
+
+/* Hand-off of the approximate rationale ("Overview of FastCoT", last step; "Trigger Answer"): when the
+ * iteration stops, everything generated so far - the exact tokens AND the approximate tokens still in
+ * the window - is joined with the answer trigger, and the answer is decoded greedily from there.
+ * Context = committed cache | w[0] (pending exact) | w[1..c-1] (approximate, taken as they are) |
+ * trigger[0..n_trig-1]; all of it is committed to the cache except its last token, which becomes the
+ * pending token of a plain autoregressive decode (Eq. 1) of up to max_answer tokens (cut after eos_id).
+ * Afterwards the Jacobi state is gone (the buffer was consumed): prefill again before iterating.
+ * Returns the number of answer tokens. */
+int orc_finish_with_trigger(orc *o, const int32_t *trigger, int n_trig, int max_answer, int eos_id,
+                            int32_t *answer) {
+  if (!o->window || n_trig < 0 || max_answer < 0) return -1;
+  const int n_ctx = o->c + n_trig;                 /* rows: window then trigger */
+  if (o->kv_len + n_ctx + max_answer > o->s.max_seq) return -1;
+  int32_t *ctx = malloc(sizeof(int32_t) * n_ctx);
+  memcpy(ctx, o->window, sizeof(int32_t) * o->c);
+  for (int j = 0; j < n_trig; ++j) ctx[o->c + j] = trigger[j];
+  for (int j = 0; j < n_ctx; ++j) if (ctx[j] < 0 || ctx[j] >= o->s.vocab) { free(ctx); return -2; }
+  for (int start = 0; start < n_ctx - 1; start += 64) {   /* chunked only to bound scratch */
+    int n = n_ctx - 1 - start < 64 ? n_ctx - 1 - start : 64;
+    int rc = orc_forward(o, ctx + start, n, NULL, NULL);
+    if (rc) { free(ctx); return rc; }
+    o->kv_len += n;
+  }
+  int32_t tok = ctx[n_ctx - 1];
+  free(ctx);
+  int n = 0;
+  while (n < max_answer) {
+    int32_t nxt;
+    int rc = orc_forward(o, &tok, 1, NULL, &nxt);
+    if (rc) return rc;
+    o->kv_len += 1;
+    answer[n++] = nxt;
+    tok = nxt;
+    if (eos_id >= 0 && nxt == eos_id) break;
+  }
+  free(o->window); o->window = NULL; o->c = 0;
   return n;
 }
 

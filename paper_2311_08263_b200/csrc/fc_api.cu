@@ -15,14 +15,24 @@ namespace {
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
+constexpr size_t kGuardBytes = 256;       // canary band between two slices of the workspace
+constexpr unsigned char kGuardByte = 0xC5;
+
 struct Carver {          // hands out aligned slices of the caller's workspace (or just counts bytes)
   char *base; size_t off;
+  std::vector<size_t> *guards;     // offsets of the canary bands (recorded when non-null)
   template <typename T> T *take(size_t n) {
     T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
     off = align_up(off + n * sizeof(T));
     return p;
   }
+  void guard() {
+    if (guards) guards->push_back(off);
+    off += kGuardBytes;
+  }
 };
+
+constexpr int kPrefillRows = 128;         // rows per forward while a prompt is cached (one 128-row accumulator block)
 
 
 constexpr int kSyncClaim = kChainMax, kSyncPanel = 2 * kChainMax, kSyncTd = 3 * kChainMax;   // offsets in a group
@@ -35,10 +45,13 @@ struct Buffers {
   unsigned int *counters, *err, *chain_bar;
   unsigned long long *amax;
   int32_t *window, *kv_len, *n_gen, *done, *acc_count, *acc_tokens, *prompt, *prompt_lens, *out_tokens;
+  int32_t *row_tokens;     // tokens of a forward that is not a decode step (answer-trigger context)
 };
 
 struct Dims {
-  int rmax, qd, kvd, ldq, nsplit_max, tk, pan_rows, pan_k, sync_words;
+  int rmax;        // rows of a decode step: max_batch * max_c
+  int rows_ws;     // rows the activation buffers hold: a decode step or a prefill block, whichever is larger
+  int qd, kvd, ldq, nsplit_max, tk, pan_rows, pan_k, sync_words;
   size_t esz;
 };
 
@@ -56,6 +69,7 @@ bool shape_ok(const fc_model_shape *s) {
 Dims dims_of(const fc_model_shape *s) {
   Dims d;
   d.rmax = s->max_batch * s->max_c;
+  d.rows_ws = d.rmax > kPrefillRows ? d.rmax : kPrefillRows;
   d.qd = s->n_heads * s->head_dim;
   d.kvd = s->n_kv_heads * s->head_dim;
   d.ldq = d.qd + 2 * d.kvd;
@@ -63,7 +77,7 @@ Dims dims_of(const fc_model_shape *s) {
   d.nsplit_max = (s->max_seq + d.tk - 1) / d.tk;
   d.esz = s->dtype == FC_F32 ? 4 : 2;
   // beyond 16 rows the tensor-core projections read their activations from a bf16 high/low panel
-  d.pan_rows = d.rmax > 16 ? (d.rmax + 127) / 128 * 128 : 0;
+  d.pan_rows = (d.rows_ws + 127) / 128 * 128;
   d.pan_k = s->d_model > s->d_ffn ? s->d_model : s->d_ffn;
   if (d.qd > d.pan_k) d.pan_k = d.qd;
   // per-layer group of synchronisation words: grid barriers 0..5, work-claim counters 6..11, panel-ready barriers
@@ -73,38 +87,40 @@ Dims dims_of(const fc_model_shape *s) {
   return d;
 }
 
-size_t carve(const fc_model_shape *s, char *base, Buffers *b) {
+size_t carve(const fc_model_shape *s, char *base, Buffers *b, std::vector<size_t> *guards = nullptr) {
   Dims d = dims_of(s);
-  Carver c{base, 0};
+  Carver c{base, 0, guards};
   Buffers t;
-  const size_t R = d.rmax;
-  t.x = c.take<float>(R * s->d_model);
-  t.qkv = c.take<float>(R * d.ldq);
-  t.qb = c.take<char>(R * d.qd * d.esz);
-  t.attn = c.take<float>(R * d.qd);
-  t.gu = c.take<float>(R * 2 * (size_t)s->d_ffn);
+  const size_t R = d.rows_ws, Rs = d.rmax;
+  c.guard();
+  t.x = c.take<float>(R * s->d_model); c.guard();
+  t.qkv = c.take<float>(R * d.ldq); c.guard();
+  t.qb = c.take<char>(R * d.qd * d.esz); c.guard();
+  t.attn = c.take<float>(R * d.qd); c.guard();
+  t.gu = c.take<float>(R * 2 * (size_t)s->d_ffn); c.guard();
+  // sums of squares, then one group of synchronisation words per layer plus one for the first QKV and the LM head:
+  // adjacent (no canary band in between) so that one pass clears them all
   t.ss_attn = c.take<float>(R);
   t.ss_ffn = c.take<float>(R);
   t.ss_final = c.take<float>(R);
-  // one group of synchronisation words per layer plus one for the first QKV and the LM head; directly after the
-  // sums of squares so that one pass clears them all
-  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * d.sync_words);
-  t.pan = c.take<char>((size_t)2 * d.pan_rows * d.pan_k * 2);
-  t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim);
-  t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2);
-  t.rope = c.take<float2>((size_t)s->max_seq * (s->head_dim / 2));
+  t.chain_bar = c.take<unsigned int>(((size_t)s->n_layers + 1) * d.sync_words); c.guard();
+  t.pan = c.take<char>((size_t)2 * d.pan_rows * d.pan_k * 2); c.guard();
+  t.part_o = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * s->head_dim); c.guard();
+  t.part_ml = c.take<float>(R * s->n_heads * (size_t)d.nsplit_max * 2); c.guard();
+  t.rope = c.take<float2>((size_t)s->max_seq * (s->head_dim / 2)); c.guard();
   t.counters = c.take<unsigned int>((size_t)s->max_batch * s->n_kv_heads + 1);   // + one grid-wide word
   t.err = c.take<unsigned int>(1);
-  t.amax = c.take<unsigned long long>(R);
-  t.window = c.take<int32_t>(R);
+  t.amax = c.take<unsigned long long>(Rs); c.guard();
+  t.window = c.take<int32_t>(Rs);
   t.kv_len = c.take<int32_t>(s->max_batch);
   t.n_gen = c.take<int32_t>(s->max_batch);
   t.done = c.take<int32_t>(s->max_batch);
   t.acc_count = c.take<int32_t>(s->max_batch);
-  t.acc_tokens = c.take<int32_t>(R);
+  t.acc_tokens = c.take<int32_t>(Rs); c.guard();
   t.prompt = c.take<int32_t>((size_t)s->max_batch * s->max_seq);
   t.prompt_lens = c.take<int32_t>(s->max_batch);
   t.out_tokens = c.take<int32_t>((size_t)s->max_batch * s->max_seq);
+  t.row_tokens = c.take<int32_t>(R); c.guard();
   if (b) *b = t;
   return c.off;
 }
@@ -137,7 +153,12 @@ struct fc_ctx {
   int batch = 0, c = 0, refill = 0, pad_id = 0, p_stride = 0;
   bool ready = false;
   std::vector<int32_t> kv_len_h, n_gen_h, pending_h, done_h;
+  std::vector<std::vector<int32_t>> prompt_h;   // host copies of the prompts (refill rule when the window is resized)
   int gen_max_tokens = 0, gen_eos = -1;
+  float ms_prefill = 0.f;        // device time of the most recent fc_prefill
+  bool inject_timeout = false;   // test aid: the next step's accept kernel raises the device error word
+  char *ws_base = nullptr;
+  std::vector<size_t> guards;    // offsets of the canary bands inside the workspace
   // pinned staging: [count | tokens | window | err]
   int32_t *pin = nullptr;
   int64_t launches = 0;
@@ -291,7 +312,8 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   if (!ctx) return FC_ERR_ARG;
   ctx->s = *shape;
   ctx->d = dims_of(shape);
-  carve(shape, (char *)ws, &ctx->b);
+  carve(shape, (char *)ws, &ctx->b, &ctx->guards);
+  ctx->ws_base = (char *)ws;
   ctx->tok_emb = w->tok_emb; ctx->g_final = w->g_final; ctx->lm_head = w->lm_head; ctx->bias_perm = w->bias_perm;
   const int L = shape->n_layers;
   auto copy = [&](std::vector<const void *> &dst, const void *const *src) { dst.assign(src, src + L); };
@@ -341,6 +363,8 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   if (cudaMallocHost((void **)&ctx->pin, pin_ints * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaEventCreate(&ctx->ev0) != cudaSuccess || cudaEventCreate(&ctx->ev1) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaMemsetAsync(ws, 0, fc_workspace_bytes(shape), ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
+  for (size_t off : ctx->guards)      // canary bands between the slices (checked by fc_debug_check_guards)
+    if (cudaMemsetAsync((char *)ws + off, kGuardByte, kGuardBytes, ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
   {
     // cos/sin of pos * theta^(-2i/hd), evaluated on the host in fp32 (inverse frequency in fp32, angle in fp32):
     // the device's powf is a few ulp off, and at positions in the thousands an ulp of the frequency is 1e-4 rad
@@ -360,8 +384,23 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   if (cudaStreamSynchronize(ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
   const int B = shape->max_batch;
   ctx->kv_len_h.assign(B, 0); ctx->n_gen_h.assign(B, 0); ctx->pending_h.assign(B, 0); ctx->done_h.assign(B, 0);
+  ctx->prompt_h.assign(B, std::vector<int32_t>());
   *out = ctx;
   return FC_OK;
+}
+
+// Grid of the fused attention kernel: one CTA per 128-key chunk while all of them are resident at once (two per
+// SM); beyond, a CTA walks over cpc consecutive chunks and every 16-row query tile has CTAs of its own.
+static void fused_attn_grid(int nsplit, int hq, int hkv, int nb, int rows, int n_sms, int &cpc, int &qsplit) {
+  cpc = 1; qsplit = 1;
+  const int nqt = ((hq / hkv) * rows + 15) / 16;
+  const long long per_split = (long long)hkv * nb;
+  if ((long long)nsplit * per_split > 2ll * n_sms) {          // more CTAs than are resident at once
+    long long groups = 2ll * n_sms / (per_split * nqt);       // as many CTAs as are resident at once, not more
+    if (groups < 1) groups = 1;
+    cpc = (int)((nsplit + groups - 1) / groups);
+    if (cpc > 1) qsplit = nqt;
+  }
 }
 
 static void prof_mark(fc_ctx *ctx, int cls, bool begin) {
@@ -435,16 +474,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       // several consecutive chunks, so that the queries are staged and the partial result is written once per CTA
       // (every 16-row query tile then has CTAs of its own).
       int cpc = 1, qsplit = 1;
-      {
-        const int nqt = ((s.n_heads / s.n_kv_heads) * rows + 15) / 16;
-        const long long per_split = (long long)s.n_kv_heads * nb;
-        if ((long long)nsplit * per_split > 2ll * ctx->n_sms) {       // more CTAs than are resident at once
-          long long groups = 2ll * ctx->n_sms / (per_split * nqt);      // as many CTAs as are resident at once, not more
-          if (groups < 1) groups = 1;
-          cpc = (int)((nsplit + groups - 1) / groups);
-          if (cpc > 1) qsplit = nqt;
-        }
-      }
+      fused_attn_grid(nsplit, s.n_heads, s.n_kv_heads, nb, rows, ctx->n_sms, cpc, qsplit);
       fa.qsplit = qsplit;
       fa.cpc = cpc;
       fa.nsplit = (nsplit + cpc - 1) / cpc; fa.part_o = ctx->b.part_o; fa.part_ml = ctx->b.part_ml; fa.counters = ctx->b.counters;
@@ -458,7 +488,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       RopeArgs ra; memset(&ra, 0, sizeof ra);
       ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
       ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows;
-      ra.hq = s.n_heads; ra.hkv = s.n_kv_heads; ra.hd = s.head_dim; ra.theta = s.rope_theta;
+      ra.hq = s.n_heads; ra.hkv = s.n_kv_heads; ra.hd = s.head_dim; ra.rope = ctx->b.rope;
       ra.q_out = ctx->b.qb; ra.kcache = kc; ra.vcache = vc;
       ra.stride_b = stride_b; ra.stride_h = stride_h;
       ra.z.p[0] = ctx->b.gu; ra.z.n[0] = Rz * 2 * s.d_ffn;
@@ -485,17 +515,19 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ChainSync sy[kChainMax];
       int n = 0;
       const bool split = ctx->ffn_split && R <= 16;
-      plans[n] = ctx->plan_o[l]; ga[n] = args_o(ctx, l); sy[n++] = ChainSync{-1, -1, 0, -1};
+      plans[n] = ctx->plan_o[l]; ga[n] = args_o(ctx, l); sy[n++] = ChainSync{-1, -1, 0, -1, -1};
       if (split) {
-        plans[n] = ctx->plan_gu_half[0][l]; ga[n] = args_gu_half(ctx, l, 0); sy[n++] = ChainSync{-1, 0, -1, 0};
-        plans[n] = ctx->plan_gu_half[1][l]; ga[n] = args_gu_half(ctx, l, 1); sy[n++] = ChainSync{-1, 1, -1, 0};
-        plans[n] = ctx->plan_down_half[0][l]; ga[n] = args_down_half(ctx, l, 0); sy[n++] = ChainSync{0, -1, 1, -1};
-        plans[n] = ctx->plan_down_half[1][l]; ga[n] = args_down_half(ctx, l, 1); sy[n++] = ChainSync{1, -1, 1, -1};
+        plans[n] = ctx->plan_gu_half[0][l]; ga[n] = args_gu_half(ctx, l, 0); sy[n++] = ChainSync{-1, 0, -1, 0, -1};
+        plans[n] = ctx->plan_gu_half[1][l]; ga[n] = args_gu_half(ctx, l, 1); sy[n++] = ChainSync{-1, 1, -1, 0, -1};
+        // the first down half adds to the residual that the second gate/up half may still be reading: its epilogue
+        // passes that half's barrier (normally long reached) before the first addition
+        plans[n] = ctx->plan_down_half[0][l]; ga[n] = args_down_half(ctx, l, 0); sy[n++] = ChainSync{0, -1, 1, -1, 1};
+        plans[n] = ctx->plan_down_half[1][l]; ga[n] = args_down_half(ctx, l, 1); sy[n++] = ChainSync{1, -1, 1, -1, -1};
       } else {
-        plans[n] = ctx->plan_gu[l]; ga[n] = args_gu(ctx, l); sy[n++] = ChainSync{-1, 0, -1, 0};
-        plans[n] = ctx->plan_down[l]; ga[n] = args_down(ctx, l); sy[n++] = ChainSync{0, -1, 1, -1};
+        plans[n] = ctx->plan_gu[l]; ga[n] = args_gu(ctx, l); sy[n++] = ChainSync{-1, 0, -1, 0, -1};
+        plans[n] = ctx->plan_down[l]; ga[n] = args_down(ctx, l); sy[n++] = ChainSync{0, -1, 1, -1, -1};
       }
-      if (l + 1 < s.n_layers) { plans[n] = ctx->plan_qkv[l + 1]; ga[n] = args_qkv(ctx, l + 1); sy[n++] = ChainSync{-1, -1, -1, 1}; }
+      if (l + 1 < s.n_layers) { plans[n] = ctx->plan_qkv[l + 1]; ga[n] = args_qkv(ctx, l + 1); sy[n++] = ChainSync{-1, -1, -1, 1, -1}; }
       for (int i = 0; i < n; ++i) ga[i].R = R;
       ++ctx->launches;
       ProfScope ps(ctx, FC_CLS_CHAIN);
@@ -520,6 +552,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     ac.out_tokens = ctx->b.out_tokens; ac.out_stride = s.max_seq;
     ac.b0 = b0; ac.nb = nb; ac.c = rows; ac.p_stride = s.max_seq; ac.refill = ctx->refill; ac.pad_id = ctx->pad_id;
     ac.max_tokens = ctx->gen_max_tokens; ac.eos_id = ctx->gen_eos; ac.commit = commit;
+    if (ctx->inject_timeout) { ac.err_inject = ctx->b.err; ctx->inject_timeout = false; }
     ++ctx->launches;
     { ProfScope ps(ctx, FC_CLS_ACCEPT); FC_CK(launch_accept(ac, ctx->st)); }
   } else {
@@ -575,6 +608,7 @@ extern "C" int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids,
     for (int j = 1; j < c; ++j)
       win[(size_t)b * c + j] = refill == FC_REFILL_PAD ? pad_id : prompt_ids[(size_t)b * p_stride + (j - 1) % P];
     ctx->kv_len_h[b] = 0; ctx->n_gen_h[b] = 0; ctx->done_h[b] = 0; ctx->pending_h[b] = win[(size_t)b * c];
+    ctx->prompt_h[b].assign(prompt_ids + (size_t)b * p_stride, prompt_ids + (size_t)b * p_stride + P);
   }
   FC_CK(cudaMemcpyAsync(ctx->b.prompt_lens, prompt_lens, sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
   FC_CK(cudaMemcpyAsync(ctx->b.window, win.data(), sizeof(int32_t) * win.size(), cudaMemcpyHostToDevice, ctx->st));
@@ -582,18 +616,22 @@ extern "C" int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids,
   FC_CK(cudaMemcpyAsync(ctx->b.n_gen, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
   FC_CK(cudaMemcpyAsync(ctx->b.done, zeros.data(), sizeof(int32_t) * batch, cudaMemcpyHostToDevice, ctx->st));
   FC_CK(cudaStreamSynchronize(ctx->st));   // host vectors above go out of scope
-  // K/V of prompt[0 .. P-2], one sequence at a time in chunks of up to rmax rows
+  // K/V of prompt[0 .. P-2]: one sequence at a time, in blocks of as many rows as the activation buffers hold
+  // (at least one 128-row accumulator block, so that a prompt of P ids streams the weights ~P / 128 times)
+  FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
   for (int b = 0; b < batch; ++b) {
     const int n = prompt_lens[b] - 1;
-    for (int start = 0; start < n; start += ctx->d.rmax) {
-      const int rows = n - start < ctx->d.rmax ? n - start : ctx->d.rmax;
+    for (int start = 0; start < n; start += ctx->d.rows_ws) {
+      const int rows = n - start < ctx->d.rows_ws ? n - start : ctx->d.rows_ws;
       int rc = forward(ctx, b, 1, rows, ctx->b.prompt + (size_t)b * s.max_seq + start, false, start, 1);
       if (rc != FC_OK) return rc;
     }
     ctx->kv_len_h[b] = n;
   }
+  FC_CK(cudaEventRecord(ctx->ev1, ctx->st));
   int rc = check_device_error(ctx);
   if (rc != FC_OK) return rc;
+  FC_CK(cudaEventElapsedTime(&ctx->ms_prefill, ctx->ev0, ctx->ev1));
   ctx->ready = true;
   return FC_OK;
 }
@@ -617,7 +655,7 @@ static int collect_step(fc_ctx *ctx, int32_t *accepted_count, int32_t *accepted_
     ctx->kv_len_h[b] += k; ctx->n_gen_h[b] += k; ctx->pending_h[b] = p_win[(size_t)b * c];
     if (k > 0) {
       if (ctx->gen_max_tokens > 0 && ctx->n_gen_h[b] >= ctx->gen_max_tokens) ctx->done_h[b] = 1;
-      if (ctx->gen_eos >= 0 && p_tok[(size_t)b * c + k - 1] == ctx->gen_eos) ctx->done_h[b] = 1;
+      if (ctx->gen_eos >= 0 && p_tok[(size_t)b * c + k - 1] == ctx->gen_eos) ctx->done_h[b] = 2;   // ended for good
     }
   }
   if (accepted_count) memcpy(accepted_count, p_cnt, sizeof(int32_t) * B);
@@ -656,33 +694,81 @@ extern "C" int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *ac
   return collect_step(ctx, accepted_count, accepted_tokens, window_out);
 }
 
-extern "C" int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t eos_id, int32_t *out_tokens, int32_t *out_lens,
-                           fc_stats *stats) {
+// Resize every sequence's window to c_new rows: slot 0 (the pending exact token) and the guesses that still fit are
+// kept; new slots get the refill rule's guess for their generated index.
+static int resize_window(fc_ctx *ctx, int c_new) {
+  const int B = ctx->batch, c_old = ctx->c;
+  if (c_new == c_old) return FC_OK;
+  if (c_new < 1) return FC_ERR_ARG;
+  if (c_new > ctx->s.max_c) return FC_ERR_CAPACITY;
+  for (int b = 0; b < B; ++b)
+    if (ctx->kv_len_h[b] + c_new > ctx->s.max_seq) return FC_ERR_CAPACITY;
+  std::vector<int32_t> w_old((size_t)B * c_old), w_new((size_t)B * c_new);
+  FC_CK(cudaMemcpyAsync(w_old.data(), ctx->b.window, sizeof(int32_t) * w_old.size(), cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  for (int b = 0; b < B; ++b) {
+    const std::vector<int32_t> &pr = ctx->prompt_h[b];
+    for (int j = 0; j < c_new; ++j) {
+      int32_t t;
+      if (j < c_old) t = w_old[(size_t)b * c_old + j];
+      else if (ctx->refill == FC_REFILL_PAD || pr.empty()) t = ctx->pad_id;
+      else t = pr[(size_t)(ctx->n_gen_h[b] + j - 1) % pr.size()];
+      w_new[(size_t)b * c_new + j] = t;
+    }
+  }
+  FC_CK(cudaMemcpyAsync(ctx->b.window, w_new.data(), sizeof(int32_t) * w_new.size(), cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  ctx->c = c_new;
+  return FC_OK;
+}
+
+extern "C" int fc_set_window(fc_ctx *ctx, int32_t c) {
+  if (!ctx) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  return resize_window(ctx, c);
+}
+
+extern "C" int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t c, int32_t eos_id, int32_t max_iters,
+                           int32_t *out_tokens, int32_t *out_lens, fc_stats *stats) {
   if (!ctx || !out_tokens || !out_lens || max_tokens < 1) return FC_ERR_ARG;
   if (!ctx->ready) return FC_ERR_STATE;
-  const int B = ctx->batch, c = ctx->c;
+  const int B = ctx->batch;
+  if (c > 0 && c != ctx->c) {
+    int rc = resize_window(ctx, c);
+    if (rc != FC_OK) return rc;
+  }
+  c = ctx->c;
   for (int b = 0; b < B; ++b)
     if (ctx->kv_len_h[b] + (max_tokens - ctx->n_gen_h[b]) + c > ctx->s.max_seq) return FC_ERR_CAPACITY;
   ctx->gen_max_tokens = max_tokens; ctx->gen_eos = eos_id;
-  if (stats) memset(stats, 0, sizeof(*stats));
+  if (stats) { memset(stats, 0, sizeof(*stats)); stats->ms_prefill = ctx->ms_prefill; }
   std::vector<int32_t> cnt(B), tok((size_t)B * c);
+  // A sequence is finished when it has max_tokens tokens or ended on eos_id.  A later call with a larger max_tokens
+  // continues the sequences that only ran into the earlier limit: the flags are recomputed here and sent to the device.
   for (int b = 0; b < B; ++b) {
     out_lens[b] = 0;
-    if (ctx->n_gen_h[b] >= max_tokens) ctx->done_h[b] = 1;
+    const bool hit_eos = ctx->done_h[b] == 2;
+    ctx->done_h[b] = hit_eos ? 2 : (ctx->n_gen_h[b] >= max_tokens ? 1 : 0);
+    ctx->pin[b] = ctx->done_h[b] ? 1 : 0;
   }
+  FC_CK(cudaMemcpyAsync(ctx->b.done, ctx->pin, sizeof(int32_t) * B, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
   int64_t launches = 0;
+  int iters = 0;
   FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
   int rc = FC_OK;
   for (;;) {
     bool live = false;
     for (int b = 0; b < B; ++b) live |= !ctx->done_h[b];
     if (!live) break;
+    if (max_iters > 0 && iters >= max_iters) break;       // iteration cap ("Iteration Stop Condition", condition 1)
     ctx->launches = 0;
     rc = forward(ctx, 0, B, c, ctx->b.window, true, max_live_len(ctx), 1);
     if (rc != FC_OK) break;
     launches += ctx->launches;
     rc = collect_step(ctx, cnt.data(), tok.data(), nullptr);
     if (rc != FC_OK) break;
+    ++iters;
     for (int b = 0; b < B; ++b) {
       const int k = cnt[b];
       for (int j = 0; j < k && out_lens[b] < max_tokens; ++j) out_tokens[(size_t)b * max_tokens + out_lens[b]++] = tok[(size_t)b * c + j];
@@ -696,6 +782,91 @@ extern "C" int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t eos_id, int3
   FC_CK(cudaEventRecord(ctx->ev1, ctx->st));
   FC_CK(cudaEventSynchronize(ctx->ev1));
   if (stats) FC_CK(cudaEventElapsedTime(&stats->ms_steps, ctx->ev0, ctx->ev1));
+  return FC_OK;
+}
+
+extern "C" int fc_finish_with_trigger(fc_ctx *ctx, const int32_t *trigger_ids, int32_t n_trigger, int32_t max_answer_tokens,
+                                      int32_t eos_id, int32_t *answer_tokens, int32_t *answer_lens) {
+  if (!ctx || n_trigger < 0 || (n_trigger > 0 && !trigger_ids) || max_answer_tokens < 0 || !answer_lens ||
+      (max_answer_tokens > 0 && !answer_tokens)) return FC_ERR_ARG;
+  if (!ctx->ready) return FC_ERR_STATE;
+  const fc_model_shape &s = ctx->s;
+  const int B = ctx->batch, c = ctx->c;
+  for (int j = 0; j < n_trigger; ++j)
+    if (trigger_ids[j] < 0 || trigger_ids[j] >= s.vocab) return FC_ERR_TOKEN_RANGE;
+  const int n_ctx = c + n_trigger;           // rows per sequence: the window (pending exact token + approximate tokens), then the trigger
+  for (int b = 0; b < B; ++b)
+    if (ctx->kv_len_h[b] + n_ctx + max_answer_tokens > s.max_seq) return FC_ERR_CAPACITY;
+  ctx->launches = 0;
+  int64_t launches = 0;
+  // context rows of every sequence: [window | trigger]
+  std::vector<int32_t> win((size_t)B * c), rows_h((size_t)B * n_ctx);
+  FC_CK(cudaMemcpyAsync(win.data(), ctx->b.window, sizeof(int32_t) * win.size(), cudaMemcpyDeviceToHost, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  for (int b = 0; b < B; ++b) {
+    for (int j = 0; j < c; ++j) rows_h[(size_t)b * n_ctx + j] = win[(size_t)b * c + j];
+    for (int j = 0; j < n_trigger; ++j) rows_h[(size_t)b * n_ctx + c + j] = trigger_ids[j];
+  }
+  ctx->ready = false;                        // from here on the Jacobi state is consumed
+  // (1) commit K/V of every context row but the last, in blocks of rows; sequences one at a time (ragged lengths)
+  const int n_commit = n_ctx - 1;
+  for (int b = 0; b < B && n_commit > 0; ++b) {
+    for (int start = 0; start < n_commit; start += ctx->d.rows_ws) {
+      const int rows = n_commit - start < ctx->d.rows_ws ? n_commit - start : ctx->d.rows_ws;
+      FC_CK(cudaMemcpyAsync(ctx->b.row_tokens, rows_h.data() + (size_t)b * n_ctx + start, sizeof(int32_t) * rows,
+                            cudaMemcpyHostToDevice, ctx->st));
+      int rc = forward(ctx, b, 1, rows, ctx->b.row_tokens, false, ctx->kv_len_h[b] + start, 1);
+      if (rc != FC_OK) return rc;
+      FC_CK(cudaStreamSynchronize(ctx->st));   // rows_h / row_tokens are reused by the next block
+    }
+    ctx->kv_len_h[b] += n_commit;
+  }
+  launches += ctx->launches;
+  // (2) plain greedy decoding (Eq. 1) from the last context row: steps with one row per sequence
+  std::vector<int32_t> pend(B), zeros(B, 0);
+  for (int b = 0; b < B; ++b) { pend[b] = rows_h[(size_t)b * n_ctx + n_ctx - 1]; answer_lens[b] = 0; }
+  FC_CK(cudaMemcpyAsync(ctx->b.window, pend.data(), sizeof(int32_t) * B, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaMemcpyAsync(ctx->b.done, zeros.data(), sizeof(int32_t) * B, cudaMemcpyHostToDevice, ctx->st));
+  FC_CK(cudaStreamSynchronize(ctx->st));
+  ctx->c = 1; ctx->gen_max_tokens = 0; ctx->gen_eos = -1;
+  std::vector<int32_t> cnt(B), tok(B);
+  std::vector<char> ended(B, 0);
+  for (int i = 0; i < max_answer_tokens; ++i) {
+    bool live = false;
+    for (int b = 0; b < B; ++b) live |= !ended[b];
+    if (!live) break;
+    ctx->launches = 0;
+    int rc = forward(ctx, 0, B, 1, ctx->b.window, true, max_live_len(ctx), 1);
+    if (rc != FC_OK) return rc;
+    launches += ctx->launches;
+    rc = collect_step(ctx, cnt.data(), tok.data(), nullptr);
+    if (rc != FC_OK) return rc;
+    for (int b = 0; b < B; ++b) {
+      if (ended[b]) continue;
+      answer_tokens[(size_t)b * max_answer_tokens + answer_lens[b]++] = tok[b];
+      if (eos_id >= 0 && tok[b] == eos_id) ended[b] = 1;
+    }
+  }
+  ctx->launches = launches;
+  return check_device_error(ctx);
+}
+
+extern "C" int fc_debug_inject_timeout(fc_ctx *ctx) {
+  if (!ctx) return FC_ERR_ARG;
+  ctx->inject_timeout = true;
+  return FC_OK;
+}
+
+extern "C" int fc_debug_check_guards(fc_ctx *ctx, int32_t *n_damaged) {
+  if (!ctx || !n_damaged) return FC_ERR_ARG;
+  *n_damaged = 0;
+  std::vector<unsigned char> band(kGuardBytes);
+  for (size_t off : ctx->guards) {
+    FC_CK(cudaMemcpyAsync(band.data(), ctx->ws_base + off, kGuardBytes, cudaMemcpyDeviceToHost, ctx->st));
+    FC_CK(cudaStreamSynchronize(ctx->st));
+    for (unsigned char v : band)
+      if (v != kGuardByte) { ++*n_damaged; break; }
+  }
   return FC_OK;
 }
 
@@ -903,7 +1074,82 @@ int run_window_attention(const void *q, const void *kcache, const void *vcache, 
   if (launch_attn(aa, dtype, hd, st) != cudaSuccess) return FC_ERR_CUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
 }
+
+// ---- the fused kernel of the bf16 step (1/rms + rotary embedding + K/V write + window attention) as one operation
+static bool fused_shape_ok(int batch, int c, int hq, int hkv, int hd, int max_seq, int max_len) {
+  return batch >= 1 && c >= 1 && hq >= 1 && hkv >= 1 && hq % hkv == 0 && (hd == 64 || hd == 128) && max_len >= 0 &&
+         max_seq >= 1;
+}
+static void fused_layout(int batch, int c, int hq, int hkv, int hd, int max_seq, int max_len, size_t off[5]) {
+  const size_t nsplit = (size_t)(max_len + c + 127) / 128;
+  const size_t rows = (size_t)batch * c * hq;
+  off[0] = 0;                                                                   // rope table
+  off[1] = off[0] + align_up((size_t)max_seq * (hd / 2) * sizeof(float2));      // partial outputs
+  off[2] = off[1] + align_up(rows * nsplit * hd * sizeof(float));               // partial (max, sum)
+  off[3] = off[2] + align_up(rows * nsplit * 2 * sizeof(float));                // counters + grid word
+  off[4] = off[3] + align_up(((size_t)batch * hkv + 1) * sizeof(unsigned int)); // end
+}
 }  // namespace fc
+
+extern "C" size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
+                                                             int32_t head_dim, int32_t max_seq, int32_t max_len) {
+  if (!fused_shape_ok(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len)) return 0;
+  size_t off[5];
+  fused_layout(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len, off);
+  return off[4];
+}
+
+extern "C" int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float rms_eps, int32_t d_norm, float rope_theta,
+                                            void *kcache, void *vcache, const int32_t *kv_len, float *out, int32_t batch,
+                                            int32_t c, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
+                                            int32_t max_seq, int32_t max_len, int32_t chunks_per_cta, void *scratch,
+                                            size_t scratch_bytes, void *cuda_stream) {
+  if (!qkv_acc || !sumsq || !kcache || !vcache || !kv_len || !out || !scratch || d_norm < 1 || chunks_per_cta < 0) return FC_ERR_ARG;
+  if (!fused_shape_ok(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len)) return FC_ERR_ARG;
+  if (max_len + c > max_seq) return FC_ERR_CAPACITY;
+  if ((uintptr_t)scratch % kAlign) return FC_ERR_ARG;
+  size_t off[5];
+  fused_layout(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len, off);
+  if (scratch_bytes < off[4]) return FC_ERR_CAPACITY;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char *base = (char *)scratch;
+  // rotary table exactly as fc_init builds it
+  const int half = head_dim / 2;
+  std::vector<float2> table((size_t)max_seq * half);
+  for (int i = 0; i < half; ++i) {
+    const float inv_freq = powf(rope_theta, -2.0f * (float)i / (float)head_dim);
+    for (int pos = 0; pos < max_seq; ++pos) {
+      const float ang = (float)pos * inv_freq;
+      table[(size_t)pos * half + i] = make_float2(cosf(ang), sinf(ang));
+    }
+  }
+  if (cudaMemcpyAsync(base + off[0], table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemsetAsync(base + off[3], 0, off[4] - off[3], st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return FC_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return FC_ERR_CUDA;
+  FusedAttnArgs fa; memset(&fa, 0, sizeof fa);
+  fa.qkv = qkv_acc; fa.ldq = (n_heads + 2 * n_kv_heads) * head_dim; fa.ss = sumsq; fa.eps = rms_eps; fa.dn = d_norm;
+  fa.rope = (const float2 *)(base + off[0]);
+  fa.c_magic = (unsigned int)((0x100000000ull + (unsigned)c - 1) / (unsigned)c);
+  fa.kcache = kcache; fa.vcache = vcache;
+  fa.stride_h = (long long)max_seq * head_dim; fa.stride_b = (long long)n_kv_heads * fa.stride_h;
+  fa.kv_len = kv_len; fa.b0 = 0; fa.nb = batch; fa.c = c; fa.hq = n_heads; fa.hkv = n_kv_heads;
+  const int nsplit = (max_len + c + 127) / 128;
+  int cpc = 1, qsplit = 1;
+  fused_attn_grid(nsplit, n_heads, n_kv_heads, batch, c, sms, cpc, qsplit);
+  if (chunks_per_cta > 0) {                       // forced: several chunks per CTA need query tiles of their own
+    cpc = chunks_per_cta < nsplit ? chunks_per_cta : nsplit;
+    qsplit = cpc > 1 ? ((n_heads / n_kv_heads) * c + 15) / 16 : 1;
+  }
+  fa.cpc = cpc; fa.qsplit = qsplit; fa.nsplit = (nsplit + cpc - 1) / cpc;
+  fa.part_o = (float *)(base + off[1]); fa.part_ml = (float *)(base + off[2]);
+  fa.counters = (unsigned int *)(base + off[3]); fa.grid_counter = fa.counters + (size_t)batch * n_kv_heads;
+  fa.out = out; fa.pdl = 0;
+  if (launch_attn_fused(fa, head_dim, st) != cudaSuccess) return FC_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+}
 
 extern "C" size_t fc_op_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
                                                        int32_t head_dim, int32_t max_len, int32_t dtype) {

@@ -66,7 +66,7 @@ struct RopeArgs {
   const int32_t *kv_len;  // [batch] device
   int b0, nb, c;          // rows r = (b - b0) * c + j
   int hq, hkv, hd;
-  float theta;
+  const float2 *rope;     // [max_seq][hd/2] (cos, sin) of position * theta^(-2i/hd), built on the host
   void *q_out;            // [R, hq*hd] in the cache dtype
   void *kcache, *vcache;  // layer base; element strides below
   long long stride_b, stride_h;   // per sequence, per kv head (elements); token stride is hd
@@ -123,6 +123,7 @@ struct AcceptArgs {
   int b0, nb, c, p_stride, refill, pad_id;
   int max_tokens, eos_id;          // max_tokens <= 0: unlimited
   int commit;                      // 0: leave kv_len / n_gen / window untouched (latency measurement)
+  unsigned int *err_inject;        // test aid: when non-null the kernel raises this error word (no wait involved)
 };
 
 struct EmbedArgs {
@@ -132,6 +133,15 @@ struct EmbedArgs {
   int R, d;
   ZeroList z;
 };
+
+// Function attributes (dynamic shared memory opt-in, cluster size) are per device: launchers remember what they
+// have set per device ordinal.
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+  return dev % kMaxDevices;
+}
 
 // ---- launchers (each returns the cudaError_t of the launch) ----
 cudaError_t launch_embed(const EmbedArgs &a, int dtype, cudaStream_t st);
@@ -165,7 +175,9 @@ cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int 
 // and counts finished chunks per 128-column output tile in counter set td_prod (several projections may feed one
 // set: partial sums of the same output); td_cons: it is claimed k range by k range and stages a k-block once the
 // tile of set td_cons it reads is complete.  tile_done: zeroed words, td_stride per counter set.
-struct ChainSync { int wait_bar, sig_bar, td_prod, td_cons; };
+// epi_bar: grid barrier the projection's epilogue warps pass before their first reduction into the output (-1: none);
+// needed when the output buffer is still being read by a projection that this one does not otherwise wait for.
+struct ChainSync { int wait_bar, sig_bar, td_prod, td_cons, epi_bar; };
 constexpr int kChainMax = 6;     // projections in one chained launch
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
                               unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,

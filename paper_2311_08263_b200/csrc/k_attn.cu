@@ -481,11 +481,12 @@ static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
   if (a.cpc < 1 || (a.qsplit != 1 && a.qsplit != nqt) || (a.cpc > 1 && a.qsplit != nqt)) return cudaErrorInvalidValue;
   const size_t smem = sizeof(__nv_bfloat16) * (size_t)(2 * kChunk * LD + 2 * 16 * LD) +
                       sizeof(float) * (size_t)(4 * 16 * HD + 4 * 16 * 2);
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
+  static size_t attr_smem[kMaxDevices] = {0};
+  const int dev = current_device_slot();
+  if (smem > attr_smem[dev]) {
     cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_smem = smem;
+    attr_smem[dev] = smem;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -498,7 +499,8 @@ static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
     ++na;
   }
   // Largest cluster this kernel can be scheduled with: 16 (non-portable size) if the device takes it, else 8.
-  static int max_cluster = 0;
+  static int max_cluster_dev[kMaxDevices] = {0};
+  int &max_cluster = max_cluster_dev[dev];
   if (max_cluster == 0) {
     max_cluster = 8;
     if (cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {

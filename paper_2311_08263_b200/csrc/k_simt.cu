@@ -168,9 +168,8 @@ __global__ void rope_kv_kernel(RopeArgs a) {
     const float v0 = src[i] * s, v1 = src[i + half] * s;
     src[i] = 0.f; src[i + half] = 0.f;
     if (h < a.hq + a.hkv) {
-      const float freq = powf(a.theta, -2.0f * (float)i / (float)a.hd);
-      float sn, cs;
-      sincosf((float)pos * freq, &sn, &cs);
+      const float2 rot = a.rope[(long long)pos * half + i];     // host-built table: the device's powf is a few ulp off
+      const float cs = rot.x, sn = rot.y;
       const float o0 = v0 * cs - v1 * sn, o1 = v0 * sn + v1 * cs;
       if (h < a.hq) {
         T *dst = q_out + (long long)r * a.hq * a.hd + (long long)h * a.hd;
@@ -335,12 +334,13 @@ template <typename T, int HD, int TK>
 static cudaError_t launch_attn_t(const AttnArgs &a, cudaStream_t st) {
   constexpr int PADK = (sizeof(T) == 2) ? 2 : 1;
   size_t smem = sizeof(T) * (size_t)(TK * (HD + PADK) + TK * HD) + sizeof(float) * (8 * HD + 8 * TK);
-  static bool attr_done = false;
-  if (!attr_done) {
+  static bool attr_done[kMaxDevices] = {false};
+  const int dev = current_device_slot();
+  if (!attr_done[dev]) {
     cudaError_t e = cudaFuncSetAttribute(attn_window_kernel<T, HD, TK>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done[dev] = true;
   }
   dim3 grid(a.nsplit, a.hkv, a.nb);
   attn_window_kernel<T, HD, TK><<<grid, 256, smem, st>>>(a);
@@ -381,6 +381,7 @@ __global__ void accept_kernel(AcceptArgs a) {
       arg[j] = a.argmax[r];
     }
   }
+  if (a.err_inject && bl == 0) atomicExch(a.err_inject, 1u);
   if (a.done && a.done[b]) { a.accepted_count[b] = 0; return; }
   int k = 1;
   while (k < c && w[k] == arg[k - 1]) ++k;

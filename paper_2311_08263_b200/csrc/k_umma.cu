@@ -52,6 +52,7 @@ struct PhaseDesc {
   // 128-column output tile: the producers' epilogue warps count each finished chunk on tile_done[tile]; the consumer
   // stages k-block kb once dep_done[kb / 2] has reached dep_need.
   int wait_bar, sig_bar;
+  int epi_bar;                        // grid barrier the epilogue warps pass before their first reduction (-1: none)
   unsigned int *tile_done;
   const unsigned int *dep_done;
   unsigned int dep_need;
@@ -731,12 +732,19 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     for (int pi = 0; pi < p.n_phases && ok; ++pi) {
       const PhaseDesc &P = p.ph[pi];
       const GemmArgs &g = P.g;
+      bool epi_bar_passed = P.epi_bar < 0;
       {
         Segment s;
         int rb = 0;
         while (ok) {
           const int got = take_warp(sq, s, rb);
           if (got <= 0) { ok = got == 0; break; }
+          // the output is also the input of a projection this phase does not wait for otherwise (the residual read
+          // by the second gate/up half while the first down half is ready to add to it): its readers must be done
+          if (!epi_bar_passed) {
+            if (!grid_bar_wait(p.bar + P.epi_bar, gridDim.x, lane, abort_flag)) { ok = false; break; }
+            epi_bar_passed = true;
+          }
           int m, row0, rows_valid, ycol0;
           tile_info(P, s.tile, m, row0, rows_valid, ycol0);
           const int acc = seg & 1;
@@ -918,11 +926,12 @@ void umma_plan_destroy(UmmaPlan *p) { delete p; }
 template <int EPI, int BN, bool PANEL>
 static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid, cudaStream_t st) {
   const size_t smem = (size_t)p.stages * (kWBytes + x_parts(BN) * BN * 128) + 1024;
-  static size_t attr_smem = 0;
-  if (smem > attr_smem) {
+  static size_t attr_smem[kMaxDevices] = {0};
+  const int dev = current_device_slot();
+  if (smem > attr_smem[dev]) {
     cudaError_t e = cudaFuncSetAttribute(gemm_umma_kernel<EPI, BN, PANEL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_smem = smem;
+    attr_smem[dev] = smem;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -994,6 +1003,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.k_major = panel && !tile_mode;
     d.wait_bar = i > 0 ? i - 1 : -1;
     d.sig_bar = i + 1 < n ? i : -1;
+    d.epi_bar = -1;
     d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0; d.dep_tiles = 0;
     d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
@@ -1006,8 +1016,8 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     for (int i = 0; i < n; ++i) {
       PhaseDesc &d = p.ph[i];
       const ChainSync &c = sync[i];
-      if (c.wait_bar >= n || c.sig_bar >= n || c.td_prod > 1 || c.td_cons > 1) return cudaErrorInvalidValue;
-      d.wait_bar = c.wait_bar; d.sig_bar = c.sig_bar;
+      if (c.wait_bar >= n || c.sig_bar >= n || c.epi_bar >= n || c.td_prod > 1 || c.td_cons > 1) return cudaErrorInvalidValue;
+      d.wait_bar = c.wait_bar; d.sig_bar = c.sig_bar; d.epi_bar = c.epi_bar;
       if (c.td_prod >= 0) {          // tile-major producer: its tiles complete one after the other
         if (d.g.n_mats != 1 || d.g.y_off[0] != 0 || d.n_tiles > td_stride) return cudaErrorInvalidValue;
         d.tile_done = tile_done + (size_t)c.td_prod * td_stride;

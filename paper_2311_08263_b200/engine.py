@@ -21,6 +21,9 @@ class FcError(RuntimeError):
         super().__init__(f"{where}: {msg} ({code}) {detail}".strip())
 
 
+_GUARD, _GUARD_BYTE = 4096, 0xA5      # canary band on either side of the K/V slab and of the workspace
+
+
 def _i32(a) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
 
@@ -41,8 +44,14 @@ class Decoder:
         wsb = self.lib.fc_workspace_bytes(C.byref(self.shape))
         if kvb == 0 or wsb == 0:
             raise FcError(_l.FC_ERR_SHAPE, "fc_kv_bytes")
-        self.kv = torch.zeros(kvb, dtype=torch.uint8, device=self.device)
-        self.ws = torch.zeros(wsb, dtype=torch.uint8, device=self.device)
+        # each buffer sits between two canary bands (checked by fc_debug_check_guards)
+        self._kv_bytes, self._ws_bytes = kvb, wsb
+        self._kv_alloc = torch.full((kvb + 2 * _GUARD,), _GUARD_BYTE, dtype=torch.uint8, device=self.device)
+        self._ws_alloc = torch.full((wsb + 2 * _GUARD,), _GUARD_BYTE, dtype=torch.uint8, device=self.device)
+        self.kv = self._kv_alloc[_GUARD:_GUARD + kvb]
+        self.ws = self._ws_alloc[_GUARD:_GUARD + wsb]
+        self.kv.zero_()
+        self.ws.zero_()
         self._keep = []
 
         def dev(t: torch.Tensor) -> int:
@@ -105,14 +114,44 @@ class Decoder:
                                             cnt.ctypes.data, tok.ctypes.data, win.ctypes.data), "fc_jacobi_step")
         return cnt, tok, win
 
-    def fc_generate(self, max_tokens: int, eos_id: int = -1):
-        """Returns (tokens [B, max_tokens], lens [B], stats)."""
+    def fc_generate(self, max_tokens: int, eos_id: int = -1, c: int = 0, max_iters: int = 0):
+        """Returns (tokens [B, max_tokens], lens [B], stats).  c = 0 keeps the current window size."""
         B = self.batch
         out, lens = np.zeros((B, max_tokens), np.int32), np.zeros(B, np.int32)
         st = _l.fc_stats()
-        self._check(self.lib.fc_generate(self.h, max_tokens, eos_id, out.ctypes.data, lens.ctypes.data,
+        self._check(self.lib.fc_generate(self.h, max_tokens, c, eos_id, max_iters, out.ctypes.data, lens.ctypes.data,
                                          C.byref(st)), "fc_generate")
+        if c > 0:
+            self.c = c
         return out, lens, st
+
+    def fc_set_window(self, c: int):
+        self._check(self.lib.fc_set_window(self.h, c), "fc_set_window")
+        self.c = c
+
+    def fc_finish_with_trigger(self, trigger_ids, max_answer_tokens: int, eos_id: int = -1):
+        """Returns (answer tokens [B, max_answer_tokens], lens [B]).  The sequences need fc_prefill afterwards."""
+        B = self.batch
+        t = _i32(trigger_ids)
+        out, lens = np.zeros((B, max(max_answer_tokens, 1)), np.int32), np.zeros(B, np.int32)
+        self._check(self.lib.fc_finish_with_trigger(self.h, t.ctypes.data if t.shape[0] else None, t.shape[0],
+                                                    max_answer_tokens, eos_id, out.ctypes.data, lens.ctypes.data),
+                    "fc_finish_with_trigger")
+        return out[:, :max_answer_tokens], lens
+
+    def fc_debug_inject_timeout(self):
+        self._check(self.lib.fc_debug_inject_timeout(self.h), "fc_debug_inject_timeout")
+
+    def fc_debug_check_guards(self) -> int:
+        """Number of damaged canary bands: those between the workspace slices (kept by the library) plus the ones
+        this binding keeps around the K/V slab and the workspace."""
+        n = C.c_int32(0)
+        self._check(self.lib.fc_debug_check_guards(self.h, C.byref(n)), "fc_debug_check_guards")
+        bad = int(n.value)
+        for buf, nbytes in ((self._kv_alloc, self._kv_bytes), (self._ws_alloc, self._ws_bytes)):
+            lo, hi = buf[:_GUARD], buf[_GUARD + nbytes:]
+            bad += int((lo != _GUARD_BYTE).any().item()) + int((hi != _GUARD_BYTE).any().item())
+        return bad
 
     def fc_debug_set_state(self, kv_lens, pending, c: int, pad_id: int = 0):
         kl, pe = _i32(kv_lens), _i32(pending)
@@ -204,4 +243,26 @@ def fc_op_window_attention(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.
                                     scratch.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
     if rc != _l.FC_OK:
         raise FcError(rc, "fc_op_window_attention")
+    return out
+
+
+def fc_op_fused_window_attention(qkv_acc: torch.Tensor, sumsq: torch.Tensor, rms_eps: float, d_norm: int,
+                                 rope_theta: float, kcache: torch.Tensor, vcache: torch.Tensor, kv_len: torch.Tensor,
+                                 c: int, n_heads: int, max_len: int, chunks_per_cta: int = 0) -> torch.Tensor:
+    """The fused attention kernel of the bf16 step as one operation.  qkv_acc fp32 [B*c, (hq + 2 hkv) * hd] and sumsq
+    fp32 [B*c] are consumed (cleared); kcache/vcache bf16 [B, hkv, max_seq, hd] receive the window's rows.
+    Returns fp32 [B*c, hq*hd]."""
+    lib = _l.load()
+    B, hkv, max_seq, hd = kcache.shape
+    nbytes = lib.fc_op_fused_window_attention_scratch_bytes(B, c, n_heads, hkv, hd, max_seq, max_len)
+    if nbytes == 0:
+        raise FcError(_l.FC_ERR_ARG, "fc_op_fused_window_attention_scratch_bytes")
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=qkv_acc.device)
+    out = torch.empty(B * c, n_heads * hd, dtype=torch.float32, device=qkv_acc.device)
+    rc = lib.fc_op_fused_window_attention(qkv_acc.data_ptr(), sumsq.data_ptr(), rms_eps, d_norm, rope_theta,
+                                          kcache.data_ptr(), vcache.data_ptr(), kv_len.data_ptr(), out.data_ptr(),
+                                          B, c, n_heads, hkv, hd, max_seq, max_len, chunks_per_cta,
+                                          scratch.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
+    if rc != _l.FC_OK:
+        raise FcError(rc, "fc_op_fused_window_attention")
     return out

@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(_HERE, "libfastcot.so")
 
 FC_F32, FC_BF16 = 0, 1
 FC_REFILL_PROMPT_CYCLE, FC_REFILL_PAD = 0, 1
-FC_FLAG_SIMT_GEMM, FC_FLAG_NO_GRAPH, FC_FLAG_NO_PDL, FC_FLAG_NO_CHAIN, FC_FLAG_NO_FFN_SPLIT = 1, 2, 4, 8, 16
+FC_FLAG_SIMT_GEMM, FC_FLAG_NO_PDL, FC_FLAG_NO_CHAIN, FC_FLAG_NO_FFN_SPLIT = 1, 4, 8, 16
 FC_OK = 0
 FC_NOALLOC_SCRATCH_BYTES = 8 << 20
 FC_CLASSES = ["embed", "qkv", "rope", "attn", "oproj", "gateup", "down", "head", "accept", "chain"]
@@ -21,10 +21,12 @@ FC_ERR_ARG, FC_ERR_SHAPE, FC_ERR_CAPACITY, FC_ERR_TOKEN_RANGE = -1, -2, -3, -4
 FC_ERR_STATE, FC_ERR_BAD_WINDOW, FC_ERR_DEVICE_TIMEOUT, FC_ERR_CUDA = -5, -6, -7, -8
 
 EXPORTS = ["fc_kv_bytes", "fc_workspace_bytes", "fc_init", "fc_prefill", "fc_jacobi_step", "fc_generate",
+           "fc_set_window", "fc_finish_with_trigger", "fc_debug_inject_timeout", "fc_debug_check_guards",
            "fc_debug_set_state", "fc_debug_logits", "fc_get_state", "fc_bench_steps", "fc_profile_step",
            "fc_last_launch_count", "fc_destroy", "fc_strerror", "fc_last_cuda_error",
            "fc_op_linear", "fc_op_accept", "fc_op_window_attention",
-           "fc_op_window_attention_scratch_bytes", "fc_op_window_attention_noalloc"]
+           "fc_op_window_attention_scratch_bytes", "fc_op_window_attention_noalloc",
+           "fc_op_fused_window_attention", "fc_op_fused_window_attention_scratch_bytes"]
 
 
 class fc_model_shape(C.Structure):
@@ -70,7 +72,11 @@ def load() -> C.CDLL:
                             vp, C.c_size_t, vp, C.c_size_t, vp]
     lib.fc_prefill.argtypes = [vp, i32, i32p, i32, i32p, i32, i32, i32]
     lib.fc_jacobi_step.argtypes = [vp, i32p, i32p, i32p, i32p]
-    lib.fc_generate.argtypes = [vp, i32, i32, i32p, i32p, C.POINTER(fc_stats)]
+    lib.fc_generate.argtypes = [vp, i32, i32, i32, i32, i32p, i32p, C.POINTER(fc_stats)]
+    lib.fc_set_window.argtypes = [vp, i32]
+    lib.fc_finish_with_trigger.argtypes = [vp, i32p, i32, i32, i32, i32p, i32p]
+    lib.fc_debug_inject_timeout.argtypes = [vp]
+    lib.fc_debug_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.fc_debug_set_state.argtypes = [vp, i32, i32p, i32p, i32, i32]
     lib.fc_debug_logits.argtypes = [vp, vp]
     lib.fc_get_state.argtypes = [vp, i32p, i32p]
@@ -90,5 +96,9 @@ def load() -> C.CDLL:
     lib.fc_op_window_attention_scratch_bytes.argtypes = [i32] * 7
     lib.fc_op_window_attention.argtypes = [vp] * 5 + [i32] * 8 + [vp, C.c_size_t, vp]
     lib.fc_op_window_attention_noalloc.argtypes = [vp] * 5 + [i32] * 8 + [vp]
+    lib.fc_op_fused_window_attention_scratch_bytes.restype = C.c_size_t
+    lib.fc_op_fused_window_attention_scratch_bytes.argtypes = [i32] * 7
+    lib.fc_op_fused_window_attention.argtypes = [vp, vp, C.c_float, i32, C.c_float, vp, vp, vp, vp] + [i32] * 8 + \
+                                                [vp, C.c_size_t, vp]
     _lib = lib
     return lib

@@ -1,10 +1,20 @@
-"""Parity at the full model shapes, in the launch configuration the benchmark times.
+"""Parity at the full model shapes (1.1B, 7B, 13B x 8), in the launch configuration the benchmark times.
 
-The oracle cannot replay whole runs at these sizes in test time, so each case compares sampled outputs
-the oracle can compute one by one: the logits, accepted tokens and refreshed window of Jacobi steps, and
-(1.1B) a stretch of the committed stream from a real prefill.  For the 7B and 13B shapes the cache is filled
-with seeded random K/V (the recipe of the window-step sweep) instead of a prefill, identically on both sides.
+Two kinds of expected values:
+  * live: the CPU oracle runs beside the GPU for single steps (all logits of a step compared);
+  * stored: tests/golden/stream_<config>.json, written by tests/golden/make_streams.py from the oracle alone - the
+    first Jacobi iterations of the stated workload (window fed, accepted tokens, refreshed window, the two largest
+    logits and the logits at fixed sampled vocabulary positions of every row) and the greedy stream of gen_tokens
+    tokens with the top-1/top-2 margin at every position.  The oracle needs minutes to hours for these at 7B / 13B,
+    the GPU seconds.
+
+Bars (bf16): logits within 3e-2 max-abs of the oracle; accepted tokens, counts and windows equal wherever the
+oracle's top-1/top-2 margin of every row up to there exceeds 0.05; streams equal except at positions whose margin is
+below 0.05, after which both sides restart from the oracle's prefix.
 """
+import json
+import os
+
 import numpy as np
 import psutil
 import pytest
@@ -17,14 +27,11 @@ pytestmark = pytest.mark.gpu
 
 LOGIT_TOL = 3e-2
 MARGIN_TOL = 0.05
-# K and V are bf16 on both sides.  Two implementations whose fp32 values differ at the 1e-6 level put about one K/V
-# element in a thousand on different sides of a bf16 rounding boundary (measured at layer 0); each such element
-# is off by a whole bf16 step (0.4-0.8 %), the next layer's K/V inherit that, and by layer 2 several per cent of
-# the window's K/V elements differ by one step.  The logit difference therefore grows with depth: measured
-# max-abs 4.5e-3 at 8 layers, below 3e-2 at 22 and 32 layers, 4.3e-2 at 40 layers (rms up to 8e-3 for the sequences with almost no cache).  The 40-layer case
-# is held to twice the bar and to the rms; its argmax/accept parity is still exact wherever the margin allows.
-LOGIT_TOL_40_LAYERS = 6e-2
-LOGIT_RMS_TOL = 1.5e-2
+# K/V storage format: the oracle that keeps K and V in fp32 (kv_bf16=False) differs from the one that rounds them to
+# the model dtype where they are stored by the storage rounding alone.  The GPU stores bf16; its distance to the
+# fp32-K/V oracle is asserted below this bound (measured 0.034 at 1.1B after a real prefill, 0.056 at 7B on random K/V).
+KV_FORMAT_GAP_TOL = 0.1
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
 
 def _host_weights(w):
@@ -39,18 +46,140 @@ def _need(gpu_gb, host_gb):
         pytest.skip(f"needs {host_gb} GB of host memory for the oracle's copy of the weights")
 
 
-def _check_step(cfg, lg_gpu, lg_ref, cnt, tok, win, k_ref, acc_ref, win_ref):
+def _golden(name):
+    path = os.path.join(GOLDEN, f"stream_{name}.json")
+    if not os.path.exists(path):
+        pytest.skip(f"{path} has not been generated")
+    g = json.load(open(path))
+    if not g["sequences"]:
+        pytest.skip(f"{path} holds no finished sequence")
+    return g
+
+
+def _exact_rows(margins):
+    """Rows whose token must match: all rows before the first one with a margin at or below the tolerance."""
+    low = np.nonzero(np.asarray(margins) <= MARGIN_TOL)[0]
+    return int(low[0]) if len(low) else len(margins)
+
+
+def _check_step(lg_gpu, lg_ref, window_in, cnt, tok, win, k_ref, acc_ref, win_ref, tol=LOGIT_TOL):
+    """Logits of one step element by element; then the accept rule row by row: the GPU's greedy token of row j must
+    equal the oracle's wherever every row up to j has a margin above MARGIN_TOL, and so must everything the accept
+    rule derives from those rows.  Returns False when a low-margin row made the two sides part ways."""
     err = np.abs(lg_gpu - lg_ref)
-    assert err.max() < (LOGIT_TOL if cfg.n_layers <= 32 else LOGIT_TOL_40_LAYERS)
-    assert np.sqrt((err ** 2).mean()) < LOGIT_RMS_TOL
+    assert err.max() < tol, float(err.max())
     srt = np.sort(lg_ref, axis=1)
-    if (srt[:, -1] - srt[:, -2]).min() > MARGIN_TOL:      # otherwise a different argmax is tolerated
-        assert cnt == k_ref and tok[:cnt].tolist() == acc_ref.tolist() and win.tolist() == win_ref.tolist()
-        return True
+    n_exact = _exact_rows(srt[:, -1] - srt[:, -2])
+    c = len(window_in)
+    am_gpu, am_ref = lg_gpu.argmax(1), lg_ref.argmax(1)
+    assert am_gpu[:n_exact].tolist() == am_ref[:n_exact].tolist()
+    if n_exact >= min(k_ref + 1, c):          # every row the accept decision looked at is exact
+        assert cnt == k_ref and tok[:cnt].tolist() == acc_ref.tolist()
+        if n_exact == c:
+            assert win.tolist() == win_ref.tolist()
+        return n_exact == c
+    assert cnt >= min(n_exact, k_ref) and tok[:min(n_exact, k_ref)].tolist() == acc_ref[:min(n_exact, k_ref)].tolist()
     return False
 
 
-def test_1b_prefill_steps_and_stream():
+def _initial_windows(ids, lens, c):
+    """The windows fc_prefill builds: the prompt's last id, then the prompt's own ids from its start."""
+    B = len(lens)
+    w = np.zeros((B, c), np.int32)
+    for b in range(B):
+        p = ids[b, :lens[b]]
+        w[b, 0] = p[-1]
+        w[b, 1:] = [p[(j - 1) % len(p)] for j in range(1, c)]
+    return w
+
+
+def _check_stored_steps(dec, golden, seqs, ids, lens, c):
+    """The first stored Jacobi iterations, the GPU fed the oracle's windows: accepted tokens / count / window equal
+    (as far as margins allow), sampled logits and the two largest logits within LOGIT_TOL.  Sequences that are not
+    compared (or that left the stored trajectory at a tolerated difference) go on with their own windows."""
+    pos = golden["positions"]
+    B = len(lens)
+    logits = dec.fc_debug_logits(True)
+    alive = {b: True for b in seqs}
+    own = _initial_windows(ids, lens, c)
+    worst = 0.0
+    for i in range(golden["n_steps"]):
+        window = own.copy()
+        for b in seqs:
+            if alive[b]:
+                window[b] = golden["sequences"][b]["steps"][i]["window_in"]
+        cnt, tok, win = dec.fc_jacobi_step(window)
+        own = win
+        lg = logits[:B * c].view(B, c, -1)
+        for b in seqs:
+            if not alive[b]:
+                continue
+            st = golden["sequences"][b]["steps"][i]
+            top = torch.tensor([r["top"] for r in st["rows"]], device=lg.device)
+            got_top = torch.gather(lg[b], 1, top).cpu().numpy()
+            got_at = lg[b][:, pos].cpu().numpy()
+            want_top = np.array([r["top_v"] for r in st["rows"]])
+            want_at = np.array([r["at"] for r in st["rows"]])
+            e = max(float(np.abs(got_top - want_top).max()), float(np.abs(got_at - want_at).max()))
+            worst = max(worst, e)
+            assert e < LOGIT_TOL, (i, b, e)
+            n_exact = _exact_rows(want_top[:, 0] - want_top[:, 1])
+            am = lg[b].argmax(1).cpu().numpy()
+            assert am[:n_exact].tolist() == [r["top"][0] for r in st["rows"]][:n_exact]
+            k = st["k"]
+            if n_exact >= min(k + 1, c):
+                assert cnt[b] == k and tok[b, :k].tolist() == st["accepted"]
+            if n_exact == c:
+                assert win[b].tolist() == st["window_out"]
+            else:
+                alive[b] = False          # a tolerated difference: this sequence leaves the stored trajectory
+    dec.fc_debug_logits(False)
+    return worst
+
+
+def _check_stored_streams(dec, cfg, golden, ids, lens, seqs, c):
+    """The whole greedy stream against the stored one, restarting from the oracle's prefix after every tolerated
+    difference.  All sequences of the batch are generated together; each is checked on its own."""
+    n = golden["gen_tokens"]
+    B = len(lens)
+    pos = {b: 0 for b in seqs}
+    tolerated = 0
+    for _ in range(64):                       # restarts
+        todo = [b for b in seqs if pos[b] < n]
+        if not todo:
+            break
+        prompts = []
+        for b in range(B):
+            p = ids[b, :lens[b]].tolist()
+            if b in pos:
+                p += golden["sequences"][b]["stream"][:pos[b]]
+            prompts.append(p)
+        pl = [len(p) for p in prompts]
+        arr = np.zeros((B, max(pl)), np.int32)
+        for b, p in enumerate(prompts):
+            arr[b, :len(p)] = p
+        dec.fc_prefill(arr, pl, c)
+        want_len = max(n - pos[b] for b in todo)
+        toks, out_lens, _ = dec.fc_generate(want_len)
+        for b in todo:
+            want = np.array(golden["sequences"][b]["stream"][pos[b]:n])
+            got = toks[b, :len(want)]
+            assert out_lens[b] >= len(want)
+            diff = np.nonzero(got != want)[0]
+            if len(diff) == 0:
+                pos[b] = n
+                continue
+            i = int(diff[0])
+            m = golden["sequences"][b]["margins"][pos[b] + i]
+            assert m < MARGIN_TOL, (b, pos[b] + i, m, int(got[i]), int(want[i]))
+            tolerated += 1
+            pos[b] += i + 1
+    assert all(pos[b] >= n for b in seqs)
+    return tolerated
+
+
+# ------------------------------------------------------------------------------------------ 1.1B (cfg 2)
+def test_1b_live_steps_and_kv_format_gap():
     cfg = wl.CONFIGS["1b"]
     _need(8, 8)
     w = wl.make_weights(cfg, device="cuda")
@@ -59,28 +188,40 @@ def test_1b_prefill_steps_and_stream():
     max_seq = cfg.prompt_len + 64 + cfg.c + 8
     dec = engine.Decoder(cfg, w, 1, cfg.c, max_seq)
     o = oracle.Oracle(cfg, wh, max_seq)
+    o32 = oracle.Oracle(cfg, wh, max_seq, kv_bf16=False)        # K/V kept in fp32: the storage-format comparison
     o.prefill(prompt, cfg.c)
+    o32.prefill(prompt, cfg.c)
     dec.fc_prefill(prompt, [len(prompt)], cfg.c)
     logits = dec.fc_debug_logits(True)
+    gap = 0.0
     for _ in range(2):
         k, acc, wnew, lg = o.jacobi_step(want_logits=True)
+        _, _, _, lg32 = o32.jacobi_step(want_logits=True)
         cnt, tok, win = dec.fc_jacobi_step()
-        if not _check_step(cfg, logits[:cfg.c].cpu().numpy(), lg, cnt[0], tok[0], win[0], k, acc, wnew):
+        got = logits[:cfg.c].cpu().numpy()
+        gap = max(gap, float(np.abs(got - lg32).max()))
+        if not _check_step(got, lg, np.zeros(cfg.c), cnt[0], tok[0], win[0], k, acc, wnew):
             break
-    dec.fc_debug_logits(False)
-    # committed stream from a fresh prefill against the oracle's greedy stream
-    n = 40
-    ar, margins = oracle.Oracle(cfg, wh, max_seq).ar_generate(prompt, n)
-    dec.fc_prefill(prompt, [len(prompt)], cfg.c)
-    toks, lens, st = dec.fc_generate(n)
-    got = toks[0, :lens[0]]
-    diff = np.nonzero(got != ar)[0]
-    if len(diff):
-        assert margins[diff[0]] < MARGIN_TOL
-    assert lens[0] == n and st.tokens == n
+    assert gap < KV_FORMAT_GAP_TOL, gap
+    assert dec.fc_debug_check_guards() == 0
 
 
-def _random_kv_case(cfg, lens, c, seqs_to_check):
+def test_1b_stored_steps_and_256_token_stream():
+    cfg = wl.CONFIGS["1b"]
+    g = _golden("1b")
+    _need(8, 2)
+    w = wl.make_weights(cfg, device="cuda")
+    ids, lens = wl.make_prompts(cfg)
+    max_seq = cfg.prompt_len + cfg.gen_tokens + cfg.c + 8
+    dec = engine.Decoder(cfg, w, 1, cfg.c, max_seq)
+    dec.fc_prefill(ids.numpy(), lens.numpy(), cfg.c)
+    _check_stored_steps(dec, g, [0], ids.numpy(), lens.tolist(), cfg.c)
+    _check_stored_streams(dec, cfg, g, ids.numpy(), lens.tolist(), [0], cfg.c)
+    assert dec.fc_debug_check_guards() == 0
+
+
+# ------------------------------------------------------------------------------------------ random-K/V single steps
+def _random_kv_case(cfg, lens, c, seqs_to_check, fp32_kv_seq=None):
     """Seeded random K/V of ragged lengths on both sides, then one Jacobi step compared per sequence."""
     B = len(lens)
     w = wl.make_weights(cfg, device="cuda")
@@ -102,23 +243,30 @@ def _random_kv_case(cfg, lens, c, seqs_to_check):
     cnt, tok, win = dec.fc_jacobi_step(window)
     lg_all = logits[:B * c].cpu().numpy().reshape(B, c, cfg.vocab)
     prompt = np.array([0], np.int32)           # refill is the pad id on both sides
+    worst = 0.0
     for b in seqs_to_check:
         L = lens[b]
-        o = oracle.Oracle(cfg, wh, L + c + 8)
-        for l in range(cfg.n_layers):
-            kv = view[l, :, b, :, :L, :].float().permute(0, 2, 1, 3).reshape(2, L, kvd).cpu().numpy()
-            o.set_kv(l, kv[0], kv[1])
-        am, lg = o.forward(window[b])
-        k_ref, acc_ref, win_ref = oracle.accept(window[b], am, 0, prompt, refill=1, pad_id=0)
-        _check_step(cfg, lg_all[b], lg, cnt[b], tok[b], win[b], k_ref, acc_ref, win_ref)
-        o.close()
-    return dec
+        for kv_bf16 in ([True, False] if b == fp32_kv_seq else [True]):
+            o = oracle.Oracle(cfg, wh, L + c + 8, kv_bf16=kv_bf16)
+            for l in range(cfg.n_layers):
+                kv = view[l, :, b, :, :L, :].float().permute(0, 2, 1, 3).reshape(2, L, kvd).cpu().numpy()
+                o.set_kv(l, kv[0], kv[1])
+            am, lg = o.forward(window[b])
+            if kv_bf16:
+                k_ref, acc_ref, win_ref = oracle.accept(window[b], am, 0, prompt, refill=1, pad_id=0)
+                worst = max(worst, float(np.abs(lg_all[b] - lg).max()))
+                _check_step(lg_all[b], lg, window[b], cnt[b], tok[b], win[b], k_ref, acc_ref, win_ref)
+            else:
+                assert np.abs(lg_all[b] - lg).max() < KV_FORMAT_GAP_TOL
+            o.close()
+    assert dec.fc_debug_check_guards() == 0
+    return dec, worst
 
 
 def test_7b_step_at_bench_configuration():
     cfg = wl.CONFIGS["7b"]
     _need(20, 22)
-    dec = _random_kv_case(cfg, [cfg.prompt_len], cfg.c, [0])
+    dec, _ = _random_kv_case(cfg, [cfg.prompt_len], cfg.c, [0], fp32_kv_seq=0)
     # the step the benchmark times launches 2 * layers + 4 kernels
     assert dec.fc_last_launch_count() == 2 * cfg.n_layers + 4
 
@@ -127,7 +275,41 @@ def test_13b_batch8_ragged_step():
     cfg = wl.CONFIGS["13b"]
     _need(45, 40)
     lens = [1024, 700, 1000, 513, 1024, 64, 900, 1]
-    _random_kv_case(cfg, lens, cfg.c, [1, 5, 7])
+    _random_kv_case(cfg, lens, cfg.c, [1, 5, 7], fp32_kv_seq=5)
+
+
+# ------------------------------------------------------------------------------------------ 7B (cfg 3), 13B x 8 (cfg 4)
+def test_7b_prefill_stored_steps_and_256_token_stream():
+    """The headline configuration end to end: fc_prefill of the 800-id prompt, the first Jacobi iterations against
+    the stored oracle values, then the 256-token stream."""
+    cfg = wl.CONFIGS["7b"]
+    g = _golden("7b")
+    _need(20, 2)
+    w = wl.make_weights(cfg, device="cuda")
+    ids, lens = wl.make_prompts(cfg)
+    max_seq = cfg.prompt_len + cfg.gen_tokens + cfg.c + 8
+    dec = engine.Decoder(cfg, w, 1, cfg.c, max_seq)
+    dec.fc_prefill(ids.numpy(), lens.numpy(), cfg.c)
+    # a prompt of 800 ids is cached in blocks of 128 rows: 7 forwards of 2 * layers + 2 kernels (+ a length bump each)
+    assert dec.fc_last_launch_count() <= 8 * (2 * cfg.n_layers + 3)
+    _check_stored_steps(dec, g, [0], ids.numpy(), lens.tolist(), cfg.c)
+    _check_stored_streams(dec, cfg, g, ids.numpy(), lens.tolist(), [0], cfg.c)
+    assert dec.fc_debug_check_guards() == 0
+
+
+def test_13b_batch8_prefill_stored_steps_and_streams():
+    cfg = wl.CONFIGS["13b"]
+    g = _golden("13b")
+    _need(45, 2)
+    seqs = list(range(len(g["sequences"])))           # the sequences whose oracle run is stored
+    w = wl.make_weights(cfg, device="cuda")
+    ids, lens = wl.make_prompts(cfg)
+    max_seq = cfg.prompt_len + cfg.gen_tokens + cfg.c + 8
+    dec = engine.Decoder(cfg, w, cfg.batch, cfg.c, max_seq)
+    dec.fc_prefill(ids.numpy(), lens.numpy(), cfg.c)
+    _check_stored_steps(dec, g, seqs, ids.numpy(), lens.tolist(), cfg.c)
+    _check_stored_streams(dec, cfg, g, ids.numpy(), lens.tolist(), seqs, cfg.c)
+    assert dec.fc_debug_check_guards() == 0
 
 
 @pytest.mark.parametrize("hd,heads,kv_heads", [(64, 8, 8), (128, 4, 4), (64, 8, 2)])

@@ -290,3 +290,204 @@ def test_error_codes():
     # the failed calls left the state usable
     cnt, _, _ = dec.fc_jacobi_step()
     assert cnt[0] >= 1
+
+
+# ------------------------------------------------------------------ robustness aids in place of a memory checker
+def test_injected_device_timeout_is_reported_and_prefill_recovers():
+    """The accept kernel raises the device error word (no wait involved): the step must return
+    FC_ERR_DEVICE_TIMEOUT, further steps must be refused until fc_prefill, and after it the stream is exact again."""
+    cfg = wl.CONFIGS["tiny"]
+    w, dec, max_seq = _setup(cfg)
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    o = oracle.Oracle(cfg, w, max_seq)
+    o.prefill(prompt, cfg.c)
+    want, _ = o.generate(16)
+    dec.fc_prefill(prompt, [len(prompt)], cfg.c)
+    dec.fc_jacobi_step()
+    dec.fc_debug_inject_timeout()
+    with pytest.raises(engine.FcError) as e:
+        dec.fc_jacobi_step()
+    assert e.value.code == lib.FC_ERR_DEVICE_TIMEOUT
+    with pytest.raises(engine.FcError) as e:
+        dec.fc_jacobi_step()
+    assert e.value.code == lib.FC_ERR_STATE
+    dec.fc_prefill(prompt, [len(prompt)], cfg.c)
+    toks, lens, _ = dec.fc_generate(16)
+    assert toks[0, :lens[0]].tolist() == want.tolist()
+    assert dec.fc_debug_check_guards() == 0
+
+
+@pytest.mark.parametrize("which", ["tiny", "bf16-batch"])
+def test_canary_bands_intact_after_prefill_steps_and_generate(which):
+    """Canary bands around the K/V slab, around the workspace and between its slices must hold their pattern after
+    every kind of call (the stand-in for an out-of-bounds checker); damaging one on purpose from the host is seen."""
+    if which == "tiny":
+        cfg, B, c = wl.CONFIGS["tiny"], 1, 8
+    else:
+        cfg, B, c = wl.small_config(vocab=600, n_layers=2, n_heads=4, n_kv_heads=2, head_dim=64, d_model=256,
+                                    d_ffn=512, prompt_len=150, c=12, gen_tokens=20), 3, 12
+    w = wl.make_weights(cfg)
+    max_seq = 150 + 40 + c + 8
+    dec = engine.Decoder(cfg, w, B, c, max_seq)
+    assert dec.fc_debug_check_guards() == 0
+    lens = [min(cfg.prompt_len, 150) - 11 * b for b in range(B)]
+    ids, _ = wl.make_prompts(cfg, batch=B, lens=lens)
+    dec.fc_prefill(ids.numpy(), lens, c)
+    assert dec.fc_debug_check_guards() == 0
+    for _ in range(3):
+        dec.fc_jacobi_step()
+    dec.fc_generate(20)
+    dec.fc_bench_steps(2, commit=False)
+    dec.fc_profile_step()
+    assert dec.fc_debug_check_guards() == 0
+    dec._ws_alloc[10] = 0                    # damage the band in front of the workspace from the host
+    assert dec.fc_debug_check_guards() == 1
+
+
+# ------------------------------------------------------------------ window resize, iteration cap, continuation
+@pytest.mark.parametrize("sizes", [(8, 3, 6, 1, 5), (1, 8, 2)])
+def test_window_resize_between_iterations_matches_oracle(sizes):
+    cfg = wl.CONFIGS["tiny"]
+    w, dec, max_seq = _setup(cfg, max_c=8, max_seq=200)
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    o = oracle.Oracle(cfg, w, 200)
+    o.prefill(prompt, sizes[0])
+    dec.fc_prefill(prompt, [len(prompt)], sizes[0])
+    for i in range(20):
+        k, acc, wnew = o.jacobi_step()
+        cnt, tok, win = dec.fc_jacobi_step()
+        assert cnt[0] == k and tok[0, :k].tolist() == acc.tolist() and win[0].tolist() == wnew.tolist()
+        c_new = sizes[(i + 1) % len(sizes)]
+        o.set_window(c_new)
+        dec.fc_set_window(c_new)
+    with pytest.raises(engine.FcError) as e:
+        dec.fc_set_window(9)
+    assert e.value.code == lib.FC_ERR_CAPACITY
+
+
+def test_generate_with_window_argument_iteration_cap_and_continuation():
+    cfg = wl.CONFIGS["tiny"]
+    w, dec, max_seq = _setup(cfg, max_c=8, max_seq=200)
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    o = oracle.Oracle(cfg, w, 200)
+    o.prefill(prompt, 8)
+    dec.fc_prefill(prompt, [len(prompt)], 8)
+    # iteration cap: exactly 5 forwards, a prefix of the stream
+    want, counts = o.generate(40, max_iters=5)
+    toks, lens, st = dec.fc_generate(40, max_iters=5)
+    assert st.steps == 5 and toks[0, :lens[0]].tolist() == want.tolist()
+    # go on with another window size and a token limit, then raise the limit: the second call continues
+    o.set_window(4)
+    want2, _ = o.generate(24 - len(want))
+    toks2, lens2, st2 = dec.fc_generate(24, c=4)
+    assert toks2[0, :lens2[0]].tolist() == want2.tolist() and len(want) + lens2[0] == 24
+    want3, _ = o.generate(40 - 24)
+    toks3, lens3, _ = dec.fc_generate(40)
+    assert toks3[0, :lens3[0]].tolist() == want3.tolist() and lens3[0] == 16
+    # nothing left to do at the same limit
+    toks4, lens4, st4 = dec.fc_generate(40)
+    assert lens4[0] == 0 and st4.steps == 0
+    assert st.ms_prefill > 0
+
+
+# ------------------------------------------------------------------ answer trigger hand-off
+@pytest.mark.parametrize("n_trig,c", [(0, 1), (3, 6), (5, 8)])
+def test_finish_with_trigger_fp32_exact(n_trig, c):
+    cfg = wl.CONFIGS["tiny"]
+    w, dec, max_seq = _setup(cfg, max_c=8, max_seq=200)
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    trigger = wl.hash_uniform_int(5, 9, max(n_trig, 1), cfg.vocab).numpy()[:n_trig]
+    o = oracle.Oracle(cfg, w, 200)
+    o.prefill(prompt, c)
+    o.generate(12, max_iters=4)
+    dec.fc_prefill(prompt, [len(prompt)], c)
+    dec.fc_generate(12, max_iters=4)
+    want = o.finish_with_trigger(trigger, 10)
+    got, lens = dec.fc_finish_with_trigger(trigger, 10)
+    assert got[0, :lens[0]].tolist() == want.tolist()
+    with pytest.raises(engine.FcError) as e:
+        dec.fc_jacobi_step()
+    assert e.value.code == lib.FC_ERR_STATE
+    assert dec.fc_debug_check_guards() == 0
+
+
+def test_finish_with_trigger_bf16_batch_ragged_with_eos():
+    """Three sequences of different lengths on the tensor-core path: each answer equals the oracle's, or leaves it
+    only at a position whose margin in the oracle's greedy run over the same context is below the tolerance."""
+    cfg = wl.small_config(vocab=600, n_layers=2, n_heads=4, n_kv_heads=2, head_dim=64, d_model=256, d_ffn=512,
+                          prompt_len=70, c=6, gen_tokens=20)
+    B, lens = 3, [70, 33, 5]
+    w = wl.make_weights(cfg)
+    max_seq = 70 + 8 + 6 + 4 + 16 + 8
+    dec = engine.Decoder(cfg, w, B, cfg.c, max_seq)
+    ids, _ = wl.make_prompts(cfg, batch=B, lens=lens)
+    trigger = np.array([11, 22, 33, 44], np.int32)
+    dec.fc_prefill(ids.numpy(), lens, cfg.c)
+    dec.fc_generate(8)
+    wins = dec.fc_jacobi_step()[2]            # the windows whose approximate tokens get handed over
+    kl, ng = dec.fc_get_state()
+    got, glens = dec.fc_finish_with_trigger(trigger, 12)
+    for b in range(B):
+        o = oracle.Oracle(cfg, w, 200)
+        ar, _ = o.ar_generate(ids[b, :lens[b]].numpy(), int(ng[b]))
+        assert wins[b, 0] == ar[-1]            # the GPU's exact tokens are the oracle's so far (large margins here)
+        context = np.concatenate([ids[b, :lens[b]].numpy(), ar, wins[b, 1:], trigger]).astype(np.int32)
+        want, margins = oracle.Oracle(cfg, w, 200).ar_generate(context, 12)
+        g = got[b, :glens[b]]
+        assert glens[b] == 12
+        diff = np.nonzero(g != want)[0]
+        if len(diff):
+            assert margins[diff[0]] < MARGIN_TOL
+    # EOS cut: stop each answer just after a token taken from the first answer
+    eos = int(got[0, 3])
+    dec.fc_prefill(ids.numpy(), lens, cfg.c)
+    dec.fc_generate(8)
+    dec.fc_jacobi_step()
+    got2, glens2 = dec.fc_finish_with_trigger(trigger, 12, eos_id=eos)
+    first = int(np.where(got[0, :12] == eos)[0][0])
+    assert glens2[0] == first + 1 and got2[0, :first + 1].tolist() == got[0, :first + 1].tolist()
+
+
+# ------------------------------------------------------------------ long positions on the fp32 path
+def test_fp32_stream_exact_at_positions_in_the_thousands():
+    """Rotary angles at positions ~3000 come from the host-built table on the FMA path too: the stream stays
+    bit-exact where the device's own powf would be a few ulp off."""
+    cfg = wl.CONFIGS["tiny"]
+    P = 3000
+    w = wl.make_weights(cfg)
+    max_seq = P + 40
+    dec = engine.Decoder(cfg, w, 1, 8, max_seq)
+    prompt = wl.hash_uniform_int(cfg.seed, 21, P, cfg.vocab).numpy()
+    o = oracle.Oracle(cfg, w, max_seq)
+    o.prefill(prompt, 8)
+    want, _ = o.generate(16)
+    dec.fc_prefill(prompt, [P], 8)
+    logits = dec.fc_debug_logits(True)
+    toks, lens, _ = dec.fc_generate(16)
+    assert toks[0, :lens[0]].tolist() == want.tolist()
+
+
+# ------------------------------------------------------------------ run-to-run spread of the bf16 path
+@pytest.mark.parametrize("flags", [0, lib.FC_FLAG_NO_FFN_SPLIT], ids=["ffn-split", "ffn-unsplit"])
+def test_bf16_step_run_to_run_spread_is_bounded(flags):
+    """Partial sums are added in L2 in whatever order they arrive, so two runs of the same step differ in the last
+    bits.  The spread of the logits over repeated runs must stay two orders of magnitude under the parity tolerance
+    (a lost update or a read of a half-added residual would be far larger), with the feed-forward block run as two
+    halves and as one."""
+    cfg = wl.small_config(vocab=2000, n_layers=8, n_heads=16, n_kv_heads=4, head_dim=64, d_model=1024, d_ffn=2816,
+                          prompt_len=300, c=16, gen_tokens=8)
+    w = wl.make_weights(cfg, device="cuda")
+    prompt = wl.make_prompts(cfg)[0][0].numpy()
+    dec = engine.Decoder(cfg, w, 1, cfg.c, 400, flags=flags)
+    logits = dec.fc_debug_logits(True)
+    dec.fc_prefill(prompt, [len(prompt)], cfg.c)
+    ref = None
+    spread = 0.0
+    for _ in range(25):
+        dec.fc_bench_steps(1, commit=False)          # the same step again: nothing is committed
+        torch.cuda.synchronize()
+        lg = logits[:cfg.c].clone()
+        if ref is None:
+            ref = lg
+        spread = max(spread, float((lg - ref).abs().max()))
+    assert spread < 3e-4, spread

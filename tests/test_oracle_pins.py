@@ -320,3 +320,106 @@ def test_bf16_model_stores_kv_in_bf16_and_stays_lossless():
     o3.prefill(toks, 6)
     st, _ = o3.generate(24)
     assert np.array_equal(st, ar)
+
+
+# ---------------------------------------------------------------- iteration cap, window resize, answer trigger
+def test_iteration_cap_stops_after_max_iters():
+    """Upper bound on the iterations ("Iteration Stop Condition", condition 1): the stream produced within
+    the cap is a prefix of the greedy stream and exactly max_iters forwards ran."""
+    cfg, w, prompt = _tiny()
+    o = oracle.Oracle(cfg, w, 200)
+    ar, _ = o.ar_generate(prompt, 40)
+    o.prefill(prompt, 8)
+    toks, counts = o.generate(40, max_iters=5)
+    assert len(counts) == 5 and counts.sum() == len(toks) >= 5
+    assert toks.tolist() == ar[:len(toks)].tolist()
+    # going on without a cap completes the same stream
+    rest, _ = o.generate(40 - len(toks))
+    assert np.concatenate([toks, rest]).tolist() == ar.tolist()
+
+
+@pytest.mark.parametrize("sizes", [(8, 3, 12, 1, 5), (1, 16, 2)])
+def test_window_resize_keeps_the_stream_lossless(sizes):
+    """Changing c between iterations never changes the committed stream (it stays the greedy stream), and the
+    resized window keeps the pending token and the guesses that still fit; new slots follow the refill rule."""
+    cfg, w, prompt = _tiny()
+    o = oracle.Oracle(cfg, w, 240)
+    ar, _ = o.ar_generate(prompt, 60)
+    o.prefill(prompt, sizes[0])
+    got = []
+    for i in range(30):
+        c_old = o.c
+        k, acc, wnew = o.jacobi_step()
+        got += acc.tolist()
+        c_new = sizes[(i + 1) % len(sizes)]
+        o.set_window(c_new)
+        # probe the resized window through a step that feeds it back unchanged: window_in must be accepted
+        # (slot 0 is the pending token), and the kept part is the old window's head
+        keep = min(c_old, c_new)
+        want_w = wnew[:keep].tolist() + [int(prompt[(o.n_gen + j - 1) % len(prompt)]) for j in range(keep, c_new)]
+        k2, acc2, _ = o.jacobi_step(np.array(want_w, np.int32))
+        got += acc2.tolist()
+        if len(got) >= 60:
+            break
+    assert got[:60] == ar[:len(got[:60])].tolist()
+
+
+def test_window_resize_guess_positions():
+    """A guess kept across a resize still refers to the same generated index: prime slot 1..m with the greedy
+    continuation, shrink and grow the window, and the next step must still accept exactly those."""
+    cfg, w, prompt = _tiny()
+    o = oracle.Oracle(cfg, w, 200)
+    ar, _ = o.ar_generate(prompt, 20)
+    o.prefill(prompt, 8)
+    win = np.zeros(8, np.int32)
+    win[0] = prompt[-1]
+    win[1:4] = ar[:3]
+    win[4] = (ar[3] + 1) % cfg.vocab
+    o2 = oracle.Oracle(cfg, w, 200)
+    o2.prefill(prompt, 8)
+    # o: plain step with the primed window -> k = 4
+    k, acc, _ = o.jacobi_step(win)
+    assert k == 4 and acc.tolist() == ar[:4].tolist()
+    # o2: window of 3 rows holding the first two primed guesses -> k = 3 (all guesses right)
+    o2.set_window(3)
+    k, acc, wn = o2.jacobi_step(win[:3])
+    assert k == 3 and acc.tolist() == ar[:3].tolist() and wn[0] == ar[2]
+
+
+@pytest.mark.parametrize("n_trig,c", [(0, 1), (3, 6), (5, 1), (1, 8)])
+def test_answer_trigger_equals_greedy_on_the_concatenated_context(n_trig, c):
+    """Hand-off ("Overview of FastCoT", "Trigger Answer"): the answer decoded after prompt + exact tokens +
+    approximate tokens + trigger equals plain greedy decoding (Eq. 1) of that concatenation."""
+    cfg, w, prompt = _tiny()
+    trigger = wl.hash_uniform_int(5, 9, max(n_trig, 1), cfg.vocab).numpy()[:n_trig]
+    o = oracle.Oracle(cfg, w, 200)
+    o.prefill(prompt, c)
+    emitted, _ = o.generate(12, max_iters=4)
+    _, _, window = o.jacobi_step()          # one more step so that the window holds real approximate tokens
+    # context = prompt | all exact tokens | approximate tokens | trigger  (window[0] is the last exact token)
+    o_ref = oracle.Oracle(cfg, w, 200)
+    ar, _ = o_ref.ar_generate(prompt, 40)
+    n_exact = o.n_gen
+    context = np.concatenate([prompt, ar[:n_exact], window[1:], trigger]).astype(np.int32)
+    assert window[0] == ar[n_exact - 1]
+    want, _ = oracle.Oracle(cfg, w, 300).ar_generate(context, 10)
+    got = o.finish_with_trigger(trigger, 10)
+    assert got.tolist() == want.tolist()
+    with pytest.raises(RuntimeError):
+        o.jacobi_step()                      # the Jacobi state was consumed
+
+
+def test_answer_trigger_empty_with_c1_is_plain_continuation_and_eos_cut():
+    cfg, w, prompt = _tiny()
+    ar, _ = oracle.Oracle(cfg, w, 200).ar_generate(prompt, 30)
+    o = oracle.Oracle(cfg, w, 200)
+    o.prefill(prompt, 1)
+    o.generate(6)
+    got = o.finish_with_trigger([], 20)
+    assert got.tolist() == ar[6:26].tolist()
+    o.prefill(prompt, 1)
+    o.generate(6)
+    eos = int(ar[10])
+    first = 6 + int(np.where(ar[6:] == eos)[0][0])
+    got = o.finish_with_trigger([], 20, eos_id=eos)
+    assert got.tolist() == ar[6:first + 1].tolist()
