@@ -82,8 +82,10 @@ def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, cpc):
         # the window's K/V rows as stored: within one bf16 step of the oracle's, nearly all identical
         for got_t, want in ((kcd, want_k[b]), (vcd, want_v[b])):
             got = got_t[b, :, L:L + c].float().cpu().transpose(0, 1).reshape(c, hkv * hd).numpy()
-            step = np.maximum(np.abs(want), 1e-30) * 2.0 ** -7       # one step of an 8-bit significand, at most
-            assert (np.abs(got - want) <= step).all()
+            # one step of an 8-bit significand at most; elements that are small through cancellation carry the fp32
+            # summation-order difference of their 256 terms instead (absolute, ~1e-6)
+            step = np.maximum(np.abs(want) * 2.0 ** -7, 1e-5)
+            assert (np.abs(got - want) <= step).all(), float((np.abs(got - want) - step).max())
             assert (got != want).mean() < 0.01
         vmax = max(float(np.abs(want_v[b]).max()), float(vc[b].abs().max()))
         err = np.abs(out[b] - want_attn[b])
