@@ -215,14 +215,17 @@ int fc_op_window_attention(const void *q, const void *kcache, const void *vcache
  * rows as bf16 at cache slots kv_len[b] .. kv_len[b]+c-1, and computes the window attention of Eq. 4's forward as
  * fc_op_window_attention does.  qkv_acc: fp32 [batch*c, (n_heads + 2 n_kv_heads) * head_dim] = (q | k | v), cleared by
  * the call; sumsq: fp32 [batch*c], cleared by the call; kcache/vcache: bf16 [batch][n_kv_heads][max_seq][head_dim],
- * in/out; out: fp32 [batch*c, n_heads*head_dim].  chunks_per_cta: 0 = the grid fc_jacobi_step would choose, > 0 forces
- * that many 128-key chunks per CTA.  scratch: device, 256-byte aligned, >= ..._scratch_bytes(...). */
+ * in/out, 16-byte aligned (cached K/V tiles are fetched by TMA); out: fp32 [batch*c, n_heads*head_dim].  c <= 128.
+ * n_splits: 0 = the grid fc_jacobi_step would choose, 1..8 forces that many CTAs (one thread-block cluster) per
+ * (sequence, kv head, group of query tiles), each over a run of consecutive 64-key tiles.  scratch: device, 256-byte
+ * aligned, >= ..._scratch_bytes(...) (rotary table and an error word).  Returns FC_ERR_DEVICE_TIMEOUT when a bounded
+ * wait inside the kernel gave up. */
 size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
                                                   int32_t head_dim, int32_t max_seq, int32_t max_len);
 int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float rms_eps, int32_t d_norm, float rope_theta,
                                  void *kcache, void *vcache, const int32_t *kv_len, float *out, int32_t batch,
                                  int32_t c, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_seq,
-                                 int32_t max_len, int32_t chunks_per_cta, void *scratch, size_t scratch_bytes,
+                                 int32_t max_len, int32_t n_splits, void *scratch, size_t scratch_bytes,
                                  void *cuda_stream);
 
 /* The same window attention for callers that may not allocate device memory (the paper has no

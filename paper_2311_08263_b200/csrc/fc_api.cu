@@ -143,6 +143,7 @@ struct fc_ctx {
   bool pdl;          // chain the tensor-core kernels by programmatic dependent launch
   bool chain;        // run O -> gate/up -> down -> next layer's QKV as one launch with grid barriers
   bool fused_attn;   // bf16 with head_dim 64/128: rotary embedding and K/V write happen inside the attention kernel
+  KvTensorMap kv_map; // TMA view of the whole K/V slab: (head_dim, max_seq, layers * 2 * max_batch * kv heads)
   int n_sms;
   std::vector<UmmaPlan *> plan_qkv, plan_o, plan_gu, plan_down;
   std::vector<UmmaPlan *> plan_gu_half[2], plan_down_half[2];   // the FFN in two halves of d_ffn (chained launch, <= 16 rows)
@@ -359,6 +360,12 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
     if (rc == FC_OK && !(ctx->plan_head = umma_plan_create(args_head(ctx), PRO_GAIN, EPI_ARGMAX, ctx->n_sms, ctx->b.err, msg, sizeof msg))) rc = FC_ERR_CUDA;
     if (rc != FC_OK) { fprintf(stderr, "fc_init: %s\n", msg); return fail(rc); }
   }
+  if (ctx->fused_attn &&
+      make_kv_tensor_map(&ctx->kv_map, kv, shape->head_dim, shape->max_seq,
+                         (long long)L * 2 * shape->max_batch * shape->n_kv_heads) != cudaSuccess) {
+    fprintf(stderr, "fc_init: tensor map over the K/V slab could not be encoded\n");
+    return fail(FC_ERR_CUDA);
+  }
   const size_t pin_ints = (size_t)shape->max_batch * (1 + 2 * shape->max_c) + 4;
   if (cudaMallocHost((void **)&ctx->pin, pin_ints * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaEventCreate(&ctx->ev0) != cudaSuccess || cudaEventCreate(&ctx->ev1) != cudaSuccess) return fail(FC_ERR_CUDA);
@@ -389,20 +396,6 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   return FC_OK;
 }
 
-// Grid of the fused attention kernel: one CTA per 128-key chunk while all of them are resident at once (two per
-// SM); beyond, a CTA walks over cpc consecutive chunks and every 16-row query tile has CTAs of its own.
-static void fused_attn_grid(int nsplit, int hq, int hkv, int nb, int rows, int n_sms, int &cpc, int &qsplit) {
-  cpc = 1; qsplit = 1;
-  const int nqt = ((hq / hkv) * rows + 15) / 16;
-  const long long per_split = (long long)hkv * nb;
-  if ((long long)nsplit * per_split > 2ll * n_sms) {          // more CTAs than are resident at once
-    long long groups = 2ll * n_sms / (per_split * nqt);       // as many CTAs as are resident at once, not more
-    if (groups < 1) groups = 1;
-    cpc = (int)((nsplit + groups - 1) / groups);
-    if (cpc > 1) qsplit = nqt;
-  }
-}
-
 static void prof_mark(fc_ctx *ctx, int cls, bool begin) {
   if (!ctx->prof) return;
   cudaEvent_t e;
@@ -429,11 +422,11 @@ static unsigned int *claim_word(fc_ctx *ctx, int l, int which) {
 }
 
 static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R, int pro, int epi, int cls,
-                            unsigned int *claim) {
+                            unsigned int *claim, const ZeroList *zero = nullptr) {
   ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
-  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + (kSyncPanel - kSyncClaim), ctx->pdl && !ctx->prof, ctx->st);   // panel-ready word
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + (kSyncPanel - kSyncClaim), zero, ctx->pdl && !ctx->prof, ctx->st);   // panel-ready word
   return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
 }
 
@@ -469,21 +462,15 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       fa.qkv = ctx->b.qkv; fa.ldq = d.ldq; fa.ss = ctx->b.ss_attn; fa.eps = s.rms_eps; fa.dn = s.d_model;
       fa.rope = ctx->b.rope; fa.c_magic = (unsigned int)((0x100000000ull + (unsigned)rows - 1) / (unsigned)rows);
       fa.kcache = kc; fa.vcache = vc; fa.stride_b = stride_b; fa.stride_h = stride_h;
+      fa.k_plane0 = (l * 2) * s.max_batch * s.n_kv_heads; fa.v_plane0 = (l * 2 + 1) * s.max_batch * s.n_kv_heads;
       fa.kv_len = ctx->b.kv_len; fa.b0 = b0; fa.nb = nb; fa.c = rows; fa.hq = s.n_heads; fa.hkv = s.n_kv_heads;
-      // One CTA per 128-key chunk while all of them are resident at once (two per SM); beyond, a CTA walks over
-      // several consecutive chunks, so that the queries are staged and the partial result is written once per CTA
-      // (every 16-row query tile then has CTAs of its own).
-      int cpc = 1, qsplit = 1;
-      fused_attn_grid(nsplit, s.n_heads, s.n_kv_heads, nb, rows, ctx->n_sms, cpc, qsplit);
-      fa.qsplit = qsplit;
-      fa.cpc = cpc;
-      fa.nsplit = (nsplit + cpc - 1) / cpc; fa.part_o = ctx->b.part_o; fa.part_ml = ctx->b.part_ml; fa.counters = ctx->b.counters;
-      fa.grid_counter = ctx->b.counters + (size_t)s.max_batch * s.n_kv_heads;
+      fused_attn_plan(max_len_host, rows, s.n_heads, s.n_kv_heads, nb, ctx->n_sms, fa.nsplit, fa.qt);
+      fa.err = ctx->b.err;
       fa.out = ctx->b.attn; fa.pdl = ctx->pdl && !ctx->prof;
       fa.z.p[0] = ctx->b.gu; fa.z.n[0] = Rz * 2 * s.d_ffn;
       fa.z.p[1] = ctx->b.ss_ffn; fa.z.n[1] = Rz;
       ++ctx->launches;
-      { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn_fused(fa, s.head_dim, ctx->st)); }
+      { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn_fused(ctx->kv_map, ctx->kv_map, fa, s.head_dim, ctx->st)); }
     } else {
       RopeArgs ra; memset(&ra, 0, sizeof ra);
       ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
@@ -504,6 +491,12 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ++ctx->launches;
       { ProfScope ps(ctx, FC_CLS_ATTN); FC_CK(launch_attn(aa, s.dtype, s.head_dim, ctx->st)); }
     }
+    // The fused attention kernel only reads the QKV accumulators and the sums of squares of the attention norm; the
+    // projection launch that follows it clears them (its next-QKV phase, or the next QKV launch, accumulates again).
+    ZeroList zl; memset(&zl, 0, sizeof zl);
+    zl.p[0] = ctx->b.qkv; zl.n[0] = Rz * d.ldq;
+    zl.p[1] = ctx->b.ss_attn; zl.n[1] = Rz;
+    const ZeroList *zero = ctx->fused_attn ? &zl : nullptr;
     if (chained) {
       // O projection, gate/up, down and the next layer's QKV: one persistent launch.
       // Up to 16 rows the phases are tied together without a stall where the data allow it (see ChainSync): gate/up
@@ -533,9 +526,9 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ProfScope ps(ctx, FC_CLS_CHAIN);
       unsigned int *grp = ctx->b.chain_bar + (size_t)l * d.sync_words;
       FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + kSyncClaim, grp + kSyncPanel, R <= 16 ? sy : nullptr, grp + kSyncTd,
-                              (s.d_model + 127) / 128, ctx->pdl && !ctx->prof, ctx->st));
+                              (s.d_model + 127) / 128, zero, ctx->pdl && !ctx->prof, ctx->st));
     } else {
-      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O)));
+      FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O), zero));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_down[l] : nullptr, args_down(ctx, l), R, PRO_SILU_MUL, EPI_ATOMIC_ADD, FC_CLS_DOWN, claim_word(ctx, l, GEMM_DOWN)));
     }
@@ -563,6 +556,14 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     }
   }
   return FC_OK;
+}
+
+// Rows of one forward while tokens are only cached (prompt, answer-trigger context): what the activation buffers
+// hold, and no more than the fused attention kernel takes as one window.
+static int block_rows(const fc_ctx *ctx) {
+  int r = ctx->d.rows_ws;
+  if (ctx->fused_attn && r > attn_fused_max_rows()) r = attn_fused_max_rows();
+  return r;
 }
 
 static int check_device_error(fc_ctx *ctx) {
@@ -621,8 +622,9 @@ extern "C" int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids,
   FC_CK(cudaEventRecord(ctx->ev0, ctx->st));
   for (int b = 0; b < batch; ++b) {
     const int n = prompt_lens[b] - 1;
-    for (int start = 0; start < n; start += ctx->d.rows_ws) {
-      const int rows = n - start < ctx->d.rows_ws ? n - start : ctx->d.rows_ws;
+    const int blk = block_rows(ctx);
+    for (int start = 0; start < n; start += blk) {
+      const int rows = n - start < blk ? n - start : blk;
       int rc = forward(ctx, b, 1, rows, ctx->b.prompt + (size_t)b * s.max_seq + start, false, start, 1);
       if (rc != FC_OK) return rc;
     }
@@ -811,8 +813,9 @@ extern "C" int fc_finish_with_trigger(fc_ctx *ctx, const int32_t *trigger_ids, i
   // (1) commit K/V of every context row but the last, in blocks of rows; sequences one at a time (ragged lengths)
   const int n_commit = n_ctx - 1;
   for (int b = 0; b < B && n_commit > 0; ++b) {
-    for (int start = 0; start < n_commit; start += ctx->d.rows_ws) {
-      const int rows = n_commit - start < ctx->d.rows_ws ? n_commit - start : ctx->d.rows_ws;
+    const int blk = block_rows(ctx);
+    for (int start = 0; start < n_commit; start += blk) {
+      const int rows = n_commit - start < blk ? n_commit - start : blk;
       FC_CK(cudaMemcpyAsync(ctx->b.row_tokens, rows_h.data() + (size_t)b * n_ctx + start, sizeof(int32_t) * rows,
                             cudaMemcpyHostToDevice, ctx->st));
       int rc = forward(ctx, b, 1, rows, ctx->b.row_tokens, false, ctx->kv_len_h[b] + start, 1);
@@ -1009,7 +1012,7 @@ extern "C" int fc_op_linear(const float *x, const void *w, float *y, int32_t R, 
   char msg[200];
   UmmaPlan *pl = umma_plan_create(a, PRO_NONE, EPI_ATOMIC_ADD, sms, err_word, msg, sizeof msg);
   if (!pl) { fprintf(stderr, "fc_op_linear: %s\n", msg); return FC_ERR_CUDA; }
-  cudaError_t e = launch_gemm_umma(pl, a, err_word + 1, nullptr, 0, st);
+  cudaError_t e = launch_gemm_umma(pl, a, err_word + 1, nullptr, nullptr, 0, st);
   unsigned int herr = 0;
   if (e == cudaSuccess) e = cudaMemcpyAsync(&herr, err_word, sizeof herr, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -1077,40 +1080,36 @@ int run_window_attention(const void *q, const void *kcache, const void *vcache, 
 
 // ---- the fused kernel of the bf16 step (1/rms + rotary embedding + K/V write + window attention) as one operation
 static bool fused_shape_ok(int batch, int c, int hq, int hkv, int hd, int max_seq, int max_len) {
-  return batch >= 1 && c >= 1 && hq >= 1 && hkv >= 1 && hq % hkv == 0 && (hd == 64 || hd == 128) && max_len >= 0 &&
-         max_seq >= 1;
+  return batch >= 1 && c >= 1 && c <= attn_fused_max_rows() && hq >= 1 && hkv >= 1 && hq % hkv == 0 &&
+         (hd == 64 || hd == 128) && max_len >= 0 && max_seq >= 1;
 }
-static void fused_layout(int batch, int c, int hq, int hkv, int hd, int max_seq, int max_len, size_t off[5]) {
-  const size_t nsplit = (size_t)(max_len + c + 127) / 128;
-  const size_t rows = (size_t)batch * c * hq;
+static void fused_layout(int hd, int max_seq, size_t off[3]) {
   off[0] = 0;                                                                   // rope table
-  off[1] = off[0] + align_up((size_t)max_seq * (hd / 2) * sizeof(float2));      // partial outputs
-  off[2] = off[1] + align_up(rows * nsplit * hd * sizeof(float));               // partial (max, sum)
-  off[3] = off[2] + align_up(rows * nsplit * 2 * sizeof(float));                // counters + grid word
-  off[4] = off[3] + align_up(((size_t)batch * hkv + 1) * sizeof(unsigned int)); // end
+  off[1] = off[0] + align_up((size_t)max_seq * (hd / 2) * sizeof(float2));      // error word
+  off[2] = off[1] + align_up(sizeof(unsigned int));                             // end
 }
 }  // namespace fc
 
 extern "C" size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
                                                              int32_t head_dim, int32_t max_seq, int32_t max_len) {
   if (!fused_shape_ok(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len)) return 0;
-  size_t off[5];
-  fused_layout(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len, off);
-  return off[4];
+  size_t off[3];
+  fused_layout(head_dim, max_seq, off);
+  return off[2];
 }
 
 extern "C" int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float rms_eps, int32_t d_norm, float rope_theta,
                                             void *kcache, void *vcache, const int32_t *kv_len, float *out, int32_t batch,
                                             int32_t c, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
-                                            int32_t max_seq, int32_t max_len, int32_t chunks_per_cta, void *scratch,
+                                            int32_t max_seq, int32_t max_len, int32_t n_splits, void *scratch,
                                             size_t scratch_bytes, void *cuda_stream) {
-  if (!qkv_acc || !sumsq || !kcache || !vcache || !kv_len || !out || !scratch || d_norm < 1 || chunks_per_cta < 0) return FC_ERR_ARG;
+  if (!qkv_acc || !sumsq || !kcache || !vcache || !kv_len || !out || !scratch || d_norm < 1 || n_splits < 0 || n_splits > 8) return FC_ERR_ARG;
   if (!fused_shape_ok(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len)) return FC_ERR_ARG;
   if (max_len + c > max_seq) return FC_ERR_CAPACITY;
-  if ((uintptr_t)scratch % kAlign) return FC_ERR_ARG;
-  size_t off[5];
-  fused_layout(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len, off);
-  if (scratch_bytes < off[4]) return FC_ERR_CAPACITY;
+  if ((uintptr_t)scratch % kAlign || ((uintptr_t)kcache | (uintptr_t)vcache) % 16) return FC_ERR_ARG;
+  size_t off[3];
+  fused_layout(head_dim, max_seq, off);
+  if (scratch_bytes < off[2]) return FC_ERR_CAPACITY;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   char *base = (char *)scratch;
   // rotary table exactly as fc_init builds it
@@ -1124,31 +1123,35 @@ extern "C" int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float 
     }
   }
   if (cudaMemcpyAsync(base + off[0], table.data(), table.size() * sizeof(float2), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemsetAsync(base + off[3], 0, off[4] - off[3], st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+      cudaMemsetAsync(base + off[1], 0, off[2] - off[1], st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
     return FC_ERR_CUDA;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return FC_ERR_CUDA;
+  KvTensorMap kmap, vmap;
+  const long long planes = (long long)batch * n_kv_heads;
+  if (make_kv_tensor_map(&kmap, kcache, head_dim, max_seq, planes) != cudaSuccess ||
+      make_kv_tensor_map(&vmap, vcache, head_dim, max_seq, planes) != cudaSuccess) return FC_ERR_CUDA;
   FusedAttnArgs fa; memset(&fa, 0, sizeof fa);
   fa.qkv = qkv_acc; fa.ldq = (n_heads + 2 * n_kv_heads) * head_dim; fa.ss = sumsq; fa.eps = rms_eps; fa.dn = d_norm;
   fa.rope = (const float2 *)(base + off[0]);
   fa.c_magic = (unsigned int)((0x100000000ull + (unsigned)c - 1) / (unsigned)c);
   fa.kcache = kcache; fa.vcache = vcache;
   fa.stride_h = (long long)max_seq * head_dim; fa.stride_b = (long long)n_kv_heads * fa.stride_h;
+  fa.k_plane0 = 0; fa.v_plane0 = 0;
   fa.kv_len = kv_len; fa.b0 = 0; fa.nb = batch; fa.c = c; fa.hq = n_heads; fa.hkv = n_kv_heads;
-  const int nsplit = (max_len + c + 127) / 128;
-  int cpc = 1, qsplit = 1;
-  fused_attn_grid(nsplit, n_heads, n_kv_heads, batch, c, sms, cpc, qsplit);
-  if (chunks_per_cta > 0) {                       // forced: several chunks per CTA need query tiles of their own
-    cpc = chunks_per_cta < nsplit ? chunks_per_cta : nsplit;
-    qsplit = cpc > 1 ? ((n_heads / n_kv_heads) * c + 15) / 16 : 1;
-  }
-  fa.cpc = cpc; fa.qsplit = qsplit; fa.nsplit = (nsplit + cpc - 1) / cpc;
-  fa.part_o = (float *)(base + off[1]); fa.part_ml = (float *)(base + off[2]);
-  fa.counters = (unsigned int *)(base + off[3]); fa.grid_counter = fa.counters + (size_t)batch * n_kv_heads;
+  fused_attn_plan(max_len, c, n_heads, n_kv_heads, batch, sms, fa.nsplit, fa.qt);
+  if (n_splits > 0) fa.nsplit = n_splits;
+  fa.err = (unsigned int *)(base + off[1]);
   fa.out = out; fa.pdl = 0;
-  if (launch_attn_fused(fa, head_dim, st) != cudaSuccess) return FC_ERR_CUDA;
-  return cudaStreamSynchronize(st) == cudaSuccess ? FC_OK : FC_ERR_CUDA;
+  if (launch_attn_fused(kmap, vmap, fa, head_dim, st) != cudaSuccess) return FC_ERR_CUDA;
+  // inside a step the projection launch that follows clears the accumulators; here the call does it
+  unsigned int herr = 0;
+  if (cudaMemsetAsync(qkv_acc, 0, (size_t)batch * c * fa.ldq * sizeof(float), st) != cudaSuccess ||
+      cudaMemsetAsync(sumsq, 0, (size_t)batch * c * sizeof(float), st) != cudaSuccess ||
+      cudaMemcpyAsync(&herr, fa.err, sizeof herr, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) return FC_ERR_CUDA;
+  return herr ? FC_ERR_DEVICE_TIMEOUT : FC_OK;
 }
 
 extern "C" size_t fc_op_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,

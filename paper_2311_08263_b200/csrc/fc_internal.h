@@ -87,25 +87,25 @@ struct AttnArgs {
   ZeroList z;
 };
 
+struct KvTensorMap { alignas(64) unsigned char opaque[128]; };   // storage of one TMA tensor map (CUtensorMap)
+
 struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attention in one kernel
-  float *qkv;             // [R, ldq] fp32 accumulators (q | k | v) lacking 1/rms; cleared by the kernel
+  const float *qkv;       // [R, ldq] fp32 accumulators (q | k | v) lacking 1/rms; read only
   int ldq;
-  float *ss;              // [R] sums of squares for 1/rms; cleared by the kernel
+  const float *ss;        // [R] sums of squares for 1/rms; read only
   float eps; int dn;
   const float2 *rope;     // [max_seq][hd/2] (cos, sin) of position * theta^(-2i/hd)
   unsigned int c_magic;   // ceil(2^32 / c): q / c == umulhi(q, c_magic) for the small q used here
-  void *kcache, *vcache;
-  long long stride_b, stride_h;
+  void *kcache, *vcache;  // layer base (the window's own rows are stored through these)
+  long long stride_b, stride_h;   // per sequence, per kv head (elements); stride_b == hkv * stride_h
+  int k_plane0, v_plane0; // plane (= [max_seq][hd] matrix of one sequence and kv head) of sequence 0, kv head 0 in the
+                          // K and the V tensor map: cached tiles are fetched by TMA from plane0 + b * hkv + kvh
   const int32_t *kv_len;
   int b0, nb, c, hq, hkv;
-  int nsplit;             // CTAs per (sequence, kv head); nsplit * cpc 128-key chunks cover max(kv_len) + c
-  int cpc;                // consecutive chunks per CTA
-  int qsplit;             // 1, or the number of 16-row query tiles per kv head: then every tile has CTAs of its own (needed for cpc > 1)
-  float *part_o, *part_ml;
-  unsigned int *counters; // [batch*hkv], zero on entry and on exit
-  unsigned int *grid_counter;   // one word, zero on entry and on exit
+  int nsplit;             // CTAs (one thread-block cluster, <= 8) per (sequence, kv head, query-tile group)
+  int qt;                 // 16-row query tiles per CTA: 1, 2 or 4
   int pdl;                // launched as a programmatic dependent of the previous kernel
-  int cluster;            // set by the launcher: the nsplit CTAs of one kv head form one thread-block cluster
+  unsigned int *err;      // device error word, raised when a bounded wait gives up
   float *out;             // [R, hq*hd] fp32
   ZeroList z;
 };
@@ -148,7 +148,12 @@ cudaError_t launch_embed(const EmbedArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_gemm_simt(const GemmArgs &a, int dtype, int pro, int epi, cudaStream_t st);
 cudaError_t launch_rope_kv(const RopeArgs &a, int dtype, cudaStream_t st);
 cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st);
-cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st);
+cudaError_t launch_attn_fused(const KvTensorMap &kmap, const KvTensorMap &vmap, const FusedAttnArgs &a, int hd, cudaStream_t st);
+// 3-d tensor map (head_dim, max_seq, planes) over bf16 K or V planes laid out [plane][max_seq][head_dim] from `base`.
+cudaError_t make_kv_tensor_map(KvTensorMap *out, const void *base, int hd, int max_seq, long long planes);
+// Grid of the fused attention kernel: splits per (sequence, kv head, query-tile group) and query tiles per CTA.
+void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int &nsplit, int &qt);
+int attn_fused_max_rows();   // most window rows per sequence the fused kernel takes in one launch
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 int attn_tile_keys(int dtype, int hd);   // keys per split tile
 
@@ -165,8 +170,10 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
 void umma_plan_destroy(UmmaPlan *p);
 // x/x2/y/ss pointers and R may differ per launch from those the plan was created with.
 // claim: one zeroed word per projection of the launch (the work-claim counters).
-cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b, int pdl,
-                             cudaStream_t st);
+// zero (optional): buffers the launch clears at its start, once the previous kernel is complete; only for buffers that
+// nothing reads before a later kernel or a phase behind a grid barrier of this launch accumulates into them.
+cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b,
+                             const ZeroList *zero, int pdl, cudaStream_t st);
 // Up to four projections in one launch, each consuming the previous one's reduced output; bar: n-1 zeroed words.
 // bar_b: n zeroed words (panel-ready barriers), needed when the rows exceed 16 and the plans have panels.
 // sync (optional, used up to 16 rows): how each projection is tied to the others, instead of a grid barrier
@@ -181,6 +188,6 @@ struct ChainSync { int wait_bar, sig_bar, td_prod, td_cons, epi_bar; };
 constexpr int kChainMax = 6;     // projections in one chained launch
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
                               unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,
-                              int td_stride, int pdl, cudaStream_t st);
+                              int td_stride, const ZeroList *zero, int pdl, cudaStream_t st);
 
 }  // namespace fc

@@ -1,17 +1,29 @@
 // Fused rotary embedding + in-place K/V write + split-KV window attention for bf16 (head_dim 64/128).
 //
-// grid (splits, kv heads, sequences); one CTA owns a run of consecutive 128-key chunks (one chunk when the problem is
-// small, several - with running softmax statistics - when there are more chunks than the GPU
-// holds CTAs) of one kv head of one sequence.
-// It stages a chunk's K and V in shared memory - cached keys by 16-byte copies; the window's own keys
-// (slots kv_len .. kv_len+c-1) straight from the fp32 QKV accumulators with the deferred 1/rms factor and
-// the rotation applied, writing them to the cache on the way (each window key has exactly one owner CTA).
-// Then, for every 16-row tile of the queries that map to this kv head (group heads x c window rows), the
-// four warps each take 32 keys: S = Q.K^T and P.V run on mma.sync m16n8k16 (bf16 in, fp32 accumulate),
-// softmax statistics by warp shuffles, the four warps are merged through shared memory and one partial
-// (max, sum, out) per (row, head, split) goes to scratch.  The last CTA of a (sequence, kv head) merges the
-// splits and clears the accumulators it owns; the last CTA of the grid clears the per-row sums of squares.
+// grid (splits, kv heads x query-tile groups, sequences); the splits of one (sequence, kv head, query-tile group)
+// form one thread-block cluster (at most 8).  A CTA owns a run of consecutive 64-key tiles of the cached keys of its
+// kv head and QT 16-row tiles of the queries that map to that kv head (group heads x c window rows).
+//   - Cached K/V tiles arrive by TMA (one 3-d tensor map over the K/V slab, boxes of 64 keys x 64 elements, 128-byte
+//     swizzle) into a ring of NS stages; the first NS tiles are requested before the kernel waits for the QKV
+//     projection, because cached keys were written by earlier steps.  No stage has a consumer barrier: a stage is
+//     free again when every warp has passed the next tile's first CTA barrier, and thread 0 refills it there.
+//   - The last split also owns the window's own keys (slots kv_len .. kv_len+c-1): it takes them straight from the
+//     fp32 QKV accumulators, applies the deferred 1/rms factor and the rotation, stores them as bf16 in shared
+//     memory (same swizzled layout as a TMA tile) and in the cache.  Window tiles are causal.
+//   - Per tile, warp w computes S = Q.K^T for keys 8w..8w+7 on mma.sync m16n8k16 (q as a bf16 pair high + low, fp32
+//     accumulation), the row maxima are exchanged through shared memory (quad shuffles inside the warp first), the
+//     probabilities go to shared memory as bf16 high + low, and warp w accumulates O[:, its HD/8 columns] += P.V over
+//     all keys of the tile.  So a warp holds 8 * QT * HD/64 output registers instead of a whole 16 x HD tile, there
+//     is no merge of warps, and the register count stays low enough for a CTA of the following projection kernel
+//     to be resident beside this one (its weight ring fills while the attention runs).
+//   - The splits are merged through distributed shared memory: every CTA leaves its un-normalised output and its
+//     (max, sum) per row in its own shared memory, a cluster barrier, then each CTA combines a share of the rows'
+//     columns from all splits and writes fp32 output rows.
 // Row j of sequence b sees keys 0 .. kv_len[b] + j (cache + causal part of the window).
+// Every wait is bounded: a tile that does not arrive within the budget raises the error word and the CTA skips its
+// remaining tiles (all CTAs still meet at the cluster barriers).
+#include <cuda.h>
+
 #include <cstring>
 
 #include "fc_internal.h"
@@ -20,8 +32,9 @@ namespace fc {
 
 namespace {
 
-constexpr int kChunk = 128;      // keys per CTA
-constexpr int kAttnThreads = 128;
+constexpr int kTK = 64;          // keys per tile
+constexpr int kAttnThreads = 256;
+constexpr unsigned long long kAttnSpin = 400000000ull;   // clock64 ticks (~0.2 s)
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -30,6 +43,9 @@ __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r
 __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2_t(uint32_t addr, uint32_t &r0, uint32_t &r1) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -41,95 +57,163 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
+__device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  unsigned int spins = 0;
+  while (!mbar_try(bar, parity))
+    if ((++spins & 0xFFu) == 0u && (unsigned long long)(clock64() - t0) > kAttnSpin) return false;
+  return true;
+}
+// One box of a 3-d tensor map (elements, keys, planes) into shared memory, completion counted on an mbarrier.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_dsmem_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
+// Byte offset of 16-byte piece `ch` of row `r` in a tile stored as sub-tiles of [rows][128 B] (64 bf16 per row and
+// sub-tile, sub-tiles `sub_stride` bytes apart), pieces permuted inside each 8-row group as the 128-byte TMA swizzle
+// does it: piece index ^= row & 7.  TMA tiles start on a 1024-byte boundary, so the formula matches the hardware's.
+__device__ __forceinline__ uint32_t tile_off(int r, int ch, uint32_t sub_stride) {
+  return (uint32_t)(ch >> 3) * sub_stride + (uint32_t)r * 128u + (uint32_t)(((ch & 7) ^ (r & 7)) << 4);
+}
+
+// Window tile geometry shared by host and device: rows per window tile and number of window tiles.
+__host__ __device__ inline int win_rows(int c) { return c <= kTK ? (c + 15) / 16 * 16 : kTK; }
+__host__ __device__ inline int win_tiles(int c) { return (c + kTK - 1) / kTK; }
+
+template <int HD>
+struct AttnCfg {
+  static constexpr int SUB = HD / 64;                       // 128-byte sub-tiles per row
+  static constexpr int NS = HD == 128 ? 3 : 4;              // ring stages
+  static constexpr uint32_t kSubBytes = kTK * 128;          // one sub-tile of a TMA tile
+  static constexpr uint32_t kKBytes = SUB * kSubBytes;      // K (or V) part of a stage
+  static constexpr uint32_t kStage = 2 * kKBytes;
+  static constexpr uint32_t kQTile = 2u * SUB * 2048u;      // 16 query rows: high sub-tiles, then low sub-tiles
+};
+
+template <int HD>
+size_t attn_smem_bytes(int c, int qt) {
+  using C = AttnCfg<HD>;
+  const size_t wstage = 2ull * C::SUB * win_rows(c) * 128;
+  const size_t rows = (size_t)qt * 16;
+  return 1024 + (size_t)C::NS * C::kStage + (size_t)win_tiles(c) * wstage + (size_t)qt * C::kQTile + (size_t)qt * 4096 +
+         8 * rows * 4 /* per-warp maxima / sums */ + rows * 8 /* (max, sum) */ + 8 * rows * 4 /* split weights */;
 }
 
 }  // namespace
 
-template <int HD>
-__global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs a) {
-  constexpr int LD = HD + 8;                 // padded row (elements): ldmatrix rows land in distinct banks
-  constexpr int HALF = HD / 2;
-  constexpr int ND = HD / 8;                 // 8-wide output blocks
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  // One K/V buffer even when the CTA walks over several chunks: two CTAs share an SM, and while one waits for its
-  // next chunk the other computes (measured against two buffers and one CTA per SM: 3.5 vs 5.0 ms of attention at
-  // batch 16, K/V 8192, 8 layers of the 7B shape).
-  __nv_bfloat16 *Ks = reinterpret_cast<__nv_bfloat16 *>(smem_raw);       // [kChunk][LD]
-  __nv_bfloat16 *Vs = Ks + kChunk * LD;                                  // [kChunk][LD]
-  __nv_bfloat16 *Qs = Vs + kChunk * LD;                                  // [16][LD]  high part of q
-  __nv_bfloat16 *Ql = Qs + 16 * LD;                                      // [16][LD]  low part: q - bf16(q)
-  float *Om = reinterpret_cast<float *>(Ql + 16 * LD);                   // [4][16][HD]
-  float *mls = Om + 4 * 16 * HD;                                         // [4][16][2]
-  __shared__ unsigned int s_last, s_last_grid;
+template <int HD, int QT>
+__global__ void __maxnreg__(128)
+attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const FusedAttnArgs a) {
+  using C = AttnCfg<HD>;
+  constexpr int SUB = C::SUB, NS = C::NS, HALF = HD / 2;
+  constexpr int NDW = HD / 64;               // 8-wide output blocks per warp (8 warps x NDW x 8 columns = HD)
+  constexpr int ROWS = QT * 16;
+  constexpr uint32_t kSubBytes = C::kSubBytes, kKBytes = C::kKBytes, kStage = C::kStage;
 
-  // blockIdx.x = split * qsplit + query tile: with several chunks per CTA every 16-row query tile gets CTAs of its own
-  // (they produce the same window keys and write the same values to the cache)
-  const int split = blockIdx.x / a.qsplit, kvh = blockIdx.y, bl = blockIdx.z;
-  const int b = a.b0 + bl;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int L = a.kv_len[b];
-  const int ltot = L + a.c;
-  // this CTA's chunks: ch_first .. ch_first + n_iter - 1 (one iteration with no keys for a surplus CTA)
-  const int ch_first = split * a.cpc;
-  const int n_live = min(a.cpc, (ltot - ch_first * kChunk + kChunk - 1) / kChunk);
-  const int n_iter = max(1, n_live);
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long full_bar[NS];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g4 = lane >> 2, t4 = lane & 3;
+  const int split = blockIdx.x, ns = gridDim.x;
   const int group = a.hq / a.hkv;
   const int nq = group * a.c;
+  const int nqg = ((nq + 15) / 16 + QT - 1) / QT;
+  const int kvh = blockIdx.y / nqg, qg = blockIdx.y - kvh * nqg;
+  const int bl = blockIdx.z, b = a.b0 + bl;
+  const int c = a.c;
   const int qd = a.hq * HD, kvd = a.hkv * HD;
   const unsigned int c_magic = a.c_magic;
-  auto div_c = [&](int q) -> int { return a.c == 1 ? q : (int)__umulhi((unsigned int)q, c_magic); };
-  __nv_bfloat16 *kbase = (__nv_bfloat16 *)a.kcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
-  __nv_bfloat16 *vbase = (__nv_bfloat16 *)a.vcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+  auto div_c = [&](int q) -> int { return c == 1 ? q : (int)__umulhi((unsigned int)q, c_magic); };
 
-  // ---- cached keys of a chunk: 16-byte asynchronous copies (one group per chunk); the first chunk's are issued
-  // before anything else
-  constexpr int CPR = HD / 8;                                // 16-byte pieces per row
-  auto issue_chunk = [&](int ch) {
-    const int k0c = ch * kChunk;
-    const int nkc = min(kChunk, ltot - k0c);
-    const int n_cached_c = nkc > 0 ? min(nkc, max(0, L - k0c)) : 0;
-    for (int e = tid; e < n_cached_c * CPR; e += kAttnThreads) {
-      const int t = e / CPR, p = e % CPR;
-      cp_async16(smem_addr(Ks + t * LD + p * 8), kbase + (long long)(k0c + t) * HD + p * 8);
-      cp_async16(smem_addr(Vs + t * LD + p * 8), vbase + (long long)(k0c + t) * HD + p * 8);
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
+  // ---- shared-memory layout (byte offsets from a 1024-byte boundary)
+  const uint32_t base = (smem_addr(smem_raw) + 1023u) & ~1023u;
+  unsigned char *gen = smem_raw + (base - smem_addr(smem_raw));
+  const int wrows = win_rows(c), nwt = win_tiles(c);
+  const uint32_t wsub = (uint32_t)wrows * 128u, wk = SUB * wsub, wstage = 2u * wk;
+  const uint32_t off_win = NS * kStage;
+  const uint32_t off_q = off_win + (uint32_t)nwt * wstage;
+  const uint32_t off_p = off_q + QT * C::kQTile;
+  const uint32_t off_wmax = off_p + QT * 4096u;
+  const uint32_t off_ml = off_wmax + 8u * ROWS * 4u;
+  const uint32_t off_wgt = off_ml + ROWS * 8u;
+  float *wmax = reinterpret_cast<float *>(gen + off_wmax);    // [8 warps][ROWS]
+  float *ml = reinterpret_cast<float *>(gen + off_ml);        // [ROWS][2]
+  float *wgt = reinterpret_cast<float *>(gen + off_wgt);      // [splits][ROWS]
+  float *obuf = reinterpret_cast<float *>(gen);               // [ROWS][HD], over ring stage 0 once the tiles are consumed
+
+  const int L = a.kv_len[b];
+  const int n_ct = (L + kTK - 1) / kTK;                       // tiles of cached keys
+  const int tps = (n_ct + ns - 1) / ns;
+  const int t_begin = min(n_ct, split * tps);
+  const int n_cached = min(n_ct, t_begin + tps) - t_begin;
+  const int n_win = split == ns - 1 ? nwt : 0;
+  const int plane_k = a.k_plane0 + b * a.hkv + kvh, plane_v = a.v_plane0 + b * a.hkv + kvh;
+
+  auto issue_tile = [&](int it) {                              // thread 0 only
+    const int stage = it % NS;
+    const uint32_t bar = smem_addr(&full_bar[stage]);
+    const uint32_t dst = base + stage * kStage;
+    const int y = (t_begin + it) * kTK;
+    mbar_expect_tx(bar, kStage);
+#pragma unroll
+    for (int s = 0; s < SUB; ++s) tma_load_3d(dst + s * kSubBytes, &kmap, s * 64, y, plane_k, bar);
+#pragma unroll
+    for (int s = 0; s < SUB; ++s) tma_load_3d(dst + kKBytes + s * kSubBytes, &vmap, s * 64, y, plane_v, bar);
   };
-  issue_chunk(ch_first);
-  // The cached keys above were written by earlier steps; everything below depends on the previous kernel
-  // (the QKV projection), so let the next kernel start its prefetch and wait for the previous one here.
+
+  if (tid == 0) {
+#pragma unroll
+    for (int i = 0; i < NS; ++i) mbar_init(smem_addr(&full_bar[i]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // cached keys were written by earlier steps: request the first tiles before waiting for the QKV projection
+    for (int it = 0; it < NS && it < n_cached; ++it) issue_tile(it);
+  }
+  __syncthreads();
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 
-  // Q tile registers: a thread keeps one pair index and walks the 16 rows of a tile; all loads of a tile are
-  // issued together.  The first tile's loads are issued here so that their latency overlaps the prologue.
-  constexpr int QRPI = kAttnThreads / HALF;                  // rows covered per pass
-  constexpr int QNIT = 16 / QRPI;
-  const int qi_pair = tid % HALF, q_rsub = tid / HALF;
-  float qx0[QNIT], qx1[QNIT], qss[QNIT];
-  float2 qrot[QNIT];
-  auto q_load = [&](int qt) {
-#pragma unroll
-    for (int it = 0; it < QNIT; ++it) {
-      const int qrow = qt * 16 + q_rsub + it * QRPI;
-      qx0[it] = qx1[it] = 0.f; qss[it] = 0.f; qrot[it] = make_float2(1.f, 0.f);
-      if (qrow < nq) {
-        const int g = div_c(qrow), j = qrow - g * a.c;
-        const int r = bl * a.c + j, h = kvh * group + g;
-        const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
-        qss[it] = __ldcg(a.ss + r);
-        qx0[it] = __ldcg(qacc + qi_pair); qx1[it] = __ldcg(qacc + qi_pair + HALF);
-        qrot[it] = __ldg(a.rope + (long long)(L + j) * HALF + qi_pair);
-      }
-    }
-  };
-  const int qt_first = a.qsplit > 1 ? (int)(blockIdx.x % a.qsplit) : 0;
-  q_load(qt_first);
-
-  // side clearing of buffers nobody reads during this kernel
+  // ---- side clearing of buffers nobody reads during this kernel
   {
     const unsigned long long gtid =
         ((unsigned long long)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * blockDim.x + tid;
@@ -137,7 +221,6 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       if (!a.z.p[i]) continue;
-      // 16-byte stores over the aligned bulk, scalar stores for the tail (buffers are 256-byte aligned)
       const unsigned long long n4 = a.z.n[i] >> 2;
       float4 *p4 = reinterpret_cast<float4 *>(a.z.p[i]);
       for (unsigned long long e = gtid; e < n4; e += nth) p4[e] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -145,352 +228,403 @@ __global__ void __launch_bounds__(kAttnThreads) attn_fused_kernel(FusedAttnArgs 
     }
   }
 
-  const float scale = rsqrtf((float)HD);
-  const int qt_end = a.qsplit > 1 ? qt_first + 1 : (nq + 15) / 16;   // all query tiles, or this CTA's own
-  const int g4 = lane >> 2, t4 = lane & 3;
-  // running softmax statistics and output of this warp's keys over the CTA's chunks (rows g4 and g4 + 8)
-  float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f}, oacc[ND][4];
-  for (int ci = 0; ci < n_iter; ++ci) {
-  const int k0 = (ch_first + ci) * kChunk;
-  const int nk = min(kChunk, ltot - k0);                     // <= 0 for a surplus CTA
-  const int n_cached = nk > 0 ? min(nk, max(0, L - k0)) : 0;
-  const bool has_next = ci + 1 < n_iter;
-  if (nk > 0) {
-    // ---- window keys owned by this chunk: from the accumulators, rotated, stored to smem and to the cache.
-    // A thread keeps one pair index i and walks the window rows in passes; the loads of a pass are all issued
-    // before the first use so that they share one trip to L2.
-    {
-      constexpr int RPI = kAttnThreads / HALF;               // rows covered per pass
-      constexpr int NB = 16 / RPI;                           // passes batched together: 16 window rows per trip
-      const int i = tid % HALF, rsub = tid / HALF;
-      const int n_win = nk - n_cached;
-      for (int t0 = 0; t0 < n_win; t0 += RPI * NB) {
-        float k0v[NB], k1v[NB], v0v[NB], v1v[NB], ssv[NB];
-        float2 rot[NB];
+  // ---- queries: 1/rms, rotation, bf16 high + low, into shared memory.  A thread keeps one pair index i and walks the
+  // rows; four rows' loads are issued together.
+  {
+    constexpr int RPP = kAttnThreads / HALF;                  // rows per pass
+    const int i = tid % HALF, rsub = tid / HALF;
+    for (int r0 = 0; r0 < ROWS; r0 += RPP * 4) {
+      float x0[4], x1[4], ssv[4];
+      float2 rot[4];
 #pragma unroll
-        for (int u = 0; u < NB; ++u) {
-          const int tw = t0 + u * RPI + rsub;
-          k0v[u] = k1v[u] = v0v[u] = v1v[u] = ssv[u] = 0.f; rot[u] = make_float2(1.f, 0.f);
-          if (tw < n_win) {
-            const int pos = k0 + n_cached + tw, j = pos - L;
-            const int r = bl * a.c + j;
-            const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
-            ssv[u] = __ldcg(a.ss + r);
-            k0v[u] = __ldcg(kacc + i); k1v[u] = __ldcg(kacc + i + HALF);
-            v0v[u] = __ldcg(kacc + kvd + i); v1v[u] = __ldcg(kacc + kvd + i + HALF);
-            rot[u] = __ldg(a.rope + (long long)pos * HALF + i);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < NB; ++u) {
-          const int tw = t0 + u * RPI + rsub;
-          if (tw >= n_win) continue;
-          const int t = n_cached + tw, pos = k0 + t;
-          const float sc = rsqrtf(ssv[u] / (float)a.dn + a.eps);
-          const float x0 = k0v[u] * sc, x1 = k1v[u] * sc;
-          const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * rot[u].x - x1 * rot[u].y);
-          const __nv_bfloat16 o1 = __float2bfloat16_rn(x0 * rot[u].y + x1 * rot[u].x);
-          const __nv_bfloat16 w0 = __float2bfloat16_rn(v0v[u] * sc), w1 = __float2bfloat16_rn(v1v[u] * sc);
-          Ks[t * LD + i] = o0; Ks[t * LD + i + HALF] = o1;
-          Vs[t * LD + i] = w0; Vs[t * LD + i + HALF] = w1;
-          kbase[(long long)pos * HD + i] = o0; kbase[(long long)pos * HD + i + HALF] = o1;
-          vbase[(long long)pos * HD + i] = w0; vbase[(long long)pos * HD + i + HALF] = w1;
+      for (int u = 0; u < 4; ++u) {
+        const int rl = r0 + u * RPP + rsub;
+        const int qrow = qg * ROWS + rl;
+        x0[u] = x1[u] = ssv[u] = 0.f; rot[u] = make_float2(1.f, 0.f);
+        if (rl < ROWS && qrow < nq) {
+          const int g = div_c(qrow), j = qrow - g * c;
+          const int r = bl * c + j, h = kvh * group + g;
+          const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
+          ssv[u] = __ldcg(a.ss + r);
+          x0[u] = __ldcg(qacc + i); x1[u] = __ldcg(qacc + i + HALF);
+          rot[u] = __ldg(a.rope + (long long)(L + j) * HALF + i);
         }
       }
-    }
-    // rows beyond nk: zero so that stale shared memory (possibly NaN patterns) never meets a zero weight
-    for (int e = tid; e < (kChunk - nk) * CPR; e += kAttnThreads) {
-      const int t = nk + e / CPR, p = e % CPR;
-      *reinterpret_cast<uint4 *>(Ks + t * LD + p * 8) = make_uint4(0, 0, 0, 0);
-      *reinterpret_cast<uint4 *>(Vs + t * LD + p * 8) = make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int rl = r0 + u * RPP + rsub;
+        if (rl >= ROWS) continue;
+        const float sc = rsqrtf(ssv[u] / (float)a.dn + a.eps);
+        const float a0 = x0[u] * sc, a1 = x1[u] * sc;
+        const float q0 = a0 * rot[u].x - a1 * rot[u].y, q1 = a0 * rot[u].y + a1 * rot[u].x;
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(q0), h1 = __float2bfloat16_rn(q1);
+        unsigned char *qt_base = gen + off_q + (uint32_t)(rl >> 4) * C::kQTile;
+        const int row = rl & 15;
+        const uint32_t o0 = tile_off(row, i >> 3, 2048u) + (uint32_t)(i & 7) * 2u;
+        const uint32_t o1 = tile_off(row, (i + HALF) >> 3, 2048u) + (uint32_t)(i & 7) * 2u;
+        *reinterpret_cast<__nv_bfloat16 *>(qt_base + o0) = h0;
+        *reinterpret_cast<__nv_bfloat16 *>(qt_base + o1) = h1;
+        *reinterpret_cast<__nv_bfloat16 *>(qt_base + SUB * 2048u + o0) = __float2bfloat16_rn(q0 - __bfloat162float(h0));
+        *reinterpret_cast<__nv_bfloat16 *>(qt_base + SUB * 2048u + o1) = __float2bfloat16_rn(q1 - __bfloat162float(h1));
+      }
     }
   }
 
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  for (int qt = qt_first; qt < qt_end; ++qt) {
-    __syncthreads();                                          // K/V staged; previous tile's Qs/Om/mls free
-    // ---- Q tile: 1/rms, rotation, bf16 (loads were issued earlier for the first tile); staged once per tile
-    if (ci == 0) {
-    if (qt > qt_first) q_load(qt);
+  // ---- the window's own keys (last split): from the accumulators, rotated, to shared memory and to the cache
+  if (n_win > 0) {
+    __nv_bfloat16 *kbase = (__nv_bfloat16 *)a.kcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+    __nv_bfloat16 *vbase = (__nv_bfloat16 *)a.vcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+    constexpr int RPP = kAttnThreads / HALF;
+    const int i = tid % HALF, rsub = tid / HALF;
+    for (int j0 = 0; j0 < c; j0 += RPP * 4) {
+      float k0v[4], k1v[4], v0v[4], v1v[4], ssv[4];
+      float2 rot[4];
 #pragma unroll
-    for (int it = 0; it < QNIT; ++it) {
-      const int row = q_rsub + it * QRPI;
-      const float sc = rsqrtf(qss[it] / (float)a.dn + a.eps);
-      const float a0 = qx0[it] * sc, a1 = qx1[it] * sc;
-      // q and the probabilities go through the tensor cores as a bf16 pair hi + lo, so that only the cached
-      // K and V (stored in the model dtype) carry bf16 rounding
-      const float r0 = a0 * qrot[it].x - a1 * qrot[it].y, r1 = a0 * qrot[it].y + a1 * qrot[it].x;
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(r0), h1 = __float2bfloat16_rn(r1);
-      Qs[row * LD + qi_pair] = h0; Qs[row * LD + qi_pair + HALF] = h1;
-      Ql[row * LD + qi_pair] = __float2bfloat16_rn(r0 - __bfloat162float(h0));
-      Ql[row * LD + qi_pair + HALF] = __float2bfloat16_rn(r1 - __bfloat162float(h1));
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + u * RPP + rsub;
+        k0v[u] = k1v[u] = v0v[u] = v1v[u] = ssv[u] = 0.f; rot[u] = make_float2(1.f, 0.f);
+        if (j < c) {
+          const int r = bl * c + j;
+          const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
+          ssv[u] = __ldcg(a.ss + r);
+          k0v[u] = __ldcg(kacc + i); k1v[u] = __ldcg(kacc + i + HALF);
+          v0v[u] = __ldcg(kacc + kvd + i); v1v[u] = __ldcg(kacc + kvd + i + HALF);
+          rot[u] = __ldg(a.rope + (long long)(L + j) * HALF + i);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + u * RPP + rsub;
+        if (j >= c) continue;
+        const int pos = L + j;
+        const float sc = rsqrtf(ssv[u] / (float)a.dn + a.eps);
+        const float x0 = k0v[u] * sc, x1 = k1v[u] * sc;
+        const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * rot[u].x - x1 * rot[u].y);
+        const __nv_bfloat16 o1 = __float2bfloat16_rn(x0 * rot[u].y + x1 * rot[u].x);
+        const __nv_bfloat16 w0 = __float2bfloat16_rn(v0v[u] * sc), w1 = __float2bfloat16_rn(v1v[u] * sc);
+        unsigned char *wt_base = gen + off_win + (uint32_t)(j / kTK) * wstage;
+        const int row = j % kTK;
+        const uint32_t f0 = tile_off(row, i >> 3, wsub) + (uint32_t)(i & 7) * 2u;
+        const uint32_t f1 = tile_off(row, (i + HALF) >> 3, wsub) + (uint32_t)(i & 7) * 2u;
+        *reinterpret_cast<__nv_bfloat16 *>(wt_base + f0) = o0;
+        *reinterpret_cast<__nv_bfloat16 *>(wt_base + f1) = o1;
+        *reinterpret_cast<__nv_bfloat16 *>(wt_base + wk + f0) = w0;
+        *reinterpret_cast<__nv_bfloat16 *>(wt_base + wk + f1) = w1;
+        kbase[(long long)pos * HD + i] = o0; kbase[(long long)pos * HD + i + HALF] = o1;
+        vbase[(long long)pos * HD + i] = w0; vbase[(long long)pos * HD + i + HALF] = w1;
+      }
     }
-    __syncthreads();
+    // rows of the last window tile beyond the window: zero, so that a zero probability never meets a stale NaN pattern
+    {
+      const int wt = nwt - 1;
+      const int nv = c - wt * kTK;
+      unsigned char *wt_base = gen + off_win + (uint32_t)wt * wstage;
+      for (int e = tid; e < (wrows - nv) * (HD / 8); e += kAttnThreads) {
+        const int row = nv + e / (HD / 8), ch = e % (HD / 8);
+        *reinterpret_cast<uint4 *>(wt_base + tile_off(row, ch, wsub)) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4 *>(wt_base + wk + tile_off(row, ch, wsub)) = make_uint4(0, 0, 0, 0);
+      }
+    }
+  }
+
+  // ---- per-lane row bookkeeping: window row of query rows g4 and g4 + 8 of each tile (-1: no such query)
+  int jrow[QT][2];
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) { mrun[hh] = -INFINITY; lrun[hh] = 0.f; }
+  for (int qt = 0; qt < QT; ++qt)
 #pragma unroll
-    for (int d = 0; d < ND; ++d)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) oacc[d][i] = 0.f;
+    for (int hh = 0; hh < 2; ++hh) {
+      const int qrow = qg * ROWS + qt * 16 + g4 + hh * 8;
+      jrow[qt][hh] = qrow < nq ? qrow - div_c(qrow) * c : -1;
     }
 
-    // ---- S = Q.K^T for this warp's 32 keys
-    float sacc[4][4];
+  const float scale = rsqrtf((float)HD);
+  float m_run[QT][2], l_run[QT][2], oacc[QT][NDW][4];
 #pragma unroll
-    for (int nb = 0; nb < 4; ++nb)
+  for (int qt = 0; qt < QT; ++qt) {
+    m_run[qt][0] = m_run[qt][1] = -INFINITY;
+    l_run[qt][0] = l_run[qt][1] = 0.f;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) sacc[nb][i] = 0.f;
-    if (nk > 0) {
+    for (int nd = 0; nd < NDW; ++nd)
 #pragma unroll
-      for (int ks = 0; ks < HD / 16; ++ks) {
-        uint32_t af[4], al[4];
-        ldsm_x4(smem_addr(Qs + (lane & 15) * LD + ks * 16 + (lane >> 4) * 8), af[0], af[1], af[2], af[3]);
-        ldsm_x4(smem_addr(Ql + (lane & 15) * LD + ks * 16 + (lane >> 4) * 8), al[0], al[1], al[2], al[3]);
+      for (int i = 0; i < 4; ++i) oacc[qt][nd][i] = 0.f;
+  }
+
+  __syncthreads();                                            // queries and window keys staged
+  bool all_ok = true;
+  const int n_tiles = n_cached + n_win;
+  for (int ti = 0; ti < n_tiles; ++ti) {
+    uint32_t kb, vb, sstride;
+    int koff, nvalid, rows_t;                                 // key offset relative to L for window tiles
+    bool ok = true;
+    const bool causal = ti >= n_cached;
+    if (!causal) {
+      const int stage = ti % NS;
+      ok = mbar_wait_bounded(smem_addr(&full_bar[stage]), (uint32_t)(ti / NS) & 1u);
+      kb = base + stage * kStage; vb = kb + kKBytes; sstride = kSubBytes;
+      const int key0 = (t_begin + ti) * kTK;
+      koff = 0; nvalid = min(kTK, L - key0); rows_t = kTK;
+      if (nvalid < kTK) {
+        // the tile's rows beyond the cached keys hold whatever the slab holds there: zero the V rows (the K rows are
+        // masked by a select, a zero probability would still multiply a NaN pattern in V)
+        unsigned char *vg = gen + (vb - base);
+        for (int e = tid; e < (kTK - nvalid) * (HD / 8); e += kAttnThreads) {
+          const int row = nvalid + e / (HD / 8), ch = e % (HD / 8);
+          *reinterpret_cast<uint4 *>(vg + tile_off(row, ch, kSubBytes)) = make_uint4(0, 0, 0, 0);
+        }
+      }
+    } else {
+      const int wt = ti - n_cached;
+      kb = base + off_win + (uint32_t)wt * wstage; vb = kb + wk; sstride = wsub;
+      koff = wt * kTK; nvalid = min(kTK, c - koff); rows_t = wrows;
+    }
+
+    // ---- S = Q.K^T for this warp's 8 keys
+    float s[QT][4];
 #pragma unroll
-        for (int nb = 0; nb < 4; nb += 2) {
-          // two key blocks (8 keys each) x one 16-wide k step
-          uint32_t b0, b1, b2, b3;
-          const int key = warp * 32 + nb * 8 + (lane & 7) + ((lane >> 4) & 1) * 8;
-          ldsm_x4(smem_addr(Ks + key * LD + ks * 16 + ((lane >> 3) & 1) * 8), b0, b1, b2, b3);
-          mma_bf16(sacc[nb], af, b0, b1);
-          mma_bf16(sacc[nb + 1], af, b2, b3);
-          mma_bf16(sacc[nb], al, b0, b1);
-          mma_bf16(sacc[nb + 1], al, b2, b3);
+    for (int qt = 0; qt < QT; ++qt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) s[qt][i] = 0.f;
+    const bool my_keys = warp * 8 < rows_t;
+    if (my_keys) {
+#pragma unroll
+      for (int ks2 = 0; ks2 < HD / 32; ++ks2) {
+        uint32_t kf[4];
+        ldsm_x4(kb + tile_off(warp * 8 + (lane & 7), ks2 * 4 + (lane >> 3), sstride), kf[0], kf[1], kf[2], kf[3]);
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+          const uint32_t qoff = tile_off(lane & 15, (ks2 * 2 + h2) * 2 + (lane >> 4), 2048u);
+#pragma unroll
+          for (int qt = 0; qt < QT; ++qt) {
+            uint32_t ah[4], al[4];
+            const uint32_t qb = base + off_q + (uint32_t)qt * C::kQTile + qoff;
+            ldsm_x4(qb, ah[0], ah[1], ah[2], ah[3]);
+            ldsm_x4(qb + SUB * 2048u, al[0], al[1], al[2], al[3]);
+            mma_bf16(s[qt], ah, kf[h2 * 2], kf[h2 * 2 + 1]);
+            mma_bf16(s[qt], al, kf[h2 * 2], kf[h2 * 2 + 1]);
+          }
         }
       }
     }
-    // ---- mask, scale, softmax statistics over this warp's keys (rows g4 and g4 + 8)
-    float mrow[2] = {-INFINITY, -INFINITY};
-    int jrow[2];
+    // ---- mask, scale, maxima over this warp's keys
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int qrow = qt * 16 + g4 + hh * 8;
-      jrow[hh] = (qrow < nq) ? (qrow - div_c(qrow) * a.c) : -1;
-    }
-#pragma unroll
-    for (int nb = 0; nb < 4; ++nb)
+    for (int qt = 0; qt < QT; ++qt) {
+      float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int hh = i >> 1;
-        const int key = k0 + warp * 32 + nb * 8 + t4 * 2 + (i & 1);
-        const bool ok = jrow[hh] >= 0 && key < ltot && key <= L + jrow[hh];
-        const float s = ok ? sacc[nb][i] * scale : -INFINITY;
-        sacc[nb][i] = s;
-        mrow[hh] = fmaxf(mrow[hh], s);
+        const int kl = warp * 8 + t4 * 2 + (i & 1);
+        const bool vis = my_keys && jrow[qt][hh] >= 0 && kl < nvalid && (!causal || koff + kl <= jrow[qt][hh]);
+        const float v = vis ? s[qt][i] * scale : -INFINITY;
+        s[qt][i] = v;
+        mx[hh] = fmaxf(mx[hh], v);
       }
-    float lrow[2] = {0.f, 0.f};
-    float corr[2];                                            // rescales what earlier chunks contributed
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      mrow[hh] = fmaxf(mrow[hh], __shfl_xor_sync(0xffffffffu, mrow[hh], 1));
-      mrow[hh] = fmaxf(mrow[hh], __shfl_xor_sync(0xffffffffu, mrow[hh], 2));
-      mrow[hh] = fmaxf(mrow[hh], mrun[hh]);                   // running maximum including this chunk
-      corr[hh] = (mrun[hh] == -INFINITY) ? 0.f : __expf(mrun[hh] - mrow[hh]);
-      mrun[hh] = mrow[hh];
+      for (int hh = 0; hh < 2; ++hh) {
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
+        if (t4 == 0) wmax[warp * ROWS + qt * 16 + g4 + hh * 8] = mx[hh];
+      }
     }
-    uint32_t pf[2][4], pl[2][4];                              // P (high and low parts) as A fragments: two 16-key steps
+    all_ok = __syncthreads_and(ok ? 1 : 0) != 0;              // maxima published; every warp is past the previous tile
+    if (!all_ok) break;
+    // the stage of the previous cached tile is free: request the tile NS ahead of it
+    if (tid == 0 && ti >= 1 && ti - 1 + NS < n_cached) issue_tile(ti - 1 + NS);
+
+    // ---- probabilities (bf16 high + low) to shared memory; running maximum and this warp's share of the sum
 #pragma unroll
-    for (int nb = 0; nb < 4; ++nb) {
+    for (int qt = 0; qt < QT; ++qt) {
+      float mnew[2], corr[2], lsum[2] = {0.f, 0.f};
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int row = qt * 16 + g4 + hh * 8;
+        float mx = m_run[qt][hh];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) mx = fmaxf(mx, wmax[w * ROWS + row]);
+        mnew[hh] = mx;
+        corr[hh] = (m_run[qt][hh] == -INFINITY) ? 0.f : __expf(m_run[qt][hh] - mx);
+        m_run[qt][hh] = mx;
+      }
       float p[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int hh = i >> 1;
-        p[i] = (sacc[nb][i] == -INFINITY) ? 0.f : __expf(sacc[nb][i] - mrow[hh]);
-        lrow[hh] += p[i];
+        p[i] = (s[qt][i] == -INFINITY) ? 0.f : __expf(s[qt][i] - mnew[hh]);
+        lsum[hh] += p[i];
       }
-      pf[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
-      pf[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
-      float pr[4];
+      if (my_keys) {
+        unsigned char *pb = gen + off_p + (uint32_t)qt * 4096u;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) pr[i] = p[i] - __bfloat162float(__float2bfloat16_rn(p[i]));
-      pl[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16(pr[0], pr[1]);
-      pl[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16(pr[2], pr[3]);
-    }
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      lrow[hh] += __shfl_xor_sync(0xffffffffu, lrow[hh], 1);
-      lrow[hh] += __shfl_xor_sync(0xffffffffu, lrow[hh], 2);
-      lrun[hh] = lrun[hh] * corr[hh] + lrow[hh];
-    }
-    // ---- O = O * corr + P.V
-    if (ci > 0) {
-#pragma unroll
-      for (int d = 0; d < ND; ++d) {
-        oacc[d][0] *= corr[0]; oacc[d][1] *= corr[0];
-        oacc[d][2] *= corr[1]; oacc[d][3] *= corr[1];
-      }
-    }
-    if (nk > 0) {
-#pragma unroll
-      for (int kt = 0; kt < 2; ++kt) {
-#pragma unroll
-        for (int d = 0; d < ND; d += 2) {
-          uint32_t b0, b1, b2, b3;
-          const int key = warp * 32 + kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-          ldsm_x4_t(smem_addr(Vs + key * LD + d * 8 + (lane >> 4) * 8), b0, b1, b2, b3);
-          mma_bf16(oacc[d], pf[kt], b0, b1);
-          mma_bf16(oacc[d + 1], pf[kt], b2, b3);
-          mma_bf16(oacc[d], pl[kt], b0, b1);
-          mma_bf16(oacc[d + 1], pl[kt], b2, b3);
+        for (int hh = 0; hh < 2; ++hh) {
+          const int row = g4 + hh * 8;
+          const uint32_t o = tile_off(row, warp, 2048u) + (uint32_t)t4 * 4u;
+          const float p0 = p[hh * 2], p1 = p[hh * 2 + 1];
+          *reinterpret_cast<uint32_t *>(pb + o) = pack_bf16(p0, p1);
+          *reinterpret_cast<uint32_t *>(pb + 2048u + o) = pack_bf16(p0 - bf16_round(p0), p1 - bf16_round(p1));
         }
       }
-    }
-    if (ci < n_iter - 1) continue;                            // more chunks to come: keep accumulating
-    // ---- merge the four warps (after the CTA's last chunk)
-    if (t4 == 0) {
-      mls[(warp * 16 + g4) * 2] = mrun[0]; mls[(warp * 16 + g4) * 2 + 1] = lrun[0];
-      mls[(warp * 16 + g4 + 8) * 2] = mrun[1]; mls[(warp * 16 + g4 + 8) * 2 + 1] = lrun[1];
-    }
-    __syncthreads();
-    float fac[2];
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-      const int row = g4 + hh * 8;
-      float M = -INFINITY;
+      for (int hh = 0; hh < 2; ++hh) {
+        lsum[hh] += __shfl_xor_sync(0xffffffffu, lsum[hh], 1);
+        lsum[hh] += __shfl_xor_sync(0xffffffffu, lsum[hh], 2);
+        l_run[qt][hh] = l_run[qt][hh] * corr[hh] + lsum[hh];
+      }
 #pragma unroll
-      for (int w = 0; w < 4; ++w) M = fmaxf(M, mls[(w * 16 + row) * 2]);
-      fac[hh] = (mrun[hh] == -INFINITY) ? 0.f : __expf(mrun[hh] - M);
-    }
-#pragma unroll
-    for (int d = 0; d < ND; ++d) {
-      float *o0 = Om + (warp * 16 + g4) * HD + d * 8 + t4 * 2;
-      float *o1 = Om + (warp * 16 + g4 + 8) * HD + d * 8 + t4 * 2;
-      *reinterpret_cast<float2 *>(o0) = make_float2(oacc[d][0] * fac[0], oacc[d][1] * fac[0]);
-      *reinterpret_cast<float2 *>(o1) = make_float2(oacc[d][2] * fac[1], oacc[d][3] * fac[1]);
-    }
-    __syncthreads();
-    for (int e = tid; e < 16 * (HD / 4); e += kAttnThreads) {
-      const int row = e / (HD / 4), d4 = e % (HD / 4);
-      const int qrow = qt * 16 + row;
-      if (qrow >= nq) continue;
-      const int g = div_c(qrow), j = qrow - g * a.c;
-      const int r = bl * a.c + j, h = kvh * group + g;
-      const long long pidx = ((long long)r * a.hq + h) * a.nsplit + split;
-      const float4 p0 = *reinterpret_cast<const float4 *>(Om + row * HD + d4 * 4);
-      const float4 p1 = *reinterpret_cast<const float4 *>(Om + (16 + row) * HD + d4 * 4);
-      const float4 p2 = *reinterpret_cast<const float4 *>(Om + (32 + row) * HD + d4 * 4);
-      const float4 p3 = *reinterpret_cast<const float4 *>(Om + (48 + row) * HD + d4 * 4);
-      *reinterpret_cast<float4 *>(a.part_o + pidx * HD + d4 * 4) =
-          make_float4(p0.x + p1.x + p2.x + p3.x, p0.y + p1.y + p2.y + p3.y, p0.z + p1.z + p2.z + p3.z, p0.w + p1.w + p2.w + p3.w);
-      if (d4 == 0) {
-        float M = -INFINITY;
-        for (int w = 0; w < 4; ++w) M = fmaxf(M, mls[(w * 16 + row) * 2]);
-        float lsum = 0.f;
-        for (int w = 0; w < 4; ++w) {
-          const float mw = mls[(w * 16 + row) * 2];
-          if (mw != -INFINITY) lsum += mls[(w * 16 + row) * 2 + 1] * __expf(mw - M);
-        }
-        *reinterpret_cast<float2 *>(a.part_ml + pidx * 2) = make_float2(M, lsum);
+      for (int nd = 0; nd < NDW; ++nd) {
+        oacc[qt][nd][0] *= corr[0]; oacc[qt][nd][1] *= corr[0];
+        oacc[qt][nd][2] *= corr[1]; oacc[qt][nd][3] *= corr[1];
       }
     }
-  }
-  if (has_next) {
-    __syncthreads();                                          // every warp is done with this chunk's buffer
-    issue_chunk(ch_first + ci + 1);                           // the co-resident CTA computes meanwhile
-  }
-  }
+    __syncthreads();                                          // probabilities staged (and stale V rows zeroed)
 
-  // ---- merge the splits of this (sequence, kv head) and clear the accumulators of its heads.
-  // Cluster launch (the splits of one kv head form one thread-block cluster): a hardware cluster barrier, then
-  // every CTA of the cluster merges its share of the queries.  Otherwise the last CTA to arrive merges them all.
-  int q_first, q_step;
-  unsigned int ctas_counted;
-  if (a.cluster) {
-    __threadfence();
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-    q_first = (int)blockIdx.x * 4 + warp; q_step = (int)gridDim.x * 4;
-    ctas_counted = gridDim.x * gridDim.y * gridDim.z;
-  } else {
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-      const unsigned int prev = atomicAdd(&a.counters[b * a.hkv + kvh], 1u);
-      s_last = (prev == gridDim.x - 1u);
+    // ---- O[:, this warp's columns] += P.V over the tile's keys
+    for (int kt = 0; kt < rows_t / 16; ++kt) {
+      uint32_t vf[4];
+      const int key = kt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+      if (NDW == 2) ldsm_x4_t(vb + tile_off(key, warp * 2 + (lane >> 4), sstride), vf[0], vf[1], vf[2], vf[3]);
+      else { ldsm_x2_t(vb + tile_off(key, warp, sstride), vf[0], vf[1]); vf[2] = vf[3] = 0u; }
+      const uint32_t poff = tile_off(lane & 15, kt * 2 + (lane >> 4), 2048u);
+#pragma unroll
+      for (int qt = 0; qt < QT; ++qt) {
+        uint32_t ph[4], pl[4];
+        const uint32_t pb = base + off_p + (uint32_t)qt * 4096u + poff;
+        ldsm_x4(pb, ph[0], ph[1], ph[2], ph[3]);
+        ldsm_x4(pb + 2048u, pl[0], pl[1], pl[2], pl[3]);
+#pragma unroll
+        for (int nd = 0; nd < NDW; ++nd) {
+          mma_bf16(oacc[qt][nd], ph, vf[nd * 2], vf[nd * 2 + 1]);
+          mma_bf16(oacc[qt][nd], pl, vf[nd * 2], vf[nd * 2 + 1]);
+        }
+      }
     }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    q_first = warp; q_step = 4;
-    ctas_counted = gridDim.y * gridDim.z;
   }
-  for (int qi = q_first; qi < nq; qi += q_step) {
-    const int g = div_c(qi), j = qi - g * a.c;
-    const int r = bl * a.c + j, h = kvh * group + g;
-    const long long base = ((long long)r * a.hq + h) * a.nsplit;
-    // lanes take one split each for the (max, sum) pairs; the output loads below are independent
-    const float2 *ml2 = reinterpret_cast<const float2 *>(a.part_ml) + base;
+  if (!all_ok && tid == 0) atomicExch(a.err, 1u);
+
+  // ---- this CTA's result: un-normalised output rows and (max, sum) per row, in its own shared memory
+  __syncthreads();                                            // all warps are done with the tiles and with wmax
+#pragma unroll
+  for (int qt = 0; qt < QT; ++qt)
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh)
+      if (t4 == 0) wmax[warp * ROWS + qt * 16 + g4 + hh * 8] = l_run[qt][hh];
+#pragma unroll
+  for (int qt = 0; qt < QT; ++qt)
+#pragma unroll
+    for (int nd = 0; nd < NDW; ++nd) {
+      const int col = warp * (8 * NDW) + nd * 8 + t4 * 2;
+      *reinterpret_cast<float2 *>(obuf + (qt * 16 + g4) * HD + col) = make_float2(oacc[qt][nd][0], oacc[qt][nd][1]);
+      *reinterpret_cast<float2 *>(obuf + (qt * 16 + g4 + 8) * HD + col) = make_float2(oacc[qt][nd][2], oacc[qt][nd][3]);
+    }
+  __syncthreads();
+  if (tid < ROWS) {
+    float lt = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) lt += wmax[w * ROWS + tid];
+    // every warp holds the same running maximum; take it from the lane that owns this row in warp tid / 32's layout
+    ml[tid * 2 + 1] = lt;
+  }
+  if (warp == 0 && t4 == 0) {
+#pragma unroll
+    for (int qt = 0; qt < QT; ++qt) {
+      ml[(qt * 16 + g4) * 2] = m_run[qt][0];
+      ml[(qt * 16 + g4 + 8) * 2] = m_run[qt][1];
+    }
+  }
+  if (ns > 1) cluster_sync_all(); else __syncthreads();
+
+  // ---- merge of the splits: weights per (split, row), then every CTA combines its share of the output
+  if (tid < ROWS) {
+    float ms[8], ls[8];
     float M = -INFINITY;
-    for (int s0 = 0; s0 < a.nsplit; s0 += 32) {
-      const int s = s0 + lane;
-      if (s < a.nsplit) { const float2 ml = __ldcg(ml2 + s); if (ml.y > 0.f) M = fmaxf(M, ml.x); }
+    for (int sp = 0; sp < ns; ++sp) {
+      float2 v;
+      if (ns > 1) v = ld_dsmem_f2(map_to_rank(base + off_ml + (uint32_t)tid * 8u, (uint32_t)sp));
+      else v = make_float2(ml[tid * 2], ml[tid * 2 + 1]);
+      ms[sp] = v.x; ls[sp] = v.y;
+      if (v.y > 0.f) M = fmaxf(M, v.x);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    float den = 0.f, o[HD / 32];
-#pragma unroll
-    for (int i = 0; i < HD / 32; ++i) o[i] = 0.f;
-    for (int s0 = 0; s0 < a.nsplit; s0 += 32) {
-      const int s = s0 + lane;
-      float wl = 0.f, wgt = 0.f;
-      if (s < a.nsplit) {
-        const float2 ml = __ldcg(ml2 + s);
-        if (ml.y > 0.f) { wgt = __expf(ml.x - M); wl = ml.y * wgt; }
-      }
-#pragma unroll
-      for (int sh = 16; sh > 0; sh >>= 1) wl += __shfl_xor_sync(0xffffffffu, wl, sh);
-      den += wl;
-      const int ns = min(32, a.nsplit - s0);
-      const float *po = a.part_o + (base + s0) * HD + lane;
-#pragma unroll 8
-      for (int t = 0; t < ns; ++t) {
-        const float w = __shfl_sync(0xffffffffu, wgt, t);
-#pragma unroll
-        for (int i = 0; i < HD / 32; ++i) o[i] = fmaf(w, __ldcg(po + (long long)t * HD + i * 32), o[i]);
-      }
+    float den = 0.f;
+    for (int sp = 0; sp < ns; ++sp) {
+      ms[sp] = ls[sp] > 0.f ? __expf(ms[sp] - M) : 0.f;
+      den += ls[sp] * ms[sp];
     }
-    const float inv = 1.0f / den;
-#pragma unroll
-    for (int i = 0; i < HD / 32; ++i) a.out[(long long)r * qd + h * HD + i * 32 + lane] = o[i] * inv;
-    // this head's q accumulator (and, once per row, the kv head's k and v) are no longer needed
-    float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
-    for (int i = lane; i < HD; i += 32) qacc[i] = 0.f;
-    if (g == 0) {
-      float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
-      for (int i = lane; i < HD; i += 32) { kacc[i] = 0.f; kacc[kvd + i] = 0.f; }
-    }
-  }
-  // the last CTA (of those counted) clears the per-row sums of squares: every reader is done by then
-  __syncthreads();
-  if (tid == 0) {
-    if (!a.cluster) a.counters[b * a.hkv + kvh] = 0u;
-    const unsigned int prev = atomicAdd(a.grid_counter, 1u);
-    s_last_grid = (prev == ctas_counted - 1u);
+    const float inv = den > 0.f ? 1.0f / den : 0.f;
+    for (int sp = 0; sp < ns; ++sp) wgt[sp * ROWS + tid] = ms[sp] * inv;
   }
   __syncthreads();
-  if (s_last_grid) {
-    for (int i = tid; i < a.nb * a.c; i += kAttnThreads) a.ss[i] = 0.f;
-    if (tid == 0) *a.grid_counter = 0u;
+  for (int u = split * kAttnThreads + tid; u < ROWS * (HD / 4); u += ns * kAttnThreads) {
+    const int row = u / (HD / 4), c4 = u - row * (HD / 4);
+    const int qrow = qg * ROWS + row;
+    if (qrow >= nq) continue;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sp = 0; sp < ns; ++sp) {
+      const float w = wgt[sp * ROWS + row];
+      float4 v;
+      if (ns > 1) v = ld_dsmem_f4(map_to_rank(base + (uint32_t)(row * HD + c4 * 4) * 4u, (uint32_t)sp));
+      else v = *reinterpret_cast<const float4 *>(obuf + row * HD + c4 * 4);
+      acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y); acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+    }
+    const int g = div_c(qrow), j = qrow - g * c;
+    const int r = bl * c + j, h = kvh * group + g;
+    *reinterpret_cast<float4 *>(a.out + (long long)r * qd + h * HD + c4 * 4) = acc;
   }
+  if (ns > 1) cluster_sync_all();                             // the other splits may still be reading this CTA's memory
 }
 
-template <int HD>
-static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
-  constexpr int LD = HD + 8;
-  const int nqt = ((a.hq / a.hkv) * a.c + 15) / 16;
-  if (a.cpc < 1 || (a.qsplit != 1 && a.qsplit != nqt) || (a.cpc > 1 && a.qsplit != nqt)) return cudaErrorInvalidValue;
-  const size_t smem = sizeof(__nv_bfloat16) * (size_t)(2 * kChunk * LD + 2 * 16 * LD) +
-                      sizeof(float) * (size_t)(4 * 16 * HD + 4 * 16 * 2);
+// ------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t make_kv_tensor_map(KvTensorMap *out, const void *base, int hd, int max_seq, long long planes) {
+  static_assert(sizeof(CUtensorMap) <= sizeof(KvTensorMap), "tensor map storage");
+  static EncodeTiledFn enc = nullptr;
+  if (!enc) {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    enc = (EncodeTiledFn)sym;
+  }
+  if ((hd != 64 && hd != 128) || max_seq < 1 || planes < 1 || ((uintptr_t)base & 15)) return cudaErrorInvalidValue;
+  cuuint64_t gdim[3] = {(cuuint64_t)hd, (cuuint64_t)max_seq, (cuuint64_t)planes};
+  cuuint64_t gstr[2] = {(cuuint64_t)hd * 2, (cuuint64_t)max_seq * hd * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)kTK, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(reinterpret_cast<CUtensorMap *>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), gdim,
+                   gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int &nsplit, int &qt) {
+  const int nqt = ((hq / hkv) * c + 15) / 16;
+  qt = 1;
+  while (qt < 4 && qt < nqt && (long long)nb * hkv * ((nqt + qt - 1) / qt) > 2ll * n_sms) qt *= 2;
+  const long long units = (long long)nb * hkv * ((nqt + qt - 1) / qt);
+  const int n_ct = (max_len + kTK - 1) / kTK;
+  long long s = n_sms / units;                                // one CTA per SM: the projection kernel's CTAs come in beside them
+  if (s > 8) s = 8;
+  if (s > n_ct) s = n_ct;
+  if (s < 1) s = 1;
+  nsplit = (int)s;
+}
+
+template <int HD, int QT>
+static cudaError_t launch_fused_t(const KvTensorMap &kmap, const KvTensorMap &vmap, const FusedAttnArgs &a, cudaStream_t st) {
+  const size_t smem = attn_smem_bytes<HD>(a.c, QT);
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
   static size_t attr_smem[kMaxDevices] = {0};
   const int dev = current_device_slot();
   if (smem > attr_smem[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attn_tma_kernel<HD, QT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     attr_smem[dev] = smem;
   }
+  const int nqt = ((a.hq / a.hkv) * a.c + 15) / 16;
+  const int nqg = (nqt + QT - 1) / QT;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3(a.nsplit * a.qsplit, a.hkv, a.nb); cfg.blockDim = dim3(kAttnThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cfg.gridDim = dim3(a.nsplit, a.hkv * nqg, a.nb); cfg.blockDim = dim3(kAttnThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
   cudaLaunchAttribute attr[2];
   int na = 0;
   if (a.pdl) {
@@ -498,43 +632,31 @@ static cudaError_t launch_fused_t(const FusedAttnArgs &a, cudaStream_t st) {
     attr[na].val.programmaticStreamSerializationAllowed = 1;
     ++na;
   }
-  // Largest cluster this kernel can be scheduled with: 16 (non-portable size) if the device takes it, else 8.
-  static int max_cluster_dev[kMaxDevices] = {0};
-  int &max_cluster = max_cluster_dev[dev];
-  if (max_cluster == 0) {
-    max_cluster = 8;
-    if (cudaFuncSetAttribute(attn_fused_kernel<HD>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
-      cudaLaunchConfig_t q;
-      memset(&q, 0, sizeof q);
-      q.gridDim = dim3(16, 1, 1); q.blockDim = dim3(kAttnThreads); q.dynamicSmemBytes = smem;
-      cudaLaunchAttribute qa[1];
-      qa[0].id = cudaLaunchAttributeClusterDimension;
-      qa[0].val.clusterDim.x = 16; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-      q.attrs = qa; q.numAttrs = 1;
-      int n_clusters = 0;
-      if (cudaOccupancyMaxActiveClusters(&n_clusters, attn_fused_kernel<HD>, &q) == cudaSuccess && n_clusters > 0)
-        max_cluster = 16;
-    }
-    (void)cudaGetLastError();
-  }
-  FusedAttnArgs args = a;
-  const int cta_x = a.nsplit * a.qsplit;
-  args.cluster = (cta_x >= 2 && cta_x <= max_cluster) ? 1 : 0;
-  if (args.cluster) {
+  if (a.nsplit > 1) {
     attr[na].id = cudaLaunchAttributeClusterDimension;
-    attr[na].val.clusterDim.x = (unsigned)cta_x; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+    attr[na].val.clusterDim.x = (unsigned)a.nsplit; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
     ++na;
   }
   cfg.attrs = attr; cfg.numAttrs = na;
-  return cudaLaunchKernelEx(&cfg, attn_fused_kernel<HD>, args);
+  return cudaLaunchKernelEx(&cfg, attn_tma_kernel<HD, QT>, *reinterpret_cast<const CUtensorMap *>(&kmap),
+                            *reinterpret_cast<const CUtensorMap *>(&vmap), a);
 }
 
-cudaError_t launch_attn_fused(const FusedAttnArgs &a, int hd, cudaStream_t st) {
-  if (hd == 64) return launch_fused_t<64>(a, st);
-  if (hd == 128) return launch_fused_t<128>(a, st);
+cudaError_t launch_attn_fused(const KvTensorMap &kmap, const KvTensorMap &vmap, const FusedAttnArgs &a, int hd, cudaStream_t st) {
+  if (a.nsplit < 1 || a.nsplit > 8 || a.c < 1 || a.c > 2 * kTK || !a.err) return cudaErrorInvalidValue;
+  if ((long long)a.hkv * (((a.hq / a.hkv) * a.c + 15) / 16) > 65535 || a.nb > 65535) return cudaErrorInvalidValue;
+  if (hd == 128) {
+    if (a.qt == 1) return launch_fused_t<128, 1>(kmap, vmap, a, st);
+    if (a.qt == 2) return launch_fused_t<128, 2>(kmap, vmap, a, st);
+    if (a.qt == 4) return launch_fused_t<128, 4>(kmap, vmap, a, st);
+  } else if (hd == 64) {
+    if (a.qt == 1) return launch_fused_t<64, 1>(kmap, vmap, a, st);
+    if (a.qt == 2) return launch_fused_t<64, 2>(kmap, vmap, a, st);
+    if (a.qt == 4) return launch_fused_t<64, 4>(kmap, vmap, a, st);
+  }
   return cudaErrorInvalidValue;
 }
 
-int attn_fused_chunk() { return kChunk; }
+int attn_fused_max_rows() { return 2 * kTK; }
 
 }  // namespace fc

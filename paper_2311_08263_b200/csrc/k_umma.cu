@@ -73,6 +73,7 @@ struct UmmaParams {
   unsigned int *bar;              // [n_phases - 1] grid-barrier counters, zero when the kernel starts
   unsigned int *claim;            // [n_phases] work-claim counters, zero when the kernel starts
   unsigned int *bar_b;            // [n_phases] panel-ready barriers (panel mode), zero when the kernel starts
+  ZeroList z;                     // buffers the epilogue warps clear once the previous kernel is complete
 };
 
 struct UmmaPlan {
@@ -727,6 +728,20 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     asm volatile("griddepcontrol.wait;" ::: "memory");   // outputs may still be read by the previous grid
     const int q = warp & 3;
     const int n_local = q * 32 + lane;
+    // Side clearing: buffers the previous kernel has finished reading and that a later phase of this launch (one
+    // that lies behind a grid barrier these warps arrive on) accumulates into.
+    {
+      const unsigned long long gtid = ((unsigned long long)blockIdx.x * 4 + q) * 32 + lane;
+      const unsigned long long nth = (unsigned long long)gridDim.x * 128;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (!p.z.p[i]) continue;
+        const unsigned long long n4 = p.z.n[i] >> 2;
+        float4 *p4 = reinterpret_cast<float4 *>(p.z.p[i]);
+        for (unsigned long long e = gtid; e < n4; e += nth) p4[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (unsigned long long e = (n4 << 2) + gtid; e < p.z.n[i]; e += nth) p.z.p[i][e] = 0.f;
+      }
+    }
     int seg = 0, sq = 0;
     bool ok = true;
     for (int pi = 0; pi < p.n_phases && ok; ++pi) {
@@ -969,7 +984,7 @@ static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, b
 // for the one before it.
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
                               unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,
-                              int td_stride, int pdl, cudaStream_t st) {
+                              int td_stride, const ZeroList *zero, int pdl, cudaStream_t st) {
   if (n < 1 || n > kMaxPhases || !claim) return cudaErrorInvalidValue;
   if (n > 1 && !bar) return cudaErrorInvalidValue;
   MapPack maps;
@@ -1044,6 +1059,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     maps.x[i] = plans[0]->xmap[0];
   }
   p.n_phases = n; p.pdl = pdl; p.err = plans[0]->err; p.bar = bar; p.claim = claim; p.bar_b = bar_b;
+  if (zero) p.z = *zero;
   // Staging warps own every fourth k-block and run ahead of each other; the parity waits on the ring
   // are only unambiguous while the ring is at least as deep as the number of staging warps.
   if (p.stages < 4 || p.stages > 8) return cudaErrorInvalidValue;
@@ -1053,9 +1069,9 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
   return launch_bn<EPI_ATOMIC_ADD>(maps, p, bn, panel, grid, st);
 }
 
-cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b, int pdl,
-                             cudaStream_t st) {
-  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, nullptr, 0, pdl, st);
+cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b,
+                             const ZeroList *zero, int pdl, cudaStream_t st) {
+  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, nullptr, 0, zero, pdl, st);
 }
 
 }  // namespace fc

@@ -55,19 +55,22 @@ def _case(hq, hkv, hd, c, lens, seed):
 
 
 CASES = [
-    # hq, hkv, hd, c, lens, chunks per CTA (0 = the step's choice)
-    (4, 4, 128, 16, [127, 128, 129, 0, 1], 0),        # MHA; lengths around a chunk edge, empty cache, one key
-    (8, 2, 64, 5, [260, 1, 2047], 0),                 # GQA, odd window, several chunks (cluster merge up to 16 CTAs)
+    # hq, hkv, hd, c, lens, splits per (sequence, kv head, query-tile group) (0 = the step's choice)
+    (4, 4, 128, 16, [127, 128, 129, 0, 1], 0),        # MHA; lengths around a tile edge, empty cache, one key
+    (4, 4, 128, 16, [63, 64, 65, 191, 192], 1),       # one CTA per head: every tile through the ring, ragged last tile
+    (8, 2, 64, 5, [260, 1, 2047], 0),                 # GQA, odd window, clusters of 8 splits, sequences with empty splits
     (4, 4, 128, 1, [77, 130, 2047], 0),               # c = 1: plain autoregressive attention
-    (8, 2, 64, 33, [300, 6000], 0),                   # 47 chunks per head: more than a cluster -> last-arriver merge
-    (4, 2, 128, 64, [513, 40], 0),                    # c = 64: the window spans chunk edges, 8 query tiles per kv head
-    (4, 4, 64, 16, [6000, 2047, 129], 4),             # forced: 4 consecutive chunks per CTA, running softmax statistics
-    (8, 2, 128, 16, [2047, 1], 3),                    # forced multi-chunk with grouped queries (2 query tiles)
+    (8, 2, 64, 33, [300, 6000], 0),                   # 94 tiles per head: long runs per CTA, 9 query tiles per kv head
+    (4, 2, 128, 64, [513, 40], 0),                    # c = 64: a full window tile, 8 query tiles per kv head
+    (4, 2, 128, 100, [513, 40], 2),                   # c = 100: two window tiles (the second ragged), as in a prefill block
+    (4, 4, 64, 16, [6000, 2047, 129], 4),             # forced: 4 splits, running softmax statistics over ~24 tiles each
+    (8, 2, 128, 16, [2047, 1], 3),                    # forced odd cluster size with grouped queries (2 query tiles)
+    (32, 32, 128, 16, [1000], 0),                     # the benchmark's attention shape: 32 heads, 4 splits of 4 tiles
 ]
 
 
-@pytest.mark.parametrize("hq,hkv,hd,c,lens,cpc", CASES)
-def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, cpc):
+@pytest.mark.parametrize("hq,hkv,hd,c,lens,splits", CASES)
+def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, splits):
     cfg, acc, ss, kc, vc, max_seq, want_attn, want_k, want_v = _case(hq, hkv, hd, c, lens, seed=40 + c)
     B = len(lens)
     kcd = kc.to(torch.bfloat16).cuda().contiguous()
@@ -75,7 +78,7 @@ def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, cpc):
     assert torch.equal(kcd.float().cpu(), kc)                   # the oracle's cached rows are bf16 values
     accd, ssd = acc.cuda().contiguous(), ss.cuda().contiguous()
     out = engine.fc_op_fused_window_attention(accd, ssd, cfg.rms_eps, cfg.d_model, cfg.rope_theta, kcd, vcd,
-                                              torch.tensor(lens, dtype=torch.int32).cuda(), c, hq, max(lens), cpc)
+                                              torch.tensor(lens, dtype=torch.int32).cuda(), c, hq, max(lens), splits)
     out = out.cpu().numpy().reshape(B, c, hq * hd)
     assert float(accd.abs().max()) == 0.0 and float(ssd.abs().max()) == 0.0      # consumed
     for b, L in enumerate(lens):
