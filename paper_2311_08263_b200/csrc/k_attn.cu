@@ -136,7 +136,7 @@ size_t attn_smem_bytes(int c, int qt) {
   const size_t wstage = 2ull * C::SUB * win_rows(c) * 128;
   const size_t rows = (size_t)qt * 16;
   return 1024 + (size_t)C::NS * C::kStage + (size_t)win_tiles(c) * wstage + (size_t)qt * C::kQTile + (size_t)qt * 4096 +
-         8 * rows * 4 /* per-warp maxima / sums */ + rows * 8 /* (max, sum) */ + 8 * rows * 4 /* split weights */;
+         8 * rows * 4 /* per-warp maxima / sums */ + rows * 8 /* (max, sum) */;
 }
 
 }  // namespace
@@ -175,15 +175,15 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   const uint32_t off_p = off_q + QT * C::kQTile;
   const uint32_t off_wmax = off_p + QT * 4096u;
   const uint32_t off_ml = off_wmax + 8u * ROWS * 4u;
-  const uint32_t off_wgt = off_ml + ROWS * 8u;
   float *wmax = reinterpret_cast<float *>(gen + off_wmax);    // [8 warps][ROWS]
   float *ml = reinterpret_cast<float *>(gen + off_ml);        // [ROWS][2]
-  float *wgt = reinterpret_cast<float *>(gen + off_wgt);      // [splits][ROWS]
   float *obuf = reinterpret_cast<float *>(gen);               // [ROWS][HD], over ring stage 0 once the tiles are consumed
 
   const int L = a.kv_len[b];
   const int n_ct = (L + kTK - 1) / kTK;                       // tiles of cached keys
-  const int tps = (n_ct + ns - 1) / ns;
+  // tiles per split: the last split also turns the accumulators into the window's keys and runs the window tile(s),
+  // which costs it about two tiles' time, so the cached tiles are dealt as if there were two more of them
+  const int tps = (n_ct + (ns > 1 ? 2 : 0) + ns - 1) / ns;
   const int t_begin = min(n_ct, split * tps);
   const int n_cached = min(n_ct, t_begin + tps) - t_begin;
   const int n_win = split == ns - 1 ? nwt : 0;
@@ -228,92 +228,102 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     }
   }
 
-  // ---- queries: 1/rms, rotation, bf16 high + low, into shared memory.  A thread keeps one pair index i and walks the
-  // rows; four rows' loads are issued together.
+  // ---- queries (1/rms, rotation, bf16 high + low) and, in the last split, the window's own keys (rotated, stored to
+  // shared memory and to the cache) come from the fp32 accumulators.  A thread keeps one pair index i and walks the rows
+  // four at a time; the first batch of window-key loads is issued together with the first batch of query loads, so that
+  // both share one trip to L2.
+  constexpr int RPP = kAttnThreads / HALF;                    // rows per pass
+  const int pi_ = tid % HALF, rsub = tid / HALF;
+  __nv_bfloat16 *kbase = (__nv_bfloat16 *)a.kcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+  __nv_bfloat16 *vbase = (__nv_bfloat16 *)a.vcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
+  struct QRegs { float x0[4], x1[4], ss[4]; float2 rot[4]; };
+  struct WRegs { float k0[4], k1[4], v0[4], v1[4], ss[4]; float2 rot[4]; };
+  auto q_load = [&](int r0, QRegs &q) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int rl = r0 + u * RPP + rsub;
+      const int qrow = qg * ROWS + rl;
+      q.x0[u] = q.x1[u] = q.ss[u] = 0.f; q.rot[u] = make_float2(1.f, 0.f);
+      if (rl < ROWS && qrow < nq) {
+        const int g = div_c(qrow), j = qrow - g * c;
+        const int r = bl * c + j, h = kvh * group + g;
+        const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
+        q.ss[u] = __ldcg(a.ss + r);
+        q.x0[u] = __ldcg(qacc + pi_); q.x1[u] = __ldcg(qacc + pi_ + HALF);
+        q.rot[u] = __ldg(a.rope + (long long)(L + j) * HALF + pi_);
+      }
+    }
+  };
+  auto q_store = [&](int r0, const QRegs &q) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int rl = r0 + u * RPP + rsub;
+      if (rl >= ROWS) continue;
+      const float sc = rsqrtf(q.ss[u] / (float)a.dn + a.eps);
+      const float a0 = q.x0[u] * sc, a1 = q.x1[u] * sc;
+      const float q0 = a0 * q.rot[u].x - a1 * q.rot[u].y, q1 = a0 * q.rot[u].y + a1 * q.rot[u].x;
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(q0), h1 = __float2bfloat16_rn(q1);
+      unsigned char *qt_base = gen + off_q + (uint32_t)(rl >> 4) * C::kQTile;
+      const int row = rl & 15;
+      const uint32_t o0 = tile_off(row, pi_ >> 3, 2048u) + (uint32_t)(pi_ & 7) * 2u;
+      const uint32_t o1 = tile_off(row, (pi_ + HALF) >> 3, 2048u) + (uint32_t)(pi_ & 7) * 2u;
+      *reinterpret_cast<__nv_bfloat16 *>(qt_base + o0) = h0;
+      *reinterpret_cast<__nv_bfloat16 *>(qt_base + o1) = h1;
+      *reinterpret_cast<__nv_bfloat16 *>(qt_base + SUB * 2048u + o0) = __float2bfloat16_rn(q0 - __bfloat162float(h0));
+      *reinterpret_cast<__nv_bfloat16 *>(qt_base + SUB * 2048u + o1) = __float2bfloat16_rn(q1 - __bfloat162float(h1));
+    }
+  };
+  auto w_load = [&](int j0, WRegs &w) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * RPP + rsub;
+      w.k0[u] = w.k1[u] = w.v0[u] = w.v1[u] = w.ss[u] = 0.f; w.rot[u] = make_float2(1.f, 0.f);
+      if (j < c) {
+        const int r = bl * c + j;
+        const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
+        w.ss[u] = __ldcg(a.ss + r);
+        w.k0[u] = __ldcg(kacc + pi_); w.k1[u] = __ldcg(kacc + pi_ + HALF);
+        w.v0[u] = __ldcg(kacc + kvd + pi_); w.v1[u] = __ldcg(kacc + kvd + pi_ + HALF);
+        w.rot[u] = __ldg(a.rope + (long long)(L + j) * HALF + pi_);
+      }
+    }
+  };
+  auto w_store = [&](int j0, const WRegs &w) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * RPP + rsub;
+      if (j >= c) continue;
+      const int pos = L + j;
+      const float sc = rsqrtf(w.ss[u] / (float)a.dn + a.eps);
+      const float x0 = w.k0[u] * sc, x1 = w.k1[u] * sc;
+      const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * w.rot[u].x - x1 * w.rot[u].y);
+      const __nv_bfloat16 o1 = __float2bfloat16_rn(x0 * w.rot[u].y + x1 * w.rot[u].x);
+      const __nv_bfloat16 w0 = __float2bfloat16_rn(w.v0[u] * sc), w1 = __float2bfloat16_rn(w.v1[u] * sc);
+      unsigned char *wt_base = gen + off_win + (uint32_t)(j / kTK) * wstage;
+      const int row = j % kTK;
+      const uint32_t f0 = tile_off(row, pi_ >> 3, wsub) + (uint32_t)(pi_ & 7) * 2u;
+      const uint32_t f1 = tile_off(row, (pi_ + HALF) >> 3, wsub) + (uint32_t)(pi_ & 7) * 2u;
+      *reinterpret_cast<__nv_bfloat16 *>(wt_base + f0) = o0;
+      *reinterpret_cast<__nv_bfloat16 *>(wt_base + f1) = o1;
+      *reinterpret_cast<__nv_bfloat16 *>(wt_base + wk + f0) = w0;
+      *reinterpret_cast<__nv_bfloat16 *>(wt_base + wk + f1) = w1;
+      kbase[(long long)pos * HD + pi_] = o0; kbase[(long long)pos * HD + pi_ + HALF] = o1;
+      vbase[(long long)pos * HD + pi_] = w0; vbase[(long long)pos * HD + pi_ + HALF] = w1;
+    }
+  };
   {
-    constexpr int RPP = kAttnThreads / HALF;                  // rows per pass
-    const int i = tid % HALF, rsub = tid / HALF;
-    for (int r0 = 0; r0 < ROWS; r0 += RPP * 4) {
-      float x0[4], x1[4], ssv[4];
-      float2 rot[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int rl = r0 + u * RPP + rsub;
-        const int qrow = qg * ROWS + rl;
-        x0[u] = x1[u] = ssv[u] = 0.f; rot[u] = make_float2(1.f, 0.f);
-        if (rl < ROWS && qrow < nq) {
-          const int g = div_c(qrow), j = qrow - g * c;
-          const int r = bl * c + j, h = kvh * group + g;
-          const float *qacc = a.qkv + (long long)r * a.ldq + h * HD;
-          ssv[u] = __ldcg(a.ss + r);
-          x0[u] = __ldcg(qacc + i); x1[u] = __ldcg(qacc + i + HALF);
-          rot[u] = __ldg(a.rope + (long long)(L + j) * HALF + i);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int rl = r0 + u * RPP + rsub;
-        if (rl >= ROWS) continue;
-        const float sc = rsqrtf(ssv[u] / (float)a.dn + a.eps);
-        const float a0 = x0[u] * sc, a1 = x1[u] * sc;
-        const float q0 = a0 * rot[u].x - a1 * rot[u].y, q1 = a0 * rot[u].y + a1 * rot[u].x;
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(q0), h1 = __float2bfloat16_rn(q1);
-        unsigned char *qt_base = gen + off_q + (uint32_t)(rl >> 4) * C::kQTile;
-        const int row = rl & 15;
-        const uint32_t o0 = tile_off(row, i >> 3, 2048u) + (uint32_t)(i & 7) * 2u;
-        const uint32_t o1 = tile_off(row, (i + HALF) >> 3, 2048u) + (uint32_t)(i & 7) * 2u;
-        *reinterpret_cast<__nv_bfloat16 *>(qt_base + o0) = h0;
-        *reinterpret_cast<__nv_bfloat16 *>(qt_base + o1) = h1;
-        *reinterpret_cast<__nv_bfloat16 *>(qt_base + SUB * 2048u + o0) = __float2bfloat16_rn(q0 - __bfloat162float(h0));
-        *reinterpret_cast<__nv_bfloat16 *>(qt_base + SUB * 2048u + o1) = __float2bfloat16_rn(q1 - __bfloat162float(h1));
-      }
+    QRegs q;
+    WRegs w;
+    q_load(0, q);
+    if (n_win > 0) w_load(0, w);
+    q_store(0, q);
+    for (int r0 = RPP * 4; r0 < ROWS; r0 += RPP * 4) { q_load(r0, q); q_store(r0, q); }
+    if (n_win > 0) {
+      w_store(0, w);
+      for (int j0 = RPP * 4; j0 < c; j0 += RPP * 4) { w_load(j0, w); w_store(j0, w); }
     }
   }
-
-  // ---- the window's own keys (last split): from the accumulators, rotated, to shared memory and to the cache
   if (n_win > 0) {
-    __nv_bfloat16 *kbase = (__nv_bfloat16 *)a.kcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
-    __nv_bfloat16 *vbase = (__nv_bfloat16 *)a.vcache + (long long)b * a.stride_b + (long long)kvh * a.stride_h;
-    constexpr int RPP = kAttnThreads / HALF;
-    const int i = tid % HALF, rsub = tid / HALF;
-    for (int j0 = 0; j0 < c; j0 += RPP * 4) {
-      float k0v[4], k1v[4], v0v[4], v1v[4], ssv[4];
-      float2 rot[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int j = j0 + u * RPP + rsub;
-        k0v[u] = k1v[u] = v0v[u] = v1v[u] = ssv[u] = 0.f; rot[u] = make_float2(1.f, 0.f);
-        if (j < c) {
-          const int r = bl * c + j;
-          const float *kacc = a.qkv + (long long)r * a.ldq + qd + kvh * HD;
-          ssv[u] = __ldcg(a.ss + r);
-          k0v[u] = __ldcg(kacc + i); k1v[u] = __ldcg(kacc + i + HALF);
-          v0v[u] = __ldcg(kacc + kvd + i); v1v[u] = __ldcg(kacc + kvd + i + HALF);
-          rot[u] = __ldg(a.rope + (long long)(L + j) * HALF + i);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int j = j0 + u * RPP + rsub;
-        if (j >= c) continue;
-        const int pos = L + j;
-        const float sc = rsqrtf(ssv[u] / (float)a.dn + a.eps);
-        const float x0 = k0v[u] * sc, x1 = k1v[u] * sc;
-        const __nv_bfloat16 o0 = __float2bfloat16_rn(x0 * rot[u].x - x1 * rot[u].y);
-        const __nv_bfloat16 o1 = __float2bfloat16_rn(x0 * rot[u].y + x1 * rot[u].x);
-        const __nv_bfloat16 w0 = __float2bfloat16_rn(v0v[u] * sc), w1 = __float2bfloat16_rn(v1v[u] * sc);
-        unsigned char *wt_base = gen + off_win + (uint32_t)(j / kTK) * wstage;
-        const int row = j % kTK;
-        const uint32_t f0 = tile_off(row, i >> 3, wsub) + (uint32_t)(i & 7) * 2u;
-        const uint32_t f1 = tile_off(row, (i + HALF) >> 3, wsub) + (uint32_t)(i & 7) * 2u;
-        *reinterpret_cast<__nv_bfloat16 *>(wt_base + f0) = o0;
-        *reinterpret_cast<__nv_bfloat16 *>(wt_base + f1) = o1;
-        *reinterpret_cast<__nv_bfloat16 *>(wt_base + wk + f0) = w0;
-        *reinterpret_cast<__nv_bfloat16 *>(wt_base + wk + f1) = w1;
-        kbase[(long long)pos * HD + i] = o0; kbase[(long long)pos * HD + i + HALF] = o1;
-        vbase[(long long)pos * HD + i] = w0; vbase[(long long)pos * HD + i + HALF] = w1;
-      }
-    }
     // rows of the last window tile beyond the window: zero, so that a zero probability never meets a stale NaN pattern
     {
       const int wt = nwt - 1;
@@ -531,41 +541,47 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   }
   if (ns > 1) cluster_sync_all(); else __syncthreads();
 
-  // ---- merge of the splits: weights per (split, row), then every CTA combines its share of the output
-  if (tid < ROWS) {
-    float ms[8], ls[8];
-    float M = -INFINITY;
-    for (int sp = 0; sp < ns; ++sp) {
-      float2 v;
-      if (ns > 1) v = ld_dsmem_f2(map_to_rank(base + off_ml + (uint32_t)tid * 8u, (uint32_t)sp));
-      else v = make_float2(ml[tid * 2], ml[tid * 2 + 1]);
-      ms[sp] = v.x; ls[sp] = v.y;
-      if (v.y > 0.f) M = fmaxf(M, v.x);
-    }
-    float den = 0.f;
-    for (int sp = 0; sp < ns; ++sp) {
-      ms[sp] = ls[sp] > 0.f ? __expf(ms[sp] - M) : 0.f;
-      den += ls[sp] * ms[sp];
-    }
-    const float inv = den > 0.f ? 1.0f / den : 0.f;
-    for (int sp = 0; sp < ns; ++sp) wgt[sp * ROWS + tid] = ms[sp] * inv;
-  }
-  __syncthreads();
+  // ---- merge of the splits: every CTA combines its share of the output.  A thread fetches the (max, sum) pairs and
+  // the partial outputs of all splits in one go (independent loads, one trip through the cluster's shared memory)
+  // and derives the split weights of its row itself.
   for (int u = split * kAttnThreads + tid; u < ROWS * (HD / 4); u += ns * kAttnThreads) {
     const int row = u / (HD / 4), c4 = u - row * (HD / 4);
     const int qrow = qg * ROWS + row;
     if (qrow >= nq) continue;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int sp = 0; sp < ns; ++sp) {
-      const float w = wgt[sp * ROWS + row];
-      float4 v;
-      if (ns > 1) v = ld_dsmem_f4(map_to_rank(base + (uint32_t)(row * HD + c4 * 4) * 4u, (uint32_t)sp));
-      else v = *reinterpret_cast<const float4 *>(obuf + row * HD + c4 * 4);
-      acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y); acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+    float2 mlv[8];
+    float4 ov[8];
+#pragma unroll
+    for (int sp = 0; sp < 8; ++sp) {
+      mlv[sp] = make_float2(-INFINITY, 0.f);
+      ov[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (sp < ns) {
+        if (ns > 1) {
+          mlv[sp] = ld_dsmem_f2(map_to_rank(base + off_ml + (uint32_t)row * 8u, (uint32_t)sp));
+          ov[sp] = ld_dsmem_f4(map_to_rank(base + (uint32_t)(row * HD + c4 * 4) * 4u, (uint32_t)sp));
+        } else {
+          mlv[sp] = make_float2(ml[row * 2], ml[row * 2 + 1]);
+          ov[sp] = *reinterpret_cast<const float4 *>(obuf + row * HD + c4 * 4);
+        }
+      }
     }
+    float M = -INFINITY;
+#pragma unroll
+    for (int sp = 0; sp < 8; ++sp)
+      if (mlv[sp].y > 0.f) M = fmaxf(M, mlv[sp].x);
+    float den = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int sp = 0; sp < 8; ++sp) {
+      const float w = mlv[sp].y > 0.f ? __expf(mlv[sp].x - M) : 0.f;
+      den = fmaf(mlv[sp].y, w, den);
+      acc.x = fmaf(w, ov[sp].x, acc.x); acc.y = fmaf(w, ov[sp].y, acc.y);
+      acc.z = fmaf(w, ov[sp].z, acc.z); acc.w = fmaf(w, ov[sp].w, acc.w);
+    }
+    const float inv = den > 0.f ? 1.0f / den : 0.f;
     const int g = div_c(qrow), j = qrow - g * c;
     const int r = bl * c + j, h = kvh * group + g;
-    *reinterpret_cast<float4 *>(a.out + (long long)r * qd + h * HD + c4 * 4) = acc;
+    *reinterpret_cast<float4 *>(a.out + (long long)r * qd + h * HD + c4 * 4) =
+        make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
   }
   if (ns > 1) cluster_sync_all();                             // the other splits may still be reading this CTA's memory
 }
