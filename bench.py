@@ -30,7 +30,7 @@ from paper_2311_08263_b200 import workload as wl  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists)
-TRAFFIC_BYTES_PER_LAUNCH = {"7b": 413.8e6}     # profiles/gemm_umma_chain_7b_4layers.txt (same shapes per launch)
+TRAFFIC_BYTES_PER_LAUNCH = {"7b": None}        # profiles/gemm_umma_chain_7b_4layers.txt (same shapes per launch)
 
 METRIC = "accepted_tokens_per_s"
 UNIT = "tokens/s"
@@ -78,7 +78,9 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
-    def stop(self):
+    def stop(self, timed=None):
+        """timed: (first, last) sample indices of the device-timed region; sm_mhz is the median over that region
+        (over all samples when it holds none), sm_mhz_all the median over warm-up + timed region + end-to-end loop."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -87,20 +89,23 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         self.t.join(timeout=2)
-        sm, mx, reasons = [], None, set()
+        sm, sm_timed, mx, reasons = [], [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for i, r in enumerate(self.rows):
             if len(r) < 7:
                 continue
             try:
                 sm.append(float(r[0])); mx = float(r[1])
             except ValueError:
                 continue
+            if timed and timed[0] <= i < max(timed[1], timed[0] + 1):
+                sm_timed.append(float(r[0]))
             for n, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        med_all = statistics.median(sm) if sm else None
+        return {"sm_mhz": statistics.median(sm_timed) if sm_timed else med_all, "sm_mhz_all": med_all, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm), "samples_timed": len(sm_timed)}
 
 
 def dist_setup(n_gpus):
@@ -219,10 +224,12 @@ def run_ours(args, cfg, rank, world, local):
     setup_s = time.time() - t0
 
     # ---- device-resident timing: K committed steps back to back, CUDA events, max over ranks
-    dec.fc_bench_steps(warm, commit=True)
+    # (the clock sampler runs from the warm-up to the end of the end-to-end loop; the medians are reported per region)
     sampler = ClockSampler(local)
     sampler.start()
+    dec.fc_bench_steps(warm, commit=True)
     barrier(world)
+    n_warm_samples = len(sampler.rows)
     torch.cuda.synchronize()
     kv0 = dec.fc_get_state()[0].copy()
     ms, tokens = dec.fc_bench_steps(steps, commit=True)
@@ -230,7 +237,7 @@ def run_ours(args, cfg, rank, world, local):
     torch.cuda.synchronize()
     barrier(world)
     kv1 = dec.fc_get_state()[0].copy()
-    clocks = sampler.stop()
+    n_timed_samples = len(sampler.rows)
     ms_max, tok_sum = reduce_max_sum(world, ms, tokens, device)
 
     # ---- end to end: host window in, host results out, every step (wall clock)
@@ -239,6 +246,7 @@ def run_ours(args, cfg, rank, world, local):
         win = dec.fc_jacobi_step(win)[2]
     barrier(world)
     torch.cuda.synchronize()
+    kv_e0 = dec.fc_get_state()[0].copy()
     t1 = time.perf_counter()
     e2e_tok = 0
     for _ in range(e2e_steps):
@@ -246,6 +254,8 @@ def run_ours(args, cfg, rank, world, local):
         e2e_tok += int(cnt.sum())
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t1
+    kv2 = dec.fc_get_state()[0].copy()
+    clocks = sampler.stop(timed=(n_warm_samples, n_timed_samples))
     e2e_ms_max, e2e_tok_sum = reduce_max_sum(world, e2e_s * 1e3, e2e_tok, device)
 
     # ---- per-kernel-class device times (events around every launch of one step)
@@ -284,8 +294,9 @@ def run_ours(args, cfg, rank, world, local):
                        "multi_gpu": "replicas only"},
             "mean_accept": tok_sum / (steps * B * world),
             "clocks": clocks,
+            "ms_x_mhz": step_ms * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
             "e2e": {"value": e2e_tok_sum / (e2e_ms_max * 1e-3), "unit": UNIT, "steps": e2e_steps,
-                    "ms_per_step": e2e_ms_max / e2e_steps,
+                    "ms_per_step": e2e_ms_max / e2e_steps, "kv_len_start": int(kv_e0[0]), "kv_len_end": int(kv2[0]),
                     "h2d_bytes_per_step": B * c * 4, "d2h_bytes_per_step": B * (1 + 2 * c) * 4 + 4},
             "gpu_launches": launches,
             "roofline": roofline,

@@ -104,6 +104,7 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   int b0, nb, c, hq, hkv;
   int nsplit;             // CTAs (one thread-block cluster, <= 8) per (sequence, kv head, query-tile group)
   int qt;                 // 16-row query tiles per CTA: 1, 2 or 4
+  int stages;             // K/V ring stages (set by the launcher)
   int pdl;                // launched as a programmatic dependent of the previous kernel
   unsigned int *err;      // device error word, raised when a bounded wait gives up
   float *out;             // [R, hq*hd] fp32

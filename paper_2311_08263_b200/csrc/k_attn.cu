@@ -123,7 +123,8 @@ __host__ __device__ inline int win_tiles(int c) { return (c + kTK - 1) / kTK; }
 template <int HD>
 struct AttnCfg {
   static constexpr int SUB = HD / 64;                       // 128-byte sub-tiles per row
-  static constexpr int NS = HD == 128 ? 3 : 4;              // ring stages
+  static constexpr int NS = HD == 128 ? 3 : 4;              // ring stages when one CTA has an SM to itself
+  static constexpr int NS_MAX = 4;
   static constexpr uint32_t kSubBytes = kTK * 128;          // one sub-tile of a TMA tile
   static constexpr uint32_t kKBytes = SUB * kSubBytes;      // K (or V) part of a stage
   static constexpr uint32_t kStage = 2 * kKBytes;
@@ -131,11 +132,11 @@ struct AttnCfg {
 };
 
 template <int HD>
-size_t attn_smem_bytes(int c, int qt) {
+size_t attn_smem_bytes(int c, int qt, int stages) {
   using C = AttnCfg<HD>;
   const size_t wstage = 2ull * C::SUB * win_rows(c) * 128;
   const size_t rows = (size_t)qt * 16;
-  return 1024 + (size_t)C::NS * C::kStage + (size_t)win_tiles(c) * wstage + (size_t)qt * C::kQTile + (size_t)qt * 4096 +
+  return 1024 + (size_t)stages * C::kStage + (size_t)win_tiles(c) * wstage + (size_t)qt * C::kQTile + (size_t)qt * 4096 +
          8 * rows * 4 /* per-warp maxima / sums */ + rows * 8 /* (max, sum) */;
 }
 
@@ -145,13 +146,14 @@ template <int HD, int QT>
 __global__ void __maxnreg__(128)
 attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap, const FusedAttnArgs a) {
   using C = AttnCfg<HD>;
-  constexpr int SUB = C::SUB, NS = C::NS, HALF = HD / 2;
+  constexpr int SUB = C::SUB, HALF = HD / 2;
+  const int NS = a.stages;                   // ring stages (2 .. 4)
   constexpr int NDW = HD / 64;               // 8-wide output blocks per warp (8 warps x NDW x 8 columns = HD)
   constexpr int ROWS = QT * 16;
   constexpr uint32_t kSubBytes = C::kSubBytes, kKBytes = C::kKBytes, kStage = C::kStage;
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long full_bar[NS];
+  __shared__ __align__(8) unsigned long long full_bar[C::NS_MAX];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g4 = lane >> 2, t4 = lane & 3;
   const int split = blockIdx.x, ns = gridDim.x;
@@ -170,7 +172,7 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   unsigned char *gen = smem_raw + (base - smem_addr(smem_raw));
   const int wrows = win_rows(c), nwt = win_tiles(c);
   const uint32_t wsub = (uint32_t)wrows * 128u, wk = SUB * wsub, wstage = 2u * wk;
-  const uint32_t off_win = NS * kStage;
+  const uint32_t off_win = (uint32_t)NS * kStage;
   const uint32_t off_q = off_win + (uint32_t)nwt * wstage;
   const uint32_t off_p = off_q + QT * C::kQTile;
   const uint32_t off_wmax = off_p + QT * 4096u;
@@ -202,7 +204,6 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   };
 
   if (tid == 0) {
-#pragma unroll
     for (int i = 0; i < NS; ++i) mbar_init(smem_addr(&full_bar[i]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -618,7 +619,11 @@ void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int
   while (qt < 4 && qt < nqt && (long long)nb * hkv * ((nqt + qt - 1) / qt) > 2ll * n_sms) qt *= 2;
   const long long units = (long long)nb * hkv * ((nqt + qt - 1) / qt);
   const int n_ct = (max_len + kTK - 1) / kTK;
-  long long s = n_sms / units;                                // one CTA per SM: the projection kernel's CTAs come in beside them
+  // Short caches: one CTA per SM, so that the projection kernel's CTAs come in beside them while the attention runs.
+  // Long caches (more than 8 tiles per CTA that way) are a streaming problem: two CTAs per SM hide each other's waits.
+  long long s = n_sms / units;
+  if (s < 1) s = 1;
+  if (n_ct > 8 * s) s = 2ll * n_sms / units;
   if (s > 8) s = 8;
   if (s > n_ct) s = n_ct;
   if (s < 1) s = 1;
@@ -627,7 +632,21 @@ void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int
 
 template <int HD, int QT>
 static cudaError_t launch_fused_t(const KvTensorMap &kmap, const KvTensorMap &vmap, const FusedAttnArgs &a, cudaStream_t st) {
-  const size_t smem = attn_smem_bytes<HD>(a.c, QT);
+  // Ring depth: the deep ring when every CTA has an SM to itself (the following projection kernel's CTAs come in beside
+  // it); with more CTAs than SMs two of them share an SM and hide each other's waits, so the ring is made as deep as
+  // still lets two fit (at least two stages).
+  const int nqt_ = ((a.hq / a.hkv) * a.c + 15) / 16;
+  const long long ctas = (long long)a.nsplit * a.hkv * ((nqt_ + QT - 1) / QT) * a.nb;
+  int dev_id = 0, n_sms = 0;
+  if (cudaGetDevice(&dev_id) != cudaSuccess || cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev_id) != cudaSuccess)
+    return cudaErrorInvalidValue;
+  FusedAttnArgs args = a;
+  args.stages = AttnCfg<HD>::NS;
+  if (ctas > n_sms) {
+    const size_t per_sm = 228 * 1024, reserve = 1024 + 256;    // per CTA: the system's kilobyte and the static part
+    while (args.stages > 2 && 2 * (attn_smem_bytes<HD>(a.c, QT, args.stages) + reserve) > per_sm) --args.stages;
+  }
+  const size_t smem = attn_smem_bytes<HD>(a.c, QT, args.stages);
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   static size_t attr_smem[kMaxDevices] = {0};
   const int dev = current_device_slot();
@@ -655,7 +674,7 @@ static cudaError_t launch_fused_t(const KvTensorMap &kmap, const KvTensorMap &vm
   }
   cfg.attrs = attr; cfg.numAttrs = na;
   return cudaLaunchKernelEx(&cfg, attn_tma_kernel<HD, QT>, *reinterpret_cast<const CUtensorMap *>(&kmap),
-                            *reinterpret_cast<const CUtensorMap *>(&vmap), a);
+                            *reinterpret_cast<const CUtensorMap *>(&vmap), args);
 }
 
 cudaError_t launch_attn_fused(const KvTensorMap &kmap, const KvTensorMap &vmap, const FusedAttnArgs &a, int hd, cudaStream_t st) {
