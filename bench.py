@@ -30,7 +30,7 @@ from paper_2311_08263_b200 import workload as wl  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of the current kernel exists)
-TRAFFIC_BYTES_PER_LAUNCH = {"7b": None}        # profiles/gemm_umma_chain_7b_4layers.txt (same shapes per launch)
+TRAFFIC_BYTES_PER_LAUNCH = {"7b": 415.7e6}     # profiles/gemm_umma_chain_7b_4layers.txt (same shapes per launch)
 
 METRIC = "accepted_tokens_per_s"
 UNIT = "tokens/s"
