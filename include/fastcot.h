@@ -107,7 +107,10 @@ int fc_prefill(fc_ctx *ctx, int32_t batch, const int32_t *prompt_ids, int32_t p_
 /* One Jacobi-window iteration for every live sequence (Eq. 4, Eq. 5, cache update).
  * window_in: host [batch, c] or NULL (keep the internal window); slot 0 of each row must be the
  * pending exact token.  Outputs (host, each nullable): accepted_count [batch] (k in [1, c]; 0 for a
- * finished sequence), accepted_tokens [batch, c] (first k valid), window_out [batch, c]. */
+ * finished sequence), accepted_tokens [batch, c] (first k valid), window_out [batch, c].
+ * Sequences that fc_generate has finished (max_tokens reached or EOS) take no rows of the forward: the step
+ * runs over the live sequences only (the paper's "Time Analysis" counts what padded, finished batch members
+ * cost; here they cost nothing). */
 int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *accepted_count,
                    int32_t *accepted_tokens, int32_t *window_out);
 

@@ -45,7 +45,9 @@ struct Buffers {
   unsigned int *counters, *err, *chain_bar;
   unsigned long long *amax;
   int32_t *window, *kv_len, *n_gen, *done, *acc_count, *acc_tokens, *prompt, *prompt_lens, *out_tokens;
-  int32_t *row_tokens;     // tokens of a forward that is not a decode step (answer-trigger context)
+  int32_t *row_tokens;     // tokens of a forward that is not a plain decode step (answer-trigger context; the windows of
+                           // the live sequences when finished ones are skipped)
+  int32_t *seq_map;        // [max_batch] the live sequences of a compacted step
 };
 
 struct Dims {
@@ -120,7 +122,8 @@ size_t carve(const fc_model_shape *s, char *base, Buffers *b, std::vector<size_t
   t.prompt = c.take<int32_t>((size_t)s->max_batch * s->max_seq);
   t.prompt_lens = c.take<int32_t>(s->max_batch);
   t.out_tokens = c.take<int32_t>((size_t)s->max_batch * s->max_seq);
-  t.row_tokens = c.take<int32_t>(R); c.guard();
+  t.row_tokens = c.take<int32_t>(R);
+  t.seq_map = c.take<int32_t>(s->max_batch); c.guard();
   if (b) *b = t;
   return c.off;
 }
@@ -162,6 +165,7 @@ struct fc_ctx {
   std::vector<size_t> guards;    // offsets of the canary bands inside the workspace
   // pinned staging: [count | tokens | window | err]
   int32_t *pin = nullptr;
+  int32_t *pin_map = nullptr;    // pinned [max_batch]: the live sequences of a compacted step
   int64_t launches = 0;
   char cuda_err[256] = {0};
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -223,6 +227,7 @@ extern "C" void fc_destroy(fc_ctx *ctx) {
   if (!ctx) return;
   destroy_plans(ctx);
   if (ctx->pin) cudaFreeHost(ctx->pin);
+  if (ctx->pin_map) cudaFreeHost(ctx->pin_map);
   if (ctx->ev0) cudaEventDestroy(ctx->ev0);
   if (ctx->ev1) cudaEventDestroy(ctx->ev1);
   delete ctx;
@@ -368,6 +373,7 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   }
   const size_t pin_ints = (size_t)shape->max_batch * (1 + 2 * shape->max_c) + 4;
   if (cudaMallocHost((void **)&ctx->pin, pin_ints * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
+  if (cudaMallocHost((void **)&ctx->pin_map, (size_t)shape->max_batch * sizeof(int32_t)) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaEventCreate(&ctx->ev0) != cudaSuccess || cudaEventCreate(&ctx->ev1) != cudaSuccess) return fail(FC_ERR_CUDA);
   if (cudaMemsetAsync(ws, 0, fc_workspace_bytes(shape), ctx->st) != cudaSuccess) return fail(FC_ERR_CUDA);
   for (size_t off : ctx->guards)      // canary bands between the slices (checked by fc_debug_check_guards)
@@ -432,8 +438,9 @@ static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R
 
 // One decoder forward over nb sequences (b0 .. b0+nb-1) with `rows` rows each.  tokens: device [nb*rows].
 // with_head: LM head + argmax + accept (a decode step); otherwise the rows are committed (prefill chunk).
+// seq_map (device, optional): row block i belongs to sequence seq_map[i] instead of b0 + i (finished sequences skipped).
 static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens, bool with_head, int max_len_host,
-                   int commit) {
+                   int commit, const int32_t *seq_map = nullptr) {
   const fc_model_shape &s = ctx->s;
   const Dims &d = ctx->d;
   const int R = nb * rows;
@@ -464,6 +471,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       fa.kcache = kc; fa.vcache = vc; fa.stride_b = stride_b; fa.stride_h = stride_h;
       fa.k_plane0 = (l * 2) * s.max_batch * s.n_kv_heads; fa.v_plane0 = (l * 2 + 1) * s.max_batch * s.n_kv_heads;
       fa.kv_len = ctx->b.kv_len; fa.b0 = b0; fa.nb = nb; fa.c = rows; fa.hq = s.n_heads; fa.hkv = s.n_kv_heads;
+      fa.seq_map = seq_map;
       fused_attn_plan(max_len_host, rows, s.n_heads, s.n_kv_heads, nb, ctx->n_sms, fa.nsplit, fa.qt);
       fa.err = ctx->b.err;
       fa.out = ctx->b.attn; fa.pdl = ctx->pdl && !ctx->prof;
@@ -474,7 +482,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     } else {
       RopeArgs ra; memset(&ra, 0, sizeof ra);
       ra.qkv = ctx->b.qkv; ra.ldq = d.ldq; ra.ss = ctx->b.ss_attn; ra.eps = s.rms_eps; ra.dn = s.d_model;
-      ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows;
+      ra.kv_len = ctx->b.kv_len; ra.b0 = b0; ra.nb = nb; ra.c = rows; ra.seq_map = seq_map;
       ra.hq = s.n_heads; ra.hkv = s.n_kv_heads; ra.hd = s.head_dim; ra.rope = ctx->b.rope;
       ra.q_out = ctx->b.qb; ra.kcache = kc; ra.vcache = vc;
       ra.stride_b = stride_b; ra.stride_h = stride_h;
@@ -485,6 +493,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       AttnArgs aa; memset(&aa, 0, sizeof aa);
       aa.q = ctx->b.qb; aa.kcache = kc; aa.vcache = vc; aa.stride_b = stride_b; aa.stride_h = stride_h;
       aa.kv_len = ctx->b.kv_len; aa.b0 = b0; aa.nb = nb; aa.c = rows; aa.hq = s.n_heads; aa.hkv = s.n_kv_heads;
+      aa.seq_map = seq_map;
       aa.nsplit = nsplit; aa.part_o = ctx->b.part_o; aa.part_ml = ctx->b.part_ml; aa.counters = ctx->b.counters;
       aa.out = ctx->b.attn;
       aa.z.p[0] = ctx->b.ss_attn; aa.z.n[0] = Rz;
@@ -544,6 +553,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
     ac.prompt = ctx->b.prompt; ac.prompt_lens = ctx->b.prompt_lens;
     ac.out_tokens = ctx->b.out_tokens; ac.out_stride = s.max_seq;
     ac.b0 = b0; ac.nb = nb; ac.c = rows; ac.p_stride = s.max_seq; ac.refill = ctx->refill; ac.pad_id = ctx->pad_id;
+    ac.seq_map = seq_map;
     ac.max_tokens = ctx->gen_max_tokens; ac.eos_id = ctx->gen_eos; ac.commit = commit;
     if (ctx->inject_timeout) { ac.err_inject = ctx->b.err; ctx->inject_timeout = false; }
     ++ctx->launches;
@@ -653,6 +663,7 @@ static int collect_step(fc_ctx *ctx, int32_t *accepted_count, int32_t *accepted_
     return FC_ERR_DEVICE_TIMEOUT;
   }
   for (int b = 0; b < B; ++b) {
+    if (ctx->done_h[b]) p_cnt[b] = 0;         // skipped by the step: the device word is from its last live step
     const int k = p_cnt[b];
     ctx->kv_len_h[b] += k; ctx->n_gen_h[b] += k; ctx->pending_h[b] = p_win[(size_t)b * c];
     if (k > 0) {
@@ -670,6 +681,25 @@ static int max_live_len(const fc_ctx *ctx) {
   int m = 0;
   for (int b = 0; b < ctx->batch; ++b) m = ctx->kv_len_h[b] > m ? ctx->kv_len_h[b] : m;
   return m;
+}
+
+// One decode forward over the sequences that are not finished (paper, "Time Analysis": a batch member that is done
+// otherwise keeps costing rows of every projection and its attention).  With every sequence live this is the plain
+// forward over the windows; otherwise the live sequences' windows are gathered into consecutive rows and the kernels
+// that touch per-sequence state (attention, accept) go through a map from row block to sequence.
+static int decode_forward(fc_ctx *ctx) {
+  const int B = ctx->batch, c = ctx->c;
+  int n_live = 0, maxlen = 0;
+  for (int b = 0; b < B; ++b)
+    if (!ctx->done_h[b]) {
+      ctx->pin_map[n_live++] = b;
+      maxlen = ctx->kv_len_h[b] > maxlen ? ctx->kv_len_h[b] : maxlen;
+    }
+  if (n_live == B || n_live == 0) return forward(ctx, 0, B, c, ctx->b.window, true, max_live_len(ctx), 1);
+  FC_CK(cudaMemcpyAsync(ctx->b.seq_map, ctx->pin_map, sizeof(int32_t) * n_live, cudaMemcpyHostToDevice, ctx->st));
+  ++ctx->launches;
+  FC_CK(launch_gather_rows(ctx->b.row_tokens, ctx->b.window, ctx->b.seq_map, n_live, c, ctx->st));
+  return forward(ctx, 0, n_live, c, ctx->b.row_tokens, true, maxlen, 1, ctx->b.seq_map);
 }
 
 extern "C" int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *accepted_count,
@@ -691,7 +721,7 @@ extern "C" int fc_jacobi_step(fc_ctx *ctx, const int32_t *window_in, int32_t *ac
     FC_CK(cudaMemcpyAsync(ctx->b.window, ctx->pin, sizeof(int32_t) * B * c, cudaMemcpyHostToDevice, ctx->st));
   }
   ctx->launches = 0;
-  int rc = forward(ctx, 0, B, c, ctx->b.window, true, max_live_len(ctx), 1);
+  int rc = decode_forward(ctx);
   if (rc != FC_OK) return rc;
   return collect_step(ctx, accepted_count, accepted_tokens, window_out);
 }
@@ -765,7 +795,7 @@ extern "C" int fc_generate(fc_ctx *ctx, int32_t max_tokens, int32_t c, int32_t e
     if (!live) break;
     if (max_iters > 0 && iters >= max_iters) break;       // iteration cap ("Iteration Stop Condition", condition 1)
     ctx->launches = 0;
-    rc = forward(ctx, 0, B, c, ctx->b.window, true, max_live_len(ctx), 1);
+    rc = decode_forward(ctx);
     if (rc != FC_OK) break;
     launches += ctx->launches;
     rc = collect_step(ctx, cnt.data(), tok.data(), nullptr);

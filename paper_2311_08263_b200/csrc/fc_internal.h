@@ -64,7 +64,8 @@ struct RopeArgs {
   const float *ss;        // [R] sums of squares for the 1/rms factor
   float eps; int dn;
   const int32_t *kv_len;  // [batch] device
-  int b0, nb, c;          // rows r = (b - b0) * c + j
+  const int32_t *seq_map; // optional [nb] device: the sequence behind row block i (null: b0 + i)
+  int b0, nb, c;          // rows r = i * c + j for row block i
   int hq, hkv, hd;
   const float2 *rope;     // [max_seq][hd/2] (cos, sin) of position * theta^(-2i/hd), built on the host
   void *q_out;            // [R, hq*hd] in the cache dtype
@@ -78,6 +79,7 @@ struct AttnArgs {
   const void *kcache, *vcache;
   long long stride_b, stride_h;
   const int32_t *kv_len;
+  const int32_t *seq_map; // optional [nb] device: the sequence behind row block i (null: b0 + i)
   int b0, nb, c, hq, hkv;
   int nsplit;
   float *part_o;          // [R*hq, nsplit, hd]
@@ -101,6 +103,7 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   int k_plane0, v_plane0; // plane (= [max_seq][hd] matrix of one sequence and kv head) of sequence 0, kv head 0 in the
                           // K and the V tensor map: cached tiles are fetched by TMA from plane0 + b * hkv + kvh
   const int32_t *kv_len;
+  const int32_t *seq_map; // optional [nb] device: the sequence behind row block i (null: b0 + i)
   int b0, nb, c, hq, hkv;
   int nsplit;             // CTAs (one thread-block cluster, <= 8) per (sequence, kv head, query-tile group)
   int qt;                 // 16-row query tiles per CTA: 1, 2 or 4
@@ -122,6 +125,8 @@ struct AcceptArgs {
   int32_t *out_tokens;             // [batch, out_stride] or null
   int out_stride;
   int b0, nb, c, p_stride, refill, pad_id;
+  const int32_t *seq_map;          // optional [nb] device: the sequence behind row block i (null: b0 + i); rows of the
+                                   // forward (amax / argmax) are indexed by row block, sequence state by sequence
   int max_tokens, eos_id;          // max_tokens <= 0: unlimited
   int commit;                      // 0: leave kv_len / n_gen / window untouched (latency measurement)
   unsigned int *err_inject;        // test aid: when non-null the kernel raises this error word (no wait involved)
@@ -156,6 +161,8 @@ cudaError_t make_kv_tensor_map(KvTensorMap *out, const void *base, int hd, int m
 void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int &nsplit, int &qt);
 int attn_fused_max_rows();   // most window rows per sequence the fused kernel takes in one launch
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
+// dst[i * c + j] = window[seq_map[i] * c + j]: the token rows of a forward over the sequences seq_map[0 .. nb-1]
+cudaError_t launch_gather_rows(int32_t *dst, const int32_t *window, const int32_t *seq_map, int nb, int c, cudaStream_t st);
 int attn_tile_keys(int dtype, int hd);   // keys per split tile
 
 // Standalone window attention on caller-supplied scratch (shared by the op-level entry points).

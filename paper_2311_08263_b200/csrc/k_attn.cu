@@ -161,7 +161,7 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   const int nq = group * a.c;
   const int nqg = ((nq + 15) / 16 + QT - 1) / QT;
   const int kvh = blockIdx.y / nqg, qg = blockIdx.y - kvh * nqg;
-  const int bl = blockIdx.z, b = a.b0 + bl;
+  const int bl = blockIdx.z, b = a.seq_map ? a.seq_map[bl] : a.b0 + bl;
   const int c = a.c;
   const int qd = a.hq * HD, kvd = a.hkv * HD;
   const unsigned int c_magic = a.c_magic;

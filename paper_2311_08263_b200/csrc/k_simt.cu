@@ -161,7 +161,7 @@ __global__ void rope_kv_kernel(RopeArgs a) {
     const int i = (int)(t % half);
     const int h = (int)((t / half) % heads);
     const int r = (int)(t / ((long long)half * heads));
-    const int b = a.b0 + r / a.c, j = r % a.c;
+    const int b = a.seq_map ? a.seq_map[r / a.c] : a.b0 + r / a.c, j = r % a.c;
     const int pos = a.kv_len[b] + j;
     const float s = rsqrtf(a.ss[r] / (float)a.dn + a.eps);
     float *src = a.qkv + (long long)r * a.ldq + (long long)h * a.hd;
@@ -211,7 +211,7 @@ __global__ void __launch_bounds__(256) attn_window_kernel(AttnArgs a) {
   __shared__ unsigned int s_last;
 
   const int split = blockIdx.x, kvh = blockIdx.y, bl = blockIdx.z;
-  const int b = a.b0 + bl;
+  const int b = a.seq_map ? a.seq_map[bl] : a.b0 + bl;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int L = a.kv_len[b];
   const int ltot = L + a.c;
@@ -369,7 +369,7 @@ cudaError_t launch_attn(const AttnArgs &a, int dtype, int hd, cudaStream_t st) {
 __global__ void accept_kernel(AcceptArgs a) {
   const int bl = blockIdx.x * blockDim.x + threadIdx.x;
   if (bl >= a.nb) return;
-  const int b = a.b0 + bl, c = a.c;
+  const int b = a.seq_map ? a.seq_map[bl] : a.b0 + bl, c = a.c;
   int32_t *w = a.window + (long long)b * c;
   int32_t arg[64];
   for (int j = 0; j < c; ++j) {
@@ -413,6 +413,16 @@ __global__ void accept_kernel(AcceptArgs a) {
                                                           : a.prompt[(long long)b * a.p_stride + (n1 + j - 1) % P];
   }
   for (int j = 0; j < c; ++j) w[j] = nw[j];
+}
+
+__global__ void gather_rows_kernel(int32_t *dst, const int32_t *window, const int32_t *seq_map, int nb, int c) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < nb * c) dst[i] = window[(long long)seq_map[i / c] * c + i % c];
+}
+
+cudaError_t launch_gather_rows(int32_t *dst, const int32_t *window, const int32_t *seq_map, int nb, int c, cudaStream_t st) {
+  gather_rows_kernel<<<(nb * c + 255) / 256, 256, 0, st>>>(dst, window, seq_map, nb, c);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st) {

@@ -491,3 +491,55 @@ def test_bf16_step_run_to_run_spread_is_bounded(flags):
             ref = lg
         spread = max(spread, float((lg - ref).abs().max()))
     assert spread < 3e-4, spread
+
+
+@pytest.mark.parametrize("kind", ["fp32", "bf16"])
+def test_finished_sequences_are_skipped_and_the_others_unaffected(kind):
+    """A batch in which sequences finish at different times (one on an EOS early in its stream, the others at
+    max_tokens): finished sequences no longer take rows of the forward - the step runs over the live ones only,
+    through a map from row block to sequence - and every stream still equals the oracle's autoregressive stream.
+    The launch count shows the compacted steps (one extra gather launch each); a step after the end reports 0."""
+    if kind == "fp32":
+        cfg = wl.CONFIGS["tiny"]
+        c, n_gen = 4, 24
+    else:
+        cfg = wl.small_config(vocab=600, n_layers=2, n_heads=4, n_kv_heads=2, head_dim=64, d_model=256, d_ffn=512,
+                              prompt_len=70, c=6, gen_tokens=20)
+        c, n_gen = cfg.c, cfg.gen_tokens
+    B = 4
+    lens = [40, 33, 7, 25] if kind == "fp32" else [70, 33, 1, 50]
+    w = wl.make_weights(cfg)
+    max_seq = max(lens) + n_gen + c + 8
+    dec = engine.Decoder(cfg, w, B, c, max_seq)
+    ids, _ = wl.make_prompts(cfg, batch=B, lens=lens)
+    ars, margins = [], []
+    for b in range(B):
+        o = oracle.Oracle(cfg, w, max_seq)
+        ar, m = o.ar_generate(ids[b, :lens[b]].numpy(), n_gen)
+        ars.append(ar); margins.append(m)
+        o.close()
+    # an EOS that ends sequence 1 after a few tokens and occurs nowhere in the other streams
+    eos = next(int(t) for t in ars[1][3:10] if all(int(t) not in ars[b].tolist() for b in (0, 2, 3)))
+    want = [ar[:ar.tolist().index(eos) + 1] if eos in ar.tolist() else ar for ar in ars]
+    assert len(want[1]) < n_gen and all(len(want[b]) == n_gen for b in (0, 2, 3))
+    dec.fc_prefill(ids.numpy(), lens, c)
+    toks, out_lens, st = dec.fc_generate(n_gen, eos_id=eos)
+    for b in range(B):
+        got = toks[b, :out_lens[b]]
+        if kind == "fp32":
+            assert got.tolist() == want[b].tolist(), b
+        else:
+            n = min(len(got), len(want[b]))
+            diff = np.nonzero(got[:n] != want[b][:n])[0]
+            if len(diff):
+                assert margins[b][diff[0]] < MARGIN_TOL, (b, int(diff[0]))
+            else:
+                assert len(got) == len(want[b])
+    # steps after sequence 1 ended carry a gather launch and fewer attention CTAs; the count of launches per step is
+    # the plain step's + 1 for those steps
+    per_step = (2 * cfg.n_layers + 4) if kind == "bf16" else None
+    if per_step:
+        assert st.steps * per_step < dec.fc_last_launch_count() <= st.steps * (per_step + 1)
+    cnt, _, _ = dec.fc_jacobi_step()
+    assert cnt.tolist() == [0] * B
+    assert dec.fc_debug_check_guards() == 0
