@@ -66,6 +66,11 @@ CASES = [
     (4, 4, 64, 16, [6000, 2047, 129], 4),             # forced: 4 splits, running softmax statistics over ~24 tiles each
     (8, 2, 128, 16, [2047, 1], 3),                    # forced odd cluster size with grouped queries (2 query tiles)
     (32, 32, 128, 16, [1000], 0),                     # the benchmark's attention shape: 32 heads, 4 splits of 4 tiles
+    # more (sequence, kv head, query tile) units than CTA slots: four query tiles per CTA, two CTAs per SM on a
+    # two-stage ring
+    (8, 8, 64, 64, [70, 1, 130, 257, 64] * 8, 0),
+    (8, 8, 128, 64, [70, 1, 130, 257, 64] * 8, 0),
+    (16, 8, 128, 32, [200, 5, 129] * 6, 0),           # grouped queries, four tiles per kv head, two per CTA
 ]
 
 
