@@ -313,9 +313,9 @@ def test_7b_prefill_stored_steps_and_256_token_stream():
     assert dec.fc_debug_check_guards() == 0
 
 
-# A gross-error guard, not the parity bar: the 13B shape's logit distance to the oracle sits AT the 3e-2 bar (per
-# sequence 0.018 .. 0.033 over the stored steps, and it moves by a few 1e-3 from run to run with the order of the fp32
-# reductions), so the bar itself is asserted by a test of its own that may fail (below), while this one must not.
+# A gross-error guard, not the parity bar: the 13B shape's logit distance to the oracle sits AT the 3e-2 bar (worst
+# sampled error over the stored steps 0.016 .. 0.025 for seven of the eight sequences, 0.030 .. 0.033 for sequence 3, and
+# it moves by a few 1e-3 from run to run with the order of the fp32 reductions), so the bar itself is asserted by a test of its own that may fail (below), while this one must not.
 GROSS_LOGIT_TOL = 0.1
 _WORST_13B = {}
 
@@ -345,9 +345,9 @@ def test_13b_batch8_prefill_stored_steps_and_streams():
     _run_13b_stored(check_streams=True)
 
 
-@pytest.mark.xfail(strict=False, reason="13B x 8 sits at the bar: worst sampled logit error per stored sequence 0.018 .. "
-                                        "0.033 over the first 8 iterations, varying by a few 1e-3 from run to run; the "
-                                        "bar stays 3e-2 and this test says whether this run met it")
+@pytest.mark.xfail(strict=False, reason="13B x 8 sits at the bar: worst sampled logit error over the first 8 iterations "
+                                        "0.016 .. 0.025 for seven sequences, 0.030 .. 0.033 for sequence 3, varying by a few "
+                                        "1e-3 from run to run; the bar stays 3e-2 and this test says whether this run met it")
 def test_13b_batch8_stored_logits_within_the_bar():
     if not _WORST_13B:
         _run_13b_stored(check_streams=False)
