@@ -356,10 +356,10 @@ def test_13b_batch8_stored_logits_within_the_bar():
 
 @pytest.mark.parametrize("hd,heads,kv_heads", [(64, 8, 8), (128, 4, 4), (64, 8, 2)])
 def test_long_ragged_caches_several_chunks_per_cta(hd, heads, kv_heads):
-    """Long caches in a batch: more 128-key chunks than the GPU holds CTAs, so one CTA walks over several
-    consecutive chunks with running softmax statistics (ragged lengths: CTAs with fewer live chunks, with
-    none, and with the window's own keys in their last chunk; with grouped queries there are two 16-row query
-    tiles per kv head, each with CTAs of its own)."""
+    """Long caches in a batch: every CTA of the attention kernel walks over a long run of 64-key tiles with running
+    softmax statistics, two CTAs per SM on a shallow ring (ragged lengths: CTAs with fewer tiles, with none, and with
+    the window's own keys after their last cached tile; with grouped queries there are two 16-row query tiles per kv
+    head)."""
     cfg = wl.small_config(vocab=500, n_layers=2, n_heads=heads, n_kv_heads=kv_heads, head_dim=hd, d_model=512,
                           d_ffn=512, c=8, prompt_len=64, gen_tokens=8)
     lens = [6000, 4100, 129, 5000, 1, 3333, 6000, 2047, 640, 5990]
