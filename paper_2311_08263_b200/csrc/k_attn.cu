@@ -361,6 +361,16 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   }
 
   __syncthreads();                                            // queries and window keys staged
+  // With one query tile per CTA the high parts of the query fragments stay in registers for the whole run of tiles
+  // (every warp multiplies the whole 16 x HD query tile by its 8 keys of every tile; re-reading it from shared memory
+  // for every tile is half of this kernel's shared-memory traffic); the low parts are still read per tile.
+  constexpr bool kQRegs = QT == 1;
+  uint32_t qh[kQRegs ? HD / 16 : 1][4];
+  if (kQRegs) {
+#pragma unroll
+    for (int ks = 0; ks < HD / 16; ++ks)
+      ldsm_x4(base + off_q + tile_off(lane & 15, ks * 2 + (lane >> 4), 2048u), qh[ks][0], qh[ks][1], qh[ks][2], qh[ks][3]);
+  }
   bool all_ok = true;
   const int n_tiles = n_cached + n_win;
   for (int ti = 0; ti < n_tiles; ++ti) {
@@ -406,11 +416,16 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
           const uint32_t qoff = tile_off(lane & 15, (ks2 * 2 + h2) * 2 + (lane >> 4), 2048u);
 #pragma unroll
           for (int qt = 0; qt < QT; ++qt) {
-            uint32_t ah[4], al[4];
+            uint32_t al[4];
             const uint32_t qb = base + off_q + (uint32_t)qt * C::kQTile + qoff;
-            ldsm_x4(qb, ah[0], ah[1], ah[2], ah[3]);
             ldsm_x4(qb + SUB * 2048u, al[0], al[1], al[2], al[3]);
-            mma_bf16(s[qt], ah, kf[h2 * 2], kf[h2 * 2 + 1]);
+            if (kQRegs) {
+              mma_bf16(s[qt], qh[ks2 * 2 + h2], kf[h2 * 2], kf[h2 * 2 + 1]);
+            } else {
+              uint32_t ah[4];
+              ldsm_x4(qb, ah[0], ah[1], ah[2], ah[3]);
+              mma_bf16(s[qt], ah, kf[h2 * 2], kf[h2 * 2 + 1]);
+            }
             mma_bf16(s[qt], al, kf[h2 * 2], kf[h2 * 2 + 1]);
           }
         }
