@@ -177,7 +177,7 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   const uint32_t off_p = off_q + QT * C::kQTile;
   const uint32_t off_wmax = off_p + QT * 4096u;
   const uint32_t off_ml = off_wmax + 8u * ROWS * 4u;
-  float *wmax = reinterpret_cast<float *>(gen + off_wmax);    // [8 warps][ROWS]
+  float *wmax = reinterpret_cast<float *>(gen + off_wmax);    // [ROWS][8 warps]
   float *ml = reinterpret_cast<float *>(gen + off_ml);        // [ROWS][2]
   float *obuf = reinterpret_cast<float *>(gen);               // [ROWS][HD], over ring stage 0 once the tiles are consumed
 
@@ -435,20 +435,30 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
 #pragma unroll
     for (int qt = 0; qt < QT; ++qt) {
       float mx[2] = {-INFINITY, -INFINITY};
+      if (!causal && nvalid == rows_t) {          // a full tile of cached keys: every key is visible to every query row
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int hh = i >> 1;
-        const int kl = warp * 8 + t4 * 2 + (i & 1);
-        const bool vis = my_keys && jrow[qt][hh] >= 0 && kl < nvalid && (!causal || koff + kl <= jrow[qt][hh]);
-        const float v = vis ? s[qt][i] * scale : -INFINITY;
-        s[qt][i] = v;
-        mx[hh] = fmaxf(mx[hh], v);
+        for (int i = 0; i < 4; ++i) {
+          const int hh = i >> 1;
+          const float v = (my_keys && jrow[qt][hh] >= 0) ? s[qt][i] * scale : -INFINITY;
+          s[qt][i] = v;
+          mx[hh] = fmaxf(mx[hh], v);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int hh = i >> 1;
+          const int kl = warp * 8 + t4 * 2 + (i & 1);
+          const bool vis = my_keys && jrow[qt][hh] >= 0 && kl < nvalid && (!causal || koff + kl <= jrow[qt][hh]);
+          const float v = vis ? s[qt][i] * scale : -INFINITY;
+          s[qt][i] = v;
+          mx[hh] = fmaxf(mx[hh], v);
+        }
       }
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
         mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 1));
         mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 2));
-        if (t4 == 0) wmax[warp * ROWS + qt * 16 + g4 + hh * 8] = mx[hh];
+        if (t4 == 0) wmax[(qt * 16 + g4 + hh * 8) * 8 + warp] = mx[hh];      // [row][warp]: a row's eight values in 32 bytes
       }
     }
     all_ok = __syncthreads_and(ok ? 1 : 0) != 0;              // maxima published; every warp is past the previous tile
@@ -464,8 +474,10 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
       for (int hh = 0; hh < 2; ++hh) {
         const int row = qt * 16 + g4 + hh * 8;
         float mx = m_run[qt][hh];
-#pragma unroll
-        for (int w = 0; w < 8; ++w) mx = fmaxf(mx, wmax[w * ROWS + row]);
+        {
+          const float4 w0 = *reinterpret_cast<const float4 *>(wmax + row * 8), w1 = *reinterpret_cast<const float4 *>(wmax + row * 8 + 4);
+          mx = fmaxf(mx, fmaxf(fmaxf(fmaxf(w0.x, w0.y), fmaxf(w0.z, w0.w)), fmaxf(fmaxf(w1.x, w1.y), fmaxf(w1.z, w1.w))));
+        }
         mnew[hh] = mx;
         corr[hh] = (m_run[qt][hh] == -INFINITY) ? 0.f : __expf(m_run[qt][hh] - mx);
         m_run[qt][hh] = mx;
@@ -531,7 +543,7 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   for (int qt = 0; qt < QT; ++qt)
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh)
-      if (t4 == 0) wmax[warp * ROWS + qt * 16 + g4 + hh * 8] = l_run[qt][hh];
+      if (t4 == 0) wmax[(qt * 16 + g4 + hh * 8) * 8 + warp] = l_run[qt][hh];
 #pragma unroll
   for (int qt = 0; qt < QT; ++qt)
 #pragma unroll
@@ -544,7 +556,7 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
   if (tid < ROWS) {
     float lt = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) lt += wmax[w * ROWS + tid];
+    for (int w = 0; w < 8; ++w) lt += wmax[tid * 8 + w];
     // every warp holds the same running maximum; take it from the lane that owns this row in warp tid / 32's layout
     ml[tid * 2 + 1] = lt;
   }
