@@ -55,7 +55,8 @@ enum {                        /* fc_model_shape.flags */
   FC_FLAG_SIMT_GEMM = 1,      /* run projections on the plain FMA kernels even for bf16 (debug aid) */
   FC_FLAG_NO_PDL = 4,         /* launch every kernel fully serialised (no programmatic dependent launch) */
   FC_FLAG_NO_CHAIN = 8,       /* one launch per projection instead of one chained launch per layer */
-  FC_FLAG_NO_FFN_SPLIT = 16   /* chained launch: gate/up and down as one phase each instead of two halves of d_ffn */
+  FC_FLAG_NO_FFN_SPLIT = 16,  /* chained launch: gate/up and down as one phase each instead of two halves of d_ffn */
+  FC_FLAG_NO_CTA_PAIRS = 32   /* more than 64 rows: one CTA per weight tile instead of a pair of CTAs per 256-row tile */
 };
 
 typedef struct {

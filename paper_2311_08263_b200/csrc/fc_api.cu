@@ -144,6 +144,7 @@ struct fc_ctx {
   cudaStream_t st;
   bool use_umma;
   bool pdl;          // chain the tensor-core kernels by programmatic dependent launch
+  bool cta_pairs;    // more than 64 rows: projections as clusters of two CTAs per 256-row weight tile
   bool chain;        // run O -> gate/up -> down -> next layer's QKV as one launch with grid barriers
   bool fused_attn;   // bf16 with head_dim 64/128: rotary embedding and K/V write happen inside the attention kernel
   KvTensorMap kv_map; // TMA view of the whole K/V slab: (head_dim, max_seq, layers * 2 * max_batch * kv heads)
@@ -335,6 +336,7 @@ extern "C" int fc_init(fc_ctx **out, const fc_model_shape *shape, const fc_weigh
   ctx->st = (cudaStream_t)cuda_stream;
   ctx->use_umma = shape->dtype == FC_BF16 && !(shape->flags & FC_FLAG_SIMT_GEMM);
   ctx->pdl = !(shape->flags & FC_FLAG_NO_PDL);
+  ctx->cta_pairs = !(shape->flags & FC_FLAG_NO_CTA_PAIRS);
   ctx->chain = ctx->use_umma && !(shape->flags & FC_FLAG_NO_CHAIN);
   ctx->fused_attn = shape->dtype == FC_BF16 && (shape->head_dim == 64 || shape->head_dim == 128) &&
                     !(shape->flags & FC_FLAG_SIMT_GEMM);
@@ -432,7 +434,7 @@ static cudaError_t run_gemm(fc_ctx *ctx, const UmmaPlan *plan, GemmArgs a, int R
   ProfScope ps(ctx, cls);
   a.R = R;
   ++ctx->launches;
-  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + (kSyncPanel - kSyncClaim), zero, ctx->pdl && !ctx->prof, ctx->st);   // panel-ready word
+  if (ctx->use_umma) return launch_gemm_umma(plan, a, claim, claim + (kSyncPanel - kSyncClaim), zero, ctx->pdl && !ctx->prof, ctx->st, ctx->cta_pairs);   // panel-ready word
   return launch_gemm_simt(a, ctx->s.dtype, pro, epi, ctx->st);
 }
 
@@ -535,7 +537,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ProfScope ps(ctx, FC_CLS_CHAIN);
       unsigned int *grp = ctx->b.chain_bar + (size_t)l * d.sync_words;
       FC_CK(launch_gemm_chain(plans, ga, n, grp, grp + kSyncClaim, grp + kSyncPanel, R <= 16 ? sy : nullptr, grp + kSyncTd,
-                              (s.d_model + 127) / 128, zero, ctx->pdl && !ctx->prof, ctx->st));
+                              (s.d_model + 127) / 128, zero, ctx->pdl && !ctx->prof, ctx->st, ctx->cta_pairs));
     } else {
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_o[l] : nullptr, args_o(ctx, l), R, PRO_NONE, EPI_ATOMIC_ADD, FC_CLS_OPROJ, claim_word(ctx, l, GEMM_O), zero));
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_gu[l] : nullptr, args_gu(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_GATEUP, claim_word(ctx, l, GEMM_GU)));

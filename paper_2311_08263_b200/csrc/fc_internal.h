@@ -180,8 +180,10 @@ void umma_plan_destroy(UmmaPlan *p);
 // claim: one zeroed word per projection of the launch (the work-claim counters).
 // zero (optional): buffers the launch clears at its start, once the previous kernel is complete; only for buffers that
 // nothing reads before a later kernel or a phase behind a grid barrier of this launch accumulates into them.
+// cta_pairs: with 128-row blocks in panel mode and weight matrices of whole 256-row tiles, run as clusters of two
+// CTAs that share a tile (tcgen05 cta_group::2).
 cudaError_t launch_gemm_umma(const UmmaPlan *p, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b,
-                             const ZeroList *zero, int pdl, cudaStream_t st);
+                             const ZeroList *zero, int pdl, cudaStream_t st, int cta_pairs = 0);
 // Up to four projections in one launch, each consuming the previous one's reduced output; bar: n-1 zeroed words.
 // bar_b: n zeroed words (panel-ready barriers), needed when the rows exceed 16 and the plans have panels.
 // sync (optional, used up to 16 rows): how each projection is tied to the others, instead of a grid barrier
@@ -196,6 +198,6 @@ struct ChainSync { int wait_bar, sig_bar, td_prod, td_cons, epi_bar; };
 constexpr int kChainMax = 6;     // projections in one chained launch
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
                               unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,
-                              int td_stride, const ZeroList *zero, int pdl, cudaStream_t st);
+                              int td_stride, const ZeroList *zero, int pdl, cudaStream_t st, int cta_pairs = 0);
 
 }  // namespace fc

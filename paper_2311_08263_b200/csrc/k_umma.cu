@@ -40,7 +40,8 @@ constexpr int kMaxPhases = kChainMax;   // projections chained in one launch (O 
 struct PhaseDesc {
   GemmArgs g;
   int pro;                        // ProOp applied while the activations are staged
-  int n_tiles, nkb;               // 128-row tiles over all matrices; 64-wide k blocks
+  int n_tiles, nkb;               // weight tiles over all matrices; 64-wide k blocks
+  int tile_rows;                  // weight rows per tile: 128, or 256 when a pair of CTAs shares a tile (each CTA 128 of them)
   int tiles_m[kMaxMats];
   int tx_bytes[kMaxMats];         // bytes one TMA box of matrix m delivers
   int chunk_kb, cpt, nrb, n_chunks;   // work is claimed in chunks of chunk_kb k-blocks of one tile for one block of rows:
@@ -135,6 +136,53 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+// ---- CTA pairs (cta_group::2): a cluster of two CTAs multiplies one 256-row weight tile; each CTA stages its 128
+// weight rows and its half of the activation operand, the leader (cluster rank 0) issues the MMAs for both, and the
+// accumulator rows of a CTA's 128 weight rows land in that CTA's tensor memory.
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrival on a barrier of any CTA of the cluster (address from map_to_cta)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on a barrier of the pair's leader
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc) : "memory");
+}
+// completion of the pair's MMAs so far, signalled on the barrier at this offset in both CTAs
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -176,8 +224,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
   return d;
 }
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = bn.
-__host__ __device__ constexpr uint32_t make_idesc(int bn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+__host__ __device__ constexpr uint32_t make_idesc(int bn, int m = kTileM) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ unsigned int ordered_key_u(float v) {
@@ -263,8 +311,8 @@ __device__ __forceinline__ void tile_info(const PhaseDesc &d, int tile, int &m, 
   m = 0;
   int lt = tile;
   while (m + 1 < d.g.n_mats && lt >= d.tiles_m[m]) { lt -= d.tiles_m[m]; ++m; }
-  row0 = lt * kTileM;
-  rows_valid = min(kTileM, d.g.n_rows[m] - row0);
+  row0 = lt * d.tile_rows;
+  rows_valid = min(d.tile_rows, d.g.n_rows[m] - row0);
   ycol0 = d.g.y_off[m] + row0;
 }
 
@@ -301,19 +349,24 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 // Widths up to 32 rows run two CTAs per SM (the grid barrier needs the whole grid resident).
 // PANEL: the activations come from a bf16 hi/lo panel in global memory, converted once per projection by all
 // CTAs together and streamed by TMA, instead of being converted by every CTA for every weight tile.
-template <int EPI, int BN, bool PANEL>
+// PAIR: launched as clusters of two CTAs that share 256-row weight tiles (panel mode, 128-row blocks): per k-block each
+// CTA stages 16 KB of weights and ONE of the two activation tiles (the leader the high one, its peer the low one)
+// for 2 x 128 x 256 x 64 products - half of the shared-memory traffic per product of the single-CTA form.  Chunks are
+// dealt statically (pair i takes chunks i, i + pairs, ...), so both CTAs of a pair walk the same list without talking.
+template <int EPI, int BN, bool PANEL, bool PAIR = false>
 __global__ void __launch_bounds__(kThreads, (BN <= 32 ? 2 : 1))
 gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ UmmaParams p) {
+  static_assert(!PAIR || (PANEL && BN == 128 && EPI == EPI_ATOMIC_ADD), "CTA pairs: panel mode, 128-row blocks, reductions");
   constexpr int kXParts = x_parts(BN);
   constexpr int kXBytes = BN * 128;                 // one staged activation tile (bf16, 64 k)
-  constexpr int kStageBytes = kWBytes + kXParts * kXBytes;
+  constexpr int kStageBytes = kWBytes + (PAIR ? 1 : kXParts) * kXBytes;
   // The high and the low activation tiles lie back to back in a stage, which is exactly a K-major tile of 2 * BN
   // rows: one MMA of N = 2 * BN multiplies both (columns 0..BN-1 of the accumulator take the high part's products,
   // BN..2BN-1 the low part's; the epilogue adds them).  The issuing thread is the kernel's critical path at small
   // N - an MMA costs it a fixed ~200 cycles whatever its width - so half as many instructions matter.
   constexpr int kAccCols = kXParts * BN;                        // TMEM columns of one accumulator
   constexpr uint32_t kCols = (uint32_t)(2 * kAccCols);          // two accumulators: 64 .. 512, a power of two
-  constexpr uint32_t kIdesc = make_idesc(kAccCols);
+  constexpr uint32_t kIdesc = PAIR ? make_idesc(kAccCols, 2 * kTileM) : make_idesc(kAccCols);
 
   extern __shared__ unsigned char smem_dyn[];
   __shared__ __align__(8) unsigned long long full_w[8], full_x[8], empty_b[8], accum_full[2], tmem_empty[2], ss_ready[2], drain_bar, go_bar[kMaxPhases], seg_full[kSegQ], seg_empty[kSegQ];
@@ -327,20 +380,26 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = p.stages;
   volatile int *abort_flag = &abort_s;
+  const uint32_t rank = PAIR ? cluster_rank() : 0u;          // 0: the pair's leader
 
   if (threadIdx.x == 0) {
     abort_s = 0;
     for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&full_w[i]), 1); mbar_init(smem_u32(&full_x[i]), 1); mbar_init(smem_u32(&empty_b[i]), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
+    // an accumulator is free again once the epilogue warps of the CTA (of both CTAs of a pair) have read it
+    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&accum_full[i]), 1); mbar_init(smem_u32(&tmem_empty[i]), PAIR ? 8 : 4); mbar_init(smem_u32(&ss_ready[i]), 4); }
     mbar_init(smem_u32(&drain_bar), 1);
     for (int i = 0; i < kMaxPhases; ++i) { mbar_init(smem_u32(&go_bar[i]), 1); bar_cnt_s[i] = 0u; bar_cnt_b[i] = 0u; }
     // a queue slot is read by the MMA thread, four staging warps and four epilogue warps
     for (int i = 0; i < kSegQ; ++i) { mbar_init(smem_u32(&seg_full[i]), 1); mbar_init(smem_u32(&seg_empty[i]), 9); }
     fence_barrier_init();
   }
-  if (warp == 1) tmem_alloc(smem_u32(&tmem_base_s), kCols);
+  if (warp == 1) {
+    if constexpr (PAIR) tmem_alloc_pair(smem_u32(&tmem_base_s), kCols);
+    else tmem_alloc(smem_u32(&tmem_base_s), kCols);
+  }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();      // the peer's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
   // Let the next kernel of the stream start its own set-up and weight prefetch as soon as every CTA of
@@ -373,6 +432,104 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
     return 1;
   };
 
+  // Panel mode, step 1 of a phase: all CTAs together convert pro(x) into the bf16 panel [high | low] once.  The four
+  // staging and the four epilogue warps of every CTA take part (wslot 0..7; the epilogue warps have nothing else to
+  // do between two phases); a warp takes 32 consecutive (row, 8-wide chunk) units at a time, four such groups per
+  // pass so that the loads overlap.  The warp's arrival on the panel-ready barrier follows.
+  constexpr int kConvWarps = 8;
+  auto convert_share = [&](const PhaseDesc &P, int pi, int wslot) {
+    const GemmArgs &g = P.g;
+    const int pro = P.pro;
+    {
+      const int kc8 = g.K >> 3;
+      const int units = g.R * kc8;                       // the host keeps R * K / 8 below 2^31
+      const int n_groups = (units + 31) >> 5;
+      const int warps_total = (int)gridDim.x * kConvWarps;
+      __nv_bfloat16 *pan_hi = (__nv_bfloat16 *)g.pan;
+      __nv_bfloat16 *pan_lo = pan_hi + (long long)g.pan_rows * g.K;
+      const bool want_ss = pro == PRO_GAIN && g.ss_out != nullptr;
+      for (int g0 = (int)blockIdx.x * kConvWarps + wslot; g0 < n_groups; g0 += 4 * warps_total) {
+        float4 xa[4], xb[4], ua[4], ubv[4];
+        float ssr[4];
+        uint4 gq[4];
+        int un[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          un[j] = g0 + j * warps_total < n_groups ? ((g0 + j * warps_total) << 5) + lane : units;
+          xa[j] = xb[j] = ua[j] = ubv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          ssr[j] = 0.f; gq[j] = make_uint4(0, 0, 0, 0);
+          if (un[j] < units) {
+            const int r = un[j] / kc8, k = (un[j] - r * kc8) << 3;
+            const float *px = g.x + (long long)r * g.ldx + k;
+            xa[j] = __ldcg(reinterpret_cast<const float4 *>(px));
+            xb[j] = __ldcg(reinterpret_cast<const float4 *>(px + 4));
+            if (pro == PRO_GAIN) gq[j] = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
+            if (pro == PRO_SILU_MUL) {
+              const float *pu = g.x2 + (long long)r * g.ldx + k;
+              ua[j] = __ldcg(reinterpret_cast<const float4 *>(pu));
+              ubv[j] = __ldcg(reinterpret_cast<const float4 *>(pu + 4));
+              ssr[j] = __ldcg(g.ss_in + r);
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const bool live = un[j] < units;
+          const int r = live ? un[j] / kc8 : -1;
+          float v[8] = {xa[j].x, xa[j].y, xa[j].z, xa[j].w, xb[j].x, xb[j].y, xb[j].z, xb[j].w};
+          float sq = 0.f;
+          if (pro == PRO_GAIN) {
+            const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq[j]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 gf = __bfloat1622float2(gp[i]);
+              sq = fmaf(v[2 * i], v[2 * i], sq); sq = fmaf(v[2 * i + 1], v[2 * i + 1], sq);
+              v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
+            }
+          } else if (pro == PRO_SILU_MUL) {
+            const float sr = rsqrtf(ssr[j] / (float)g.dn + g.eps);
+            const float uu[8] = {ua[j].x, ua[j].y, ua[j].z, ua[j].w, ubv[j].x, ubv[j].y, ubv[j].z, ubv[j].w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float gt = sr * v[i];
+              v[i] = __fdividef(gt, 1.0f + __expf(-gt)) * (sr * uu[i]);
+            }
+          }
+          if (want_ss) {
+            // lanes of a group usually share the row: one reduction per group, else one per lane
+            const int r0 = __shfl_sync(0xffffffffu, r, 0);
+            if (__all_sync(0xffffffffu, r == r0)) {
+              const float t = warp_sum_f(sq);
+              if (lane == 0 && r0 >= 0) atomicAdd(&g.ss_out[r0], t);
+            } else if (live) {
+              atomicAdd(&g.ss_out[r], sq);
+            }
+          }
+          if (live) {
+            const int k = (un[j] - r * kc8) << 3;
+            uint4 pk;
+            __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
+            pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+            pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+            *reinterpret_cast<uint4 *>(pan_hi + (long long)r * g.K + k) = pk;
+            const float2 h0 = __bfloat1622float2(b0), h1 = __bfloat1622float2(b1);
+            const float2 h2 = __bfloat1622float2(b2), h3 = __bfloat1622float2(b3);
+            b0 = __floats2bfloat162_rn(v[0] - h0.x, v[1] - h0.y); b1 = __floats2bfloat162_rn(v[2] - h1.x, v[3] - h1.y);
+            b2 = __floats2bfloat162_rn(v[4] - h2.x, v[5] - h2.y); b3 = __floats2bfloat162_rn(v[6] - h3.x, v[7] - h3.y);
+            pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
+            pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
+            *reinterpret_cast<uint4 *>(pan_lo + (long long)r * g.K + k) = pk;
+          }
+        }
+      }
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");      // generic-proxy stores before the TMA reads that follow the barrier
+    __threadfence();
+    __syncwarp();
+    if (lane == 0 && atomicAdd(&bar_cnt_b[pi], 1u) == (unsigned int)(kConvWarps - 1)) { __threadfence(); atomicAdd(p.bar_b + pi, 1u); }
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     // Weights depend on nothing that runs on the device, so the producer never waits for a grid barrier
@@ -384,10 +541,14 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       bool ok = true;
       for (int pi = 0; pi < p.n_phases && ok; ++pi) {
         const PhaseDesc &P = p.ph[pi];
+        int dealt = 0;
+        (void)dealt;
         for (;;) {
           const int slot = sq & (kSegQ - 1);
           if (!mbar_wait(smem_u32(&seg_empty[slot]), ((uint32_t)(sq / kSegQ) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-          const unsigned int id = atomicAdd(p.claim + pi, 1u);
+          unsigned int id;
+          if constexpr (PAIR) { id = (blockIdx.x >> 1) + (unsigned int)dealt * (gridDim.x >> 1); ++dealt; }
+          else id = atomicAdd(p.claim + pi, 1u);
           if (id >= (unsigned int)P.n_chunks) {                 // nothing left in this phase
             seg_q[slot] = make_int4(-1, 0, 0, 0);
             mbar_arrive(smem_u32(&seg_full[slot]));
@@ -406,13 +567,25 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           for (int kb = s.kb0; kb < s.kb1; ++kb, ++it) {
             if (!mbar_wait(smem_u32(&empty_b[stage]), ph ^ 1u, abort_flag)) { ok = false; break; }
             const uint32_t bar = smem_u32(&full_w[stage]);
-            mbar_expect_tx(bar, (uint32_t)P.tx_bytes[m]);
-            tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
+            if constexpr (PAIR) {
+              // the leader's barrier counts both CTAs' 16 KB; the peer's copy may land before the leader has announced
+              // it (the byte count of a phase may run negative for a while)
+              if (rank == 0) mbar_expect_tx(bar, 2u * (uint32_t)kWBytes);
+              tma_load_2d_pair(smem_base + stage * kStageBytes, mp, kb * kTileK, row0 + (int)rank * kTileM, map_to_cta(bar, 0));
+            } else {
+              mbar_expect_tx(bar, (uint32_t)P.tx_bytes[m]);
+              tma_load_2d(smem_base + stage * kStageBytes, mp, kb * kTileK, row0, bar);
+            }
             issued = it + 1;
             if (++stage == S) { stage = 0; ph ^= 1u; }
           }
           if (!ok) break;
         }
+      }
+      if constexpr (PAIR) {
+        // the leader's MMA completions arrive on this CTA's ring barriers too: all of them have landed before it leaves
+        for (int i = (it > S ? it - S : 0); i < it && ok; ++i)
+          ok = mbar_wait(smem_u32(&empty_b[i % S]), (uint32_t)(i / S) & 1u, abort_flag);
       }
     }
   } else if (warp == 1) {
@@ -431,6 +604,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           while (ok) {
             const int got = take_lane(sq, s, rb);
             if (got <= 0) { ok = got == 0; break; }
+            if (PAIR && rank != 0) { ++seg; continue; }       // the leader issues for the pair
             const int acc = seg & 1;
             if (!mbar_wait(smem_u32(&tmem_empty[acc]), (((uint32_t)seg >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -442,15 +616,27 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
               const uint32_t a_base = smem_base + stage * kStageBytes;
               const uint64_t a_desc = smem_desc_sw128(a_base), b_desc = smem_desc_sw128(a_base + kWBytes);
 #pragma unroll
-              for (int kk = 0; kk < kTileK / 16; ++kk)      // 32 bytes along k: the start-address field counts 16-byte units
-                umma_bf16(d_tmem, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), kIdesc, (kb > s.kb0 || kk > 0) ? 1u : 0u);
-              umma_commit(smem_u32(&empty_b[stage]));
+              for (int kk = 0; kk < kTileK / 16; ++kk) {    // 32 bytes along k: the start-address field counts 16-byte units
+                if constexpr (PAIR) umma_bf16_pair(d_tmem, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), kIdesc, (kb > s.kb0 || kk > 0) ? 1u : 0u);
+                else umma_bf16(d_tmem, a_desc + (uint64_t)(kk * 2), b_desc + (uint64_t)(kk * 2), kIdesc, (kb > s.kb0 || kk > 0) ? 1u : 0u);
+              }
+              if constexpr (PAIR) umma_commit_pair(smem_u32(&empty_b[stage]));
+              else umma_commit(smem_u32(&empty_b[stage]));
               if (++stage == S) { stage = 0; ph ^= 1u; }
             }
-            if (ok) umma_commit(smem_u32(&accum_full[acc]));
+            if (ok) {
+              if constexpr (PAIR) umma_commit_pair(smem_u32(&accum_full[acc]));
+              else umma_commit(smem_u32(&accum_full[acc]));
+            }
             ++seg;
           }
         }
+      }
+      if constexpr (PAIR) {
+        // the peer's epilogue warps arrive on this CTA's accumulator barriers: wait for the last two rounds
+        if (rank == 0)
+          for (int sg = (seg > 2 ? seg - 2 : 0); sg < seg && ok; ++sg)
+            ok = mbar_wait(smem_u32(&tmem_empty[sg & 1]), ((uint32_t)sg >> 1) & 1u, abort_flag);
       }
     }
   } else if (warp < 6) {
@@ -481,97 +667,9 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         if (!ok) break;
       }
       if constexpr (PANEL) {
-        // ---- (1) all CTAs together convert pro(x) into the bf16 panel [high | low] once; a warp takes 32
-        // consecutive (row, 8-wide chunk) units at a time, four such groups per pass so that the loads overlap
-        {
-          const int kc8 = g.K >> 3;
-          const int units = g.R * kc8;                       // the host keeps R * K / 8 below 2^31
-          const int n_groups = (units + 31) >> 5;
-          const int warps_total = (int)gridDim.x * 4;
-          __nv_bfloat16 *pan_hi = (__nv_bfloat16 *)g.pan;
-          __nv_bfloat16 *pan_lo = pan_hi + (long long)g.pan_rows * g.K;
-          const bool want_ss = pro == PRO_GAIN && g.ss_out != nullptr;
-          for (int g0 = (int)blockIdx.x * 4 + sw; g0 < n_groups; g0 += 4 * warps_total) {
-            float4 xa[4], xb[4], ua[4], ubv[4];
-            float ssr[4];
-            uint4 gq[4];
-            int un[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              un[j] = g0 + j * warps_total < n_groups ? ((g0 + j * warps_total) << 5) + lane : units;
-              xa[j] = xb[j] = ua[j] = ubv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-              ssr[j] = 0.f; gq[j] = make_uint4(0, 0, 0, 0);
-              if (un[j] < units) {
-                const int r = un[j] / kc8, k = (un[j] - r * kc8) << 3;
-                const float *px = g.x + (long long)r * g.ldx + k;
-                xa[j] = __ldcg(reinterpret_cast<const float4 *>(px));
-                xb[j] = __ldcg(reinterpret_cast<const float4 *>(px + 4));
-                if (pro == PRO_GAIN) gq[j] = *reinterpret_cast<const uint4 *>((const __nv_bfloat16 *)g.gain + k);
-                if (pro == PRO_SILU_MUL) {
-                  const float *pu = g.x2 + (long long)r * g.ldx + k;
-                  ua[j] = __ldcg(reinterpret_cast<const float4 *>(pu));
-                  ubv[j] = __ldcg(reinterpret_cast<const float4 *>(pu + 4));
-                  ssr[j] = __ldcg(g.ss_in + r);
-                }
-              }
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const bool live = un[j] < units;
-              const int r = live ? un[j] / kc8 : -1;
-              float v[8] = {xa[j].x, xa[j].y, xa[j].z, xa[j].w, xb[j].x, xb[j].y, xb[j].z, xb[j].w};
-              float sq = 0.f;
-              if (pro == PRO_GAIN) {
-                const __nv_bfloat162 *gp = reinterpret_cast<const __nv_bfloat162 *>(&gq[j]);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float2 gf = __bfloat1622float2(gp[i]);
-                  sq = fmaf(v[2 * i], v[2 * i], sq); sq = fmaf(v[2 * i + 1], v[2 * i + 1], sq);
-                  v[2 * i] *= gf.x; v[2 * i + 1] *= gf.y;
-                }
-              } else if (pro == PRO_SILU_MUL) {
-                const float sr = rsqrtf(ssr[j] / (float)g.dn + g.eps);
-                const float uu[8] = {ua[j].x, ua[j].y, ua[j].z, ua[j].w, ubv[j].x, ubv[j].y, ubv[j].z, ubv[j].w};
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                  const float gt = sr * v[i];
-                  v[i] = __fdividef(gt, 1.0f + __expf(-gt)) * (sr * uu[i]);
-                }
-              }
-              if (want_ss) {
-                // lanes of a group usually share the row: one reduction per group, else one per lane
-                const int r0 = __shfl_sync(0xffffffffu, r, 0);
-                if (__all_sync(0xffffffffu, r == r0)) {
-                  const float t = warp_sum_f(sq);
-                  if (lane == 0 && r0 >= 0) atomicAdd(&g.ss_out[r0], t);
-                } else if (live) {
-                  atomicAdd(&g.ss_out[r], sq);
-                }
-              }
-              if (live) {
-                const int k = (un[j] - r * kc8) << 3;
-                uint4 pk;
-                __nv_bfloat162 b0 = __floats2bfloat162_rn(v[0], v[1]), b1 = __floats2bfloat162_rn(v[2], v[3]);
-                __nv_bfloat162 b2 = __floats2bfloat162_rn(v[4], v[5]), b3 = __floats2bfloat162_rn(v[6], v[7]);
-                pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
-                pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
-                *reinterpret_cast<uint4 *>(pan_hi + (long long)r * g.K + k) = pk;
-                const float2 h0 = __bfloat1622float2(b0), h1 = __bfloat1622float2(b1);
-                const float2 h2 = __bfloat1622float2(b2), h3 = __bfloat1622float2(b3);
-                b0 = __floats2bfloat162_rn(v[0] - h0.x, v[1] - h0.y); b1 = __floats2bfloat162_rn(v[2] - h1.x, v[3] - h1.y);
-                b2 = __floats2bfloat162_rn(v[4] - h2.x, v[5] - h2.y); b3 = __floats2bfloat162_rn(v[6] - h3.x, v[7] - h3.y);
-                pk.x = *reinterpret_cast<uint32_t *>(&b0); pk.y = *reinterpret_cast<uint32_t *>(&b1);
-                pk.z = *reinterpret_cast<uint32_t *>(&b2); pk.w = *reinterpret_cast<uint32_t *>(&b3);
-                *reinterpret_cast<uint4 *>(pan_lo + (long long)r * g.K + k) = pk;
-              }
-            }
-          }
-        }
-        // ---- (2) panel-ready barrier: the four staging warps of every CTA have stored their share
-        asm volatile("fence.proxy.async;" ::: "memory");      // generic-proxy stores before the TMA reads that follow the barrier
-        __threadfence();
-        __syncwarp();
-        if (lane == 0 && atomicAdd(&bar_cnt_b[pi], 1u) == 3u) { __threadfence(); atomicAdd(p.bar_b + pi, 1u); }
+        // ---- (1) this warp's share of the panel conversion
+        convert_share(P, pi, sw);
+        // ---- (2) panel-ready barrier: the eight converting warps of every CTA have stored their share
         if (sw == 0) {
           ok = grid_bar_wait(p.bar_b + pi, gridDim.x, lane, abort_flag);
           asm volatile("fence.proxy.async;" ::: "memory");
@@ -592,10 +690,16 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
               if (lane == 0) {
                 const uint32_t bar = smem_u32(&full_x[stage]);
                 const uint32_t xs = smem_base + stage * kStageBytes + kWBytes;
-                mbar_expect_tx(bar, (uint32_t)(kXParts * kXBytes));
+                if constexpr (PAIR) {
+                  // the leader stages the high tile, its peer the low one: the two halves of the N = 256 operand
+                  if (rank == 0) mbar_expect_tx(bar, (uint32_t)(kXParts * kXBytes));
+                  tma_load_2d_pair(xs, &maps.x[pi], kb * kTileK, (int)rank * g.pan_rows + rb * BN, map_to_cta(bar, 0));
+                } else {
+                  mbar_expect_tx(bar, (uint32_t)(kXParts * kXBytes));
 #pragma unroll
-                for (int part = 0; part < kXParts; ++part)
-                  tma_load_2d(xs + part * kXBytes, &maps.x[pi], kb * kTileK, part * g.pan_rows + rb * BN, bar);
+                  for (int part = 0; part < kXParts; ++part)
+                    tma_load_2d(xs + part * kXBytes, &maps.x[pi], kb * kTileK, part * g.pan_rows + rb * BN, bar);
+                }
               }
             }
             ++seg;
@@ -748,6 +852,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       const PhaseDesc &P = p.ph[pi];
       const GemmArgs &g = P.g;
       bool epi_bar_passed = P.epi_bar < 0;
+      if constexpr (PANEL) {
+        // the previous phase's sums are complete (a staging warp polls the grid barrier and opens go_bar): this warp's
+        // share of the panel conversion
+        if (P.wait_bar >= 0 && !mbar_wait_warp(smem_u32(&go_bar[pi]), 0u, abort_flag)) { ok = false; break; }
+        convert_share(P, pi, 4 + q);
+      }
       {
         Segment s;
         int rb = 0;
@@ -762,6 +872,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           }
           int m, row0, rows_valid, ycol0;
           tile_info(P, s.tile, m, row0, rows_valid, ycol0);
+          if constexpr (PAIR) { ycol0 += (int)rank * kTileM; rows_valid = kTileM; }     // this CTA's 128 weight rows of the pair's 256
           const int acc = seg & 1;
           const uint32_t ph = ((uint32_t)seg >> 1) & 1u;
           if (!mbar_wait_warp(smem_u32(&accum_full[acc]), ph, abort_flag)) { ok = false; break; }
@@ -822,7 +933,10 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&tmem_empty[acc]));
+          if (lane == 0) {
+            if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&tmem_empty[acc]), 0));
+            else mbar_arrive(smem_u32(&tmem_empty[acc]));
+          }
           if (EPI == EPI_ATOMIC_ADD && P.tile_done) {       // this warp's share of the chunk is reduced into the tile
             __syncwarp();
             if (lane == 0) red_release_gpu(P.tile_done + s.tile, 1u);
@@ -840,9 +954,10 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   if (abort_s) {
     if (threadIdx.x == 0) {
       atomicExch(p.err, 1u);
-      // wait (bounded) for this CTA's own TMA copies still in flight
+      // wait (bounded) for this CTA's own TMA copies still in flight (a pair's copies are counted by its leader, and
+      // the peer stays until the leader has passed the cluster barrier below)
       const unsigned long long t0 = clock64();
-      for (int i = (issued > S ? issued - S : 0); i < issued; ++i) {
+      for (int i = (issued > S ? issued - S : 0); i < issued && rank == 0; ++i) {
         const uint32_t bar = smem_u32(&full_w[i % S]);
         while (!mbar_try(bar, (uint32_t)(i / S) & 1u))
           if ((unsigned long long)(clock64() - t0) > kSpinBudget / 4) break;
@@ -859,7 +974,12 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, kCols); }
+  if constexpr (PAIR) cluster_sync_all();      // neither CTA leaves, or frees tensor memory, while its peer still works
+  if (warp == 1) {
+    tc_fence_after();
+    if constexpr (PAIR) tmem_dealloc_pair(tmem_base, kCols);
+    else tmem_dealloc(tmem_base, kCols);
+  }
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -900,6 +1020,7 @@ UmmaPlan *umma_plan_create(const GemmArgs &a, int pro, int epi, int n_sms, unsig
   pl->d.pro = pro;
   pl->epi = epi; pl->n_sms = n_sms; pl->err = err_word;
   pl->d.nkb = (a.K + kTileK - 1) / kTileK;
+  pl->d.tile_rows = kTileM;
   pl->d.n_tiles = 0;
   for (int m = 0; m < a.n_mats; ++m) {
     if (a.n_rows[m] < 1) { delete pl; return fail("empty weight matrix"); }
@@ -958,6 +1079,47 @@ static cudaError_t launch_one(const MapPack &maps, const UmmaParams &p, int grid
   return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<EPI, BN, PANEL>, maps, p);
 }
 
+// CTA pairs: clusters of two, one CTA per SM, six stages of 16 KB weights + 16 KB activations.
+constexpr int kPairStages = 6;
+static size_t pair_smem_bytes() { return (size_t)kPairStages * (kWBytes + 128 * 128) + 1024; }
+static void pair_launch_config(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int grid, int pdl, cudaStream_t st) {
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = pair_smem_bytes(); cfg.stream = st;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl ? 2 : 1;
+}
+// Number of CTAs (an even number) that are certainly resident together as pairs; 0 if pairs cannot be launched.
+static int pair_grid(int n_sms) {
+  static int cached[kMaxDevices] = {0};
+  const int dev = current_device_slot();
+  if (cached[dev] == 0) {
+    auto kern = gemm_umma_kernel<EPI_ATOMIC_ADD, 128, true, true>;
+    cached[dev] = -1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pair_smem_bytes()) == cudaSuccess) {
+      cudaLaunchConfig_t cfg;
+      cudaLaunchAttribute attr[2];
+      pair_launch_config(cfg, attr, (n_sms / 2) * 2, 0, nullptr);
+      int clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) == cudaSuccess && clusters > 0)
+        cached[dev] = 2 * (clusters < n_sms / 2 ? clusters : n_sms / 2);
+      else
+        (void)cudaGetLastError();
+    } else {
+      (void)cudaGetLastError();
+    }
+  }
+  return cached[dev] > 0 ? cached[dev] : 0;
+}
+static cudaError_t launch_pair(const MapPack &maps, const UmmaParams &p, int grid, cudaStream_t st) {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[2];
+  pair_launch_config(cfg, attr, grid, p.pdl, st);
+  return cudaLaunchKernelEx(&cfg, gemm_umma_kernel<EPI_ATOMIC_ADD, 128, true, true>, maps, p);
+}
+
 template <int EPI>
 static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, bool panel, int grid, cudaStream_t st) {
   if (panel) {
@@ -984,7 +1146,7 @@ static cudaError_t launch_bn(const MapPack &maps, const UmmaParams &p, int bn, b
 // for the one before it.
 cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args, int n, unsigned int *bar,
                               unsigned int *claim, unsigned int *bar_b, const ChainSync *sync, unsigned int *tile_done,
-                              int td_stride, const ZeroList *zero, int pdl, cudaStream_t st) {
+                              int td_stride, const ZeroList *zero, int pdl, cudaStream_t st, int cta_pairs) {
   if (n < 1 || n > kMaxPhases || !claim) return cudaErrorInvalidValue;
   if (n > 1 && !bar) return cudaErrorInvalidValue;
   MapPack maps;
@@ -1000,6 +1162,13 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
   if (panel && epi == EPI_ARGMAX && !args[0].ss_out) return cudaErrorInvalidValue;
   if (args[0].R > 16 && !panel && n > 1 && sync) return cudaErrorInvalidValue;   // the caller plans `sync` for <= 16 rows
   const bool explicit_sync = sync && tile_done && !panel && !tile_mode && args[0].R <= 16;
+  // CTA pairs: 128-row blocks in panel mode, every matrix a whole number of 256-row tiles
+  bool pair = cta_pairs && panel && bn == 128 && !tile_mode;
+  for (int i = 0; i < n && pair; ++i)
+    for (int m = 0; m < plans[i]->d.g.n_mats; ++m) pair = pair && plans[i]->d.g.n_rows[m] % (2 * kTileM) == 0;
+  const int pgrid = pair ? pair_grid(plans[0]->n_sms) : 0;
+  pair = pair && pgrid >= 2;
+  if (pair) p.stages = kPairStages;
   long long max_chunks = 1;
   for (int i = 0; i < n; ++i) {
     const UmmaPlan *pl = plans[i];
@@ -1020,6 +1189,11 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.sig_bar = i + 1 < n ? i : -1;
     d.epi_bar = -1;
     d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0; d.dep_tiles = 0;
+    if (pair) {
+      d.tile_rows = 2 * kTileM;
+      d.n_tiles = 0;
+      for (int m = 0; m < d.g.n_mats; ++m) { d.tiles_m[m] = d.g.n_rows[m] / (2 * kTileM); d.n_tiles += d.tiles_m[m]; }
+    }
     d.cpt = (d.nkb + d.chunk_kb - 1) / d.chunk_kb;
     const long long chunks = (long long)nrb * d.n_tiles * d.cpt;
     if (chunks > 0x7fffffffLL) return cudaErrorInvalidValue;
@@ -1063,6 +1237,11 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
   // Staging warps own every fourth k-block and run ahead of each other; the parity waits on the ring
   // are only unambiguous while the ring is at least as deep as the number of staging warps.
   if (p.stages < 4 || p.stages > 8) return cudaErrorInvalidValue;
+  if (pair) {
+    // one chunk per pair at least; the grid barriers need every pair resident
+    const long long want = 2 * max_chunks;
+    return launch_pair(maps, p, (int)(want < pgrid ? want : pgrid), st);
+  }
   const long long resident = (long long)plans[0]->n_sms * cps;     // the grid barrier needs every CTA resident
   const int grid = (int)(resident < max_chunks ? resident : max_chunks);
   if (epi == EPI_ARGMAX) return launch_bn<EPI_ARGMAX>(maps, p, bn, panel, grid, st);
@@ -1070,8 +1249,8 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
 }
 
 cudaError_t launch_gemm_umma(const UmmaPlan *pl, const GemmArgs &a, unsigned int *claim, unsigned int *bar_b,
-                             const ZeroList *zero, int pdl, cudaStream_t st) {
-  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, nullptr, 0, zero, pdl, st);
+                             const ZeroList *zero, int pdl, cudaStream_t st, int cta_pairs) {
+  return launch_gemm_chain(&pl, &a, 1, nullptr, claim, bar_b, nullptr, nullptr, 0, zero, pdl, st, cta_pairs);
 }
 
 }  // namespace fc

@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(_HERE, "libfastcot.so")
 
 FC_F32, FC_BF16 = 0, 1
 FC_REFILL_PROMPT_CYCLE, FC_REFILL_PAD = 0, 1
-FC_FLAG_SIMT_GEMM, FC_FLAG_NO_PDL, FC_FLAG_NO_CHAIN, FC_FLAG_NO_FFN_SPLIT = 1, 4, 8, 16
+FC_FLAG_SIMT_GEMM, FC_FLAG_NO_PDL, FC_FLAG_NO_CHAIN, FC_FLAG_NO_FFN_SPLIT, FC_FLAG_NO_CTA_PAIRS = 1, 4, 8, 16, 32
 FC_OK = 0
 FC_NOALLOC_SCRATCH_BYTES = 8 << 20
 FC_CLASSES = ["embed", "qkv", "rope", "attn", "oproj", "gateup", "down", "head", "accept", "chain"]

@@ -189,18 +189,21 @@ def test_batch_ragged_prompts_independent_accepts():
 
 @pytest.mark.parametrize("B,c", [(3, 8), (4, 12), (6, 16), (10, 16), (1, 64), (3, 33)],
                          ids=["rows24", "rows48", "rows96", "rows160", "c64", "c33x3"])
-@pytest.mark.parametrize("shape", ["gqa64", "gqa32"])
+@pytest.mark.parametrize("shape", ["gqa64", "gqa32", "mha64", "mha64-single-cta-tiles"])
 def test_many_rows_prefill_and_steps(B, c, shape):
     """More than 16 rows per forward: the projections read their activations from the converted panel, for
     every accumulator width (32, 64, 128 rows) and for two blocks of rows; the prefill runs through the same path.
-    gqa32 has k extents that are not multiples of 256, so a group of conversion units spans two rows."""
+    gqa32 has k extents that are not multiples of 256, so a group of conversion units spans two rows.  In mha64 every
+    weight matrix of a layer is a whole number of 256-row tiles, so beyond 64 rows the projections run as pairs of
+    CTAs per tile (tcgen05 cta_group::2); the last shape runs the same model with that switched off."""
     kw = {"gqa64": dict(n_heads=4, n_kv_heads=2, head_dim=64, d_model=256, d_ffn=512),
-          "gqa32": dict(n_heads=8, n_kv_heads=2, head_dim=32, d_model=320, d_ffn=328)}[shape]
+          "gqa32": dict(n_heads=8, n_kv_heads=2, head_dim=32, d_model=320, d_ffn=328),
+          "mha64": dict(n_heads=4, n_kv_heads=4, head_dim=64, d_model=256, d_ffn=512)}[shape.split("-")[0]]
     cfg = wl.small_config(vocab=700, n_layers=2, prompt_len=200, c=c, gen_tokens=12, **kw)
     lens = [200 - 17 * b for b in range(B)]
     w = wl.make_weights(cfg)
     max_seq = 200 + 12 + c + 8
-    dec = engine.Decoder(cfg, w, B, c, max_seq)
+    dec = engine.Decoder(cfg, w, B, c, max_seq, flags=lib.FC_FLAG_NO_CTA_PAIRS if shape.endswith("tiles") else 0)
     ids, _ = wl.make_prompts(cfg, batch=B, lens=lens)
     dec.fc_prefill(ids.numpy(), lens, c)
     logits = dec.fc_debug_logits(True)
