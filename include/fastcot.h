@@ -221,7 +221,8 @@ int fc_op_window_attention(const void *q, const void *kcache, const void *vcache
  * the call; sumsq: fp32 [batch*c], cleared by the call; kcache/vcache: bf16 [batch][n_kv_heads][max_seq][head_dim],
  * in/out, 16-byte aligned (cached K/V tiles are fetched by TMA); out: fp32 [batch*c, n_heads*head_dim].  c <= 128.
  * n_splits: 0 = the grid fc_jacobi_step would choose, 1..8 forces that many CTAs (one thread-block cluster) per
- * (sequence, kv head, group of query tiles), each over a run of consecutive 64-key tiles.  scratch: device, 256-byte
+ * (sequence, kv head, group of query tiles), each over a run of consecutive 64-key tiles.  q_tiles: 0 = the step's
+ * choice, 1, 2 or 4 forces that many 16-row query tiles per CTA.  scratch: device, 256-byte
  * aligned, >= ..._scratch_bytes(...) (rotary table and an error word).  Returns FC_ERR_DEVICE_TIMEOUT when a bounded
  * wait inside the kernel gave up. */
 size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int32_t c, int32_t n_heads, int32_t n_kv_heads,
@@ -229,8 +230,8 @@ size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int32_t c, int3
 int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float rms_eps, int32_t d_norm, float rope_theta,
                                  void *kcache, void *vcache, const int32_t *kv_len, float *out, int32_t batch,
                                  int32_t c, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, int32_t max_seq,
-                                 int32_t max_len, int32_t n_splits, void *scratch, size_t scratch_bytes,
-                                 void *cuda_stream);
+                                 int32_t max_len, int32_t n_splits, int32_t q_tiles, void *scratch,
+                                 size_t scratch_bytes, void *cuda_stream);
 
 /* The same window attention for callers that may not allocate device memory (the paper has no
  * counterpart; this exists for hosts whose device memory is owned by someone else, e.g. a serving

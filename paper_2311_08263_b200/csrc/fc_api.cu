@@ -474,7 +474,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       fa.k_plane0 = (l * 2) * s.max_batch * s.n_kv_heads; fa.v_plane0 = (l * 2 + 1) * s.max_batch * s.n_kv_heads;
       fa.kv_len = ctx->b.kv_len; fa.b0 = b0; fa.nb = nb; fa.c = rows; fa.hq = s.n_heads; fa.hkv = s.n_kv_heads;
       fa.seq_map = seq_map;
-      fused_attn_plan(max_len_host, rows, s.n_heads, s.n_kv_heads, nb, ctx->n_sms, fa.nsplit, fa.qt);
+      fused_attn_plan(max_len_host, rows, s.n_heads, s.n_kv_heads, nb, s.head_dim, ctx->n_sms, fa.nsplit, fa.qt);
       fa.err = ctx->b.err;
       fa.out = ctx->b.attn; fa.pdl = ctx->pdl && !ctx->prof;
       fa.z.p[0] = ctx->b.gu; fa.z.n[0] = Rz * 2 * s.d_ffn;
@@ -1133,9 +1133,10 @@ extern "C" size_t fc_op_fused_window_attention_scratch_bytes(int32_t batch, int3
 extern "C" int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float rms_eps, int32_t d_norm, float rope_theta,
                                             void *kcache, void *vcache, const int32_t *kv_len, float *out, int32_t batch,
                                             int32_t c, int32_t n_heads, int32_t n_kv_heads, int32_t head_dim,
-                                            int32_t max_seq, int32_t max_len, int32_t n_splits, void *scratch,
-                                            size_t scratch_bytes, void *cuda_stream) {
+                                            int32_t max_seq, int32_t max_len, int32_t n_splits, int32_t q_tiles,
+                                            void *scratch, size_t scratch_bytes, void *cuda_stream) {
   if (!qkv_acc || !sumsq || !kcache || !vcache || !kv_len || !out || !scratch || d_norm < 1 || n_splits < 0 || n_splits > 8) return FC_ERR_ARG;
+  if (q_tiles != 0 && q_tiles != 1 && q_tiles != 2 && q_tiles != 4) return FC_ERR_ARG;
   if (!fused_shape_ok(batch, c, n_heads, n_kv_heads, head_dim, max_seq, max_len)) return FC_ERR_ARG;
   if (max_len + c > max_seq) return FC_ERR_CAPACITY;
   if ((uintptr_t)scratch % kAlign || ((uintptr_t)kcache | (uintptr_t)vcache) % 16) return FC_ERR_ARG;
@@ -1172,8 +1173,9 @@ extern "C" int fc_op_fused_window_attention(float *qkv_acc, float *sumsq, float 
   fa.stride_h = (long long)max_seq * head_dim; fa.stride_b = (long long)n_kv_heads * fa.stride_h;
   fa.k_plane0 = 0; fa.v_plane0 = 0;
   fa.kv_len = kv_len; fa.b0 = 0; fa.nb = batch; fa.c = c; fa.hq = n_heads; fa.hkv = n_kv_heads;
-  fused_attn_plan(max_len, c, n_heads, n_kv_heads, batch, sms, fa.nsplit, fa.qt);
+  fused_attn_plan(max_len, c, n_heads, n_kv_heads, batch, head_dim, sms, fa.nsplit, fa.qt);
   if (n_splits > 0) fa.nsplit = n_splits;
+  if (q_tiles > 0) fa.qt = q_tiles;
   fa.err = (unsigned int *)(base + off[1]);
   fa.out = out; fa.pdl = 0;
   if (launch_attn_fused(kmap, vmap, fa, head_dim, st) != cudaSuccess) return FC_ERR_CUDA;

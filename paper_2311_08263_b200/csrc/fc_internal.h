@@ -158,7 +158,7 @@ cudaError_t launch_attn_fused(const KvTensorMap &kmap, const KvTensorMap &vmap, 
 // 3-d tensor map (head_dim, max_seq, planes) over bf16 K or V planes laid out [plane][max_seq][head_dim] from `base`.
 cudaError_t make_kv_tensor_map(KvTensorMap *out, const void *base, int hd, int max_seq, long long planes);
 // Grid of the fused attention kernel: splits per (sequence, kv head, query-tile group) and query tiles per CTA.
-void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int &nsplit, int &qt);
+void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int hd, int n_sms, int &nsplit, int &qt);
 int attn_fused_max_rows();   // most window rows per sequence the fused kernel takes in one launch
 cudaError_t launch_accept(const AcceptArgs &a, cudaStream_t st);
 // dst[i * c + j] = window[seq_map[i] * c + j]: the token rows of a forward over the sequences seq_map[0 .. nb-1]

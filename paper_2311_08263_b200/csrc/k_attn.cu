@@ -640,10 +640,20 @@ cudaError_t make_kv_tensor_map(KvTensorMap *out, const void *base, int hd, int m
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int n_sms, int &nsplit, int &qt) {
+void fused_attn_plan(int max_len, int c, int hq, int hkv, int nb, int hd, int n_sms, int &nsplit, int &qt) {
   const int nqt = ((hq / hkv) * c + 15) / 16;
+  // Query tiles per CTA.  One is the rule: more CTAs, each small enough for two to share an SM, hide each other's
+  // waits best (measured: 13B, batch 8, c = 32: 5.2 -> 4.8 ms of attention per step against two tiles per CTA).  Only
+  // when that makes more than six waves of CTAs do several query tiles share a CTA (and with it every key tile and
+  // its barriers) - as long as two such CTAs still fit on an SM, which is what decides there (7B, K/V 8192, batch 16:
+  // c = 32, where they fit, 40.7 ms with two tiles per CTA against 43.1; c = 64, where they do not, 90.1 against 80.0).
+  auto two_fit = [&](int q) {
+    const size_t per_sm = 228 * 1024, reserve = 1024 + 256;
+    const size_t need = hd == 128 ? attn_smem_bytes<128>(c, q, 2) : attn_smem_bytes<64>(c, q, 2);
+    return 2 * (need + reserve) <= per_sm;
+  };
   qt = 1;
-  while (qt < 4 && qt < nqt && (long long)nb * hkv * ((nqt + qt - 1) / qt) > 2ll * n_sms) qt *= 2;
+  while (qt < 4 && qt < nqt && (long long)nb * hkv * ((nqt + qt - 1) / qt) > 6ll * n_sms && two_fit(qt * 2)) qt *= 2;
   const long long units = (long long)nb * hkv * ((nqt + qt - 1) / qt);
   const int n_ct = (max_len + kTK - 1) / kTK;
   // Short caches: one CTA per SM, so that the projection kernel's CTAs come in beside them while the attention runs.

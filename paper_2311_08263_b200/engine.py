@@ -248,7 +248,7 @@ def fc_op_window_attention(q: torch.Tensor, kcache: torch.Tensor, vcache: torch.
 
 def fc_op_fused_window_attention(qkv_acc: torch.Tensor, sumsq: torch.Tensor, rms_eps: float, d_norm: int,
                                  rope_theta: float, kcache: torch.Tensor, vcache: torch.Tensor, kv_len: torch.Tensor,
-                                 c: int, n_heads: int, max_len: int, n_splits: int = 0) -> torch.Tensor:
+                                 c: int, n_heads: int, max_len: int, n_splits: int = 0, q_tiles: int = 0) -> torch.Tensor:
     """The fused attention kernel of the bf16 step as one operation.  qkv_acc fp32 [B*c, (hq + 2 hkv) * hd] and sumsq
     fp32 [B*c] are consumed (cleared); kcache/vcache bf16 [B, hkv, max_seq, hd] receive the window's rows.
     Returns fp32 [B*c, hq*hd]."""
@@ -261,7 +261,7 @@ def fc_op_fused_window_attention(qkv_acc: torch.Tensor, sumsq: torch.Tensor, rms
     out = torch.empty(B * c, n_heads * hd, dtype=torch.float32, device=qkv_acc.device)
     rc = lib.fc_op_fused_window_attention(qkv_acc.data_ptr(), sumsq.data_ptr(), rms_eps, d_norm, rope_theta,
                                           kcache.data_ptr(), vcache.data_ptr(), kv_len.data_ptr(), out.data_ptr(),
-                                          B, c, n_heads, hkv, hd, max_seq, max_len, n_splits,
+                                          B, c, n_heads, hkv, hd, max_seq, max_len, n_splits, q_tiles,
                                           scratch.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
     if rc != _l.FC_OK:
         raise FcError(rc, "fc_op_fused_window_attention")

@@ -98,7 +98,7 @@ def load() -> C.CDLL:
     lib.fc_op_window_attention_noalloc.argtypes = [vp] * 5 + [i32] * 8 + [vp]
     lib.fc_op_fused_window_attention_scratch_bytes.restype = C.c_size_t
     lib.fc_op_fused_window_attention_scratch_bytes.argtypes = [i32] * 7
-    lib.fc_op_fused_window_attention.argtypes = [vp, vp, C.c_float, i32, C.c_float, vp, vp, vp, vp] + [i32] * 8 + \
+    lib.fc_op_fused_window_attention.argtypes = [vp, vp, C.c_float, i32, C.c_float, vp, vp, vp, vp] + [i32] * 9 + \
                                                 [vp, C.c_size_t, vp]
     _lib = lib
     return lib

@@ -55,27 +55,34 @@ def _case(hq, hkv, hd, c, lens, seed):
 
 
 CASES = [
-    # hq, hkv, hd, c, lens, splits per (sequence, kv head, query-tile group) (0 = the step's choice)
-    (4, 4, 128, 16, [127, 128, 129, 0, 1], 0),        # MHA; lengths around a tile edge, empty cache, one key
-    (4, 4, 128, 16, [63, 64, 65, 191, 192], 1),       # one CTA per head: every tile through the ring, ragged last tile
-    (8, 2, 64, 5, [260, 1, 2047], 0),                 # GQA, odd window, clusters of 8 splits, sequences with empty splits
-    (4, 4, 128, 1, [77, 130, 2047], 0),               # c = 1: plain autoregressive attention
-    (8, 2, 64, 33, [300, 6000], 0),                   # 94 tiles per head: long runs per CTA, 9 query tiles per kv head
-    (4, 2, 128, 64, [513, 40], 0),                    # c = 64: a full window tile, 8 query tiles per kv head
-    (4, 2, 128, 100, [513, 40], 2),                   # c = 100: two window tiles (the second ragged), as in a prefill block
-    (4, 4, 64, 16, [6000, 2047, 129], 4),             # forced: 4 splits, running softmax statistics over ~24 tiles each
-    (8, 2, 128, 16, [2047, 1], 3),                    # forced odd cluster size with grouped queries (2 query tiles)
-    (32, 32, 128, 16, [1000], 0),                     # the benchmark's attention shape: 32 heads, 4 splits of 4 tiles
-    # more (sequence, kv head, query tile) units than CTA slots: four query tiles per CTA, two CTAs per SM on a
-    # two-stage ring
-    (8, 8, 64, 64, [70, 1, 130, 257, 64] * 8, 0),
-    (8, 8, 128, 64, [70, 1, 130, 257, 64] * 8, 0),
-    (16, 8, 128, 32, [200, 5, 129] * 6, 0),           # grouped queries, four tiles per kv head, two per CTA
+    # hq, hkv, hd, c, lens, splits per (sequence, kv head, query-tile group), query tiles per CTA (0 = the step's choice)
+    (4, 4, 128, 16, [127, 128, 129, 0, 1], 0, 0),     # MHA; lengths around a tile edge, empty cache, one key
+    (4, 4, 128, 16, [63, 64, 65, 191, 192], 1, 0),    # one CTA per head: every tile through the ring, ragged last tile
+    (8, 2, 64, 5, [260, 1, 2047], 0, 0),              # GQA, odd window, clusters of 8 splits, sequences with empty splits
+    (4, 4, 128, 1, [77, 130, 2047], 0, 0),            # c = 1: plain autoregressive attention
+    (8, 2, 64, 33, [300, 6000], 0, 0),                # 94 tiles per head: long runs per CTA, 17 query tiles per kv head
+    (4, 2, 128, 64, [513, 40], 0, 0),                 # c = 64: a full window tile, 8 query tiles per kv head
+    (4, 2, 128, 64, [513, 40], 0, 2),                 # the same with two and with four query tiles per CTA
+    (4, 2, 128, 64, [513, 40], 2, 4),
+    (4, 2, 128, 100, [513, 40], 2, 0),                # c = 100: two window tiles (the second ragged), as in a prefill block
+    (4, 2, 128, 100, [513, 40], 1, 2),
+    (4, 4, 64, 16, [6000, 2047, 129], 4, 0),          # forced: 4 splits, running softmax statistics over ~24 tiles each
+    (8, 2, 128, 16, [2047, 1], 3, 0),                 # forced odd cluster size with grouped queries (2 query tiles)
+    (8, 2, 128, 16, [2047, 1], 3, 2),
+    (32, 32, 128, 16, [1000], 0, 0),                  # the benchmark's attention shape: 32 heads, 4 splits of 4 tiles
+    # more (sequence, kv head, query tile) units than CTA slots: two CTAs per SM on a two-stage ring, with one, two and
+    # four query tiles per CTA
+    (8, 8, 64, 64, [70, 1, 130, 257, 64] * 8, 0, 0),
+    (8, 8, 64, 64, [70, 1, 130, 257, 64] * 8, 0, 4),
+    (8, 8, 128, 64, [70, 1, 130, 257, 64] * 8, 0, 0),
+    (8, 8, 128, 64, [70, 1, 130, 257, 64] * 8, 0, 4),
+    (16, 8, 128, 32, [200, 5, 129] * 6, 0, 2),        # grouped queries, four tiles per kv head, two per CTA
+    (16, 8, 128, 32, [200, 5, 129] * 24, 0, 0),       # enough units (more than six waves of CTAs) for the step's own choice of two
 ]
 
 
-@pytest.mark.parametrize("hq,hkv,hd,c,lens,splits", CASES)
-def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, splits):
+@pytest.mark.parametrize("hq,hkv,hd,c,lens,splits,q_tiles", CASES)
+def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, splits, q_tiles):
     cfg, acc, ss, kc, vc, max_seq, want_attn, want_k, want_v = _case(hq, hkv, hd, c, lens, seed=40 + c)
     B = len(lens)
     kcd = kc.to(torch.bfloat16).cuda().contiguous()
@@ -83,7 +90,7 @@ def test_fused_window_attention_vs_oracle_trace(hq, hkv, hd, c, lens, splits):
     assert torch.equal(kcd.float().cpu(), kc)                   # the oracle's cached rows are bf16 values
     accd, ssd = acc.cuda().contiguous(), ss.cuda().contiguous()
     out = engine.fc_op_fused_window_attention(accd, ssd, cfg.rms_eps, cfg.d_model, cfg.rope_theta, kcd, vcd,
-                                              torch.tensor(lens, dtype=torch.int32).cuda(), c, hq, max(lens), splits)
+                                              torch.tensor(lens, dtype=torch.int32).cuda(), c, hq, max(lens), splits, q_tiles)
     out = out.cpu().numpy().reshape(B, c, hq * hd)
     assert float(accd.abs().max()) == 0.0 and float(ssd.abs().max()) == 0.0      # consumed
     for b, L in enumerate(lens):
@@ -114,7 +121,9 @@ def test_fused_window_attention_rejects_bad_arguments():
     n = l.fc_op_fused_window_attention_scratch_bytes(1, 8, 4, 4, 64, 64, 10)
     assert n > 0
     assert l.fc_op_fused_window_attention(None, t.data_ptr(), 1e-5, 8, 1e4, t.data_ptr(), t.data_ptr(), t.data_ptr(),
-                                          t.data_ptr(), 1, 8, 4, 4, 64, 64, 10, 0, t.data_ptr(), n, st) == lib.FC_ERR_ARG
+                                          t.data_ptr(), 1, 8, 4, 4, 64, 64, 10, 0, 0, t.data_ptr(), n, st) == lib.FC_ERR_ARG
+    assert l.fc_op_fused_window_attention(t.data_ptr(), t.data_ptr(), 1e-5, 8, 1e4, t.data_ptr(), t.data_ptr(), t.data_ptr(),
+                                          t.data_ptr(), 1, 8, 4, 4, 64, 64, 10, 0, 3, t.data_ptr(), n, st) == lib.FC_ERR_ARG
     assert l.fc_op_fused_window_attention(t.data_ptr(), t.data_ptr(), 1e-5, 8, 1e4, t.data_ptr(), t.data_ptr(),
-                                          t.data_ptr(), t.data_ptr(), 1, 8, 4, 4, 64, 64, 60, 0, t.data_ptr(), n,
+                                          t.data_ptr(), t.data_ptr(), 1, 8, 4, 4, 64, 64, 60, 0, 0, t.data_ptr(), n,
                                           st) == lib.FC_ERR_CAPACITY
