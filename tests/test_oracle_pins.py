@@ -423,3 +423,80 @@ def test_answer_trigger_empty_with_c1_is_plain_continuation_and_eos_cut():
     first = 6 + int(np.where(ar[6:] == eos)[0][0])
     got = o.finish_with_trigger([], 20, eos_id=eos)
     assert got.tolist() == ar[6:first + 1].tolist()
+
+
+# ---------------------------------------------------------------- layer-0 special cases with closed forms
+def _f32_small(**kw):
+    cfg = wl.small_config(dtype="f32", n_layers=1, vocab=300, **kw)
+    return cfg, wl.make_weights(cfg)
+
+
+def _normed_rows(cfg, w, tokens):
+    """RMSNorm(embedding rows) * gain of layer 0, in fp64 (Llama's definition: x / sqrt(mean x^2 + eps) * g)."""
+    x = w["tok_emb"].double()[torch.as_tensor(np.asarray(tokens)).long()]
+    return x / torch.sqrt((x * x).mean(1, keepdim=True) + cfg.rms_eps) * w["g_attn"][0].double()
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (4, 2), (4, 1)])
+def test_single_key_attention_returns_its_value_row(hq, hkv):
+    """Empty cache, one window row: the softmax over one key is 1, so every query head's output is the value row of its
+    kv head, bit for bit (head h reads kv head h // (hq / hkv))."""
+    cfg, w = _f32_small(n_heads=hq, n_kv_heads=hkv, head_dim=32, d_model=hq * 32)
+    o = oracle.Oracle(cfg, w, 8)
+    _, _, tr = o.forward([5], want_logits=True, trace=True)
+    _, v = o.get_kv(0, 1)
+    hd, group = cfg.head_dim, hq // hkv
+    for h in range(hq):
+        kvh = h // group
+        assert np.array_equal(tr["attn"][0, h * hd:(h + 1) * hd], v[0, kvh * hd:(kvh + 1) * hd])
+    o.close()
+
+
+def test_rope_is_the_identity_at_position_zero_and_a_rotation_of_half_split_pairs_elsewhere():
+    """Position 0: q and k are the plain projections of the normalised row.  Position p: element i is paired with
+    i + head_dim / 2 (not with i + 1), the pair keeps its norm and turns by p * theta^(-2i / head_dim)."""
+    cfg, w = _f32_small(n_heads=2, n_kv_heads=2, head_dim=32, d_model=64)
+    toks = [7, 11, 13, 17, 19]
+    o = oracle.Oracle(cfg, w, 16)
+    _, _, tr = o.forward(toks, want_logits=True, trace=True)
+    k, _ = o.get_kv(0, len(toks))
+    xn = _normed_rows(cfg, w, toks)
+    q_plain = (xn @ w["wq"][0].double().T).numpy()
+    k_plain = (xn @ w["wk"][0].double().T).numpy()
+    assert np.abs(tr["q"][0] - q_plain[0]).max() < 2e-6 and np.abs(k[0] - k_plain[0]).max() < 2e-6
+    hd, half = cfg.head_dim, cfg.head_dim // 2
+    for got, plain in ((tr["q"], q_plain), (k, k_plain)):
+        for p in range(1, len(toks)):
+            for h in range(cfg.n_heads):
+                a, b = plain[p, h * hd:h * hd + half], plain[p, h * hd + half:(h + 1) * hd]
+                ga, gb = got[p, h * hd:h * hd + half].astype(np.float64), got[p, h * hd + half:(h + 1) * hd].astype(np.float64)
+                assert np.abs((ga * ga + gb * gb) - (a * a + b * b)).max() < 1e-5          # norm of every pair
+                ang = p * cfg.rope_theta ** (-2.0 * np.arange(half) / hd)
+                turned = np.arctan2(gb, ga) - np.arctan2(b, a)
+                d = (turned - ang + np.pi) % (2 * np.pi) - np.pi
+                big = (a * a + b * b) > 1e-4                                               # the angle of a tiny pair is noise
+                assert np.abs(d[big]).max() < 1e-4
+    o.close()
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (4, 2)])
+def test_zero_query_projection_gives_the_causal_mean_of_the_value_rows(hq, hkv):
+    """W_q = 0: all scores are equal, so window row j attends uniformly to the L cached rows and window rows 0..j - the
+    output is their mean value row.  Fails on an off-by-one in the causal mask, a missing normalisation or a wrong
+    query-head -> kv-head map."""
+    cfg, w = _f32_small(n_heads=hq, n_kv_heads=hkv, head_dim=32, d_model=hq * 32)
+    w["wq"][0] = torch.zeros_like(w["wq"][0])
+    L, c = 6, 5
+    ids = wl.hash_uniform_int(cfg.seed, 3, L + 1, cfg.vocab).numpy()
+    o = oracle.Oracle(cfg, w, L + c + 4)
+    o.prefill(ids, c)                                      # caches ids[0 .. L-1]
+    win = wl.hash_uniform_int(cfg.seed + 1, 4, c, cfg.vocab).numpy()
+    _, _, tr = o.forward(win, want_logits=True, trace=True)
+    _, v = o.get_kv(0, L + c)
+    hd, group = cfg.head_dim, hq // hkv
+    for j in range(c):
+        want = v[:L + j + 1].astype(np.float64).mean(0)
+        for h in range(hq):
+            kvh = h // group
+            assert np.abs(tr["attn"][j, h * hd:(h + 1) * hd] - want[kvh * hd:(kvh + 1) * hd]).max() < 2e-6
+    o.close()
