@@ -496,6 +496,40 @@ def test_bf16_step_run_to_run_spread_is_bounded(flags):
     assert spread < 3e-4, spread
 
 
+@pytest.mark.parametrize("flags", [0, lib.FC_FLAG_NO_CTA_PAIRS], ids=["cta-pairs", "single-cta-tiles"])
+def test_bf16_many_row_step_spread_and_agreement_of_the_two_tilings(flags):
+    """160 rows per forward (two blocks of 128 through the activation panel; pairs of CTAs per 256-row weight tile or
+    one CTA per 128-row tile): repeated runs of the same step stay within the same small spread, and the logits agree
+    with the oracle's for every sequence."""
+    cfg = wl.small_config(vocab=1200, n_layers=4, n_heads=8, n_kv_heads=8, head_dim=64, d_model=512, d_ffn=1536,
+                          prompt_len=90, c=16, gen_tokens=4)
+    B = 10
+    w = wl.make_weights(cfg, device="cuda")
+    lens = [90 - 7 * b for b in range(B)]
+    ids, _ = wl.make_prompts(cfg, batch=B, lens=lens)
+    dec = engine.Decoder(cfg, w, B, cfg.c, 120, flags=flags)
+    logits = dec.fc_debug_logits(True)
+    dec.fc_prefill(ids.numpy(), lens, cfg.c)
+    ref = None
+    spread = 0.0
+    for _ in range(15):
+        dec.fc_bench_steps(1, commit=False)
+        torch.cuda.synchronize()
+        lg = logits[:B * cfg.c].clone()
+        if ref is None:
+            ref = lg
+        spread = max(spread, float((lg - ref).abs().max()))
+    assert spread < 3e-4, spread
+    got = ref.cpu().numpy().reshape(B, cfg.c, cfg.vocab)
+    wc = wl.make_weights(cfg)
+    for b in (0, 4, 9):
+        o = oracle.Oracle(cfg, wc, 120)
+        o.prefill(ids[b, :lens[b]].numpy(), cfg.c)
+        _, _, _, lg = o.jacobi_step(want_logits=True)
+        assert np.abs(got[b] - lg).max() < LOGIT_TOL
+        o.close()
+
+
 @pytest.mark.parametrize("kind", ["fp32", "bf16"])
 def test_finished_sequences_are_skipped_and_the_others_unaffected(kind):
     """A batch in which sequences finish at different times (one on an EOS early in its stream, the others at
