@@ -461,6 +461,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
   const long long stride_h = (long long)s.max_seq * s.head_dim;
   const long long stride_b = (long long)s.n_kv_heads * stride_h;
   const bool chained = ctx->chain;
+  const bool o_panel = chained && ctx->fused_attn && R > 16 && ctx->d.pan_rows >= R;
   for (int l = 0; l < s.n_layers; ++l) {
     if (!chained || l == 0)
       FC_CK(run_gemm(ctx, ctx->use_umma ? ctx->plan_qkv[l] : nullptr, args_qkv(ctx, l), R, PRO_GAIN, EPI_ATOMIC_ADD, FC_CLS_QKV, claim_word(ctx, l, GEMM_QKV)));
@@ -477,6 +478,9 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       fused_attn_plan(max_len_host, rows, s.n_heads, s.n_kv_heads, nb, s.head_dim, ctx->n_sms, fa.nsplit, fa.qt);
       fa.err = ctx->b.err;
       fa.out = ctx->b.attn; fa.pdl = ctx->pdl && !ctx->prof;
+      // more than 16 rows: the chained launch streams its activations from the bf16 panel; the attention kernel writes
+      // its result there directly, which saves the output projection's conversion pass and two grid-wide waits
+      if (o_panel) { fa.out_pan = ctx->b.pan; fa.pan_rows = d.pan_rows; }
       fa.z.p[0] = ctx->b.gu; fa.z.n[0] = Rz * 2 * s.d_ffn;
       fa.z.p[1] = ctx->b.ss_ffn; fa.z.n[1] = Rz;
       ++ctx->launches;
@@ -519,7 +523,7 @@ static int forward(fc_ctx *ctx, int b0, int nb, int rows, const int32_t *tokens,
       ChainSync sy[kChainMax];
       int n = 0;
       const bool split = ctx->ffn_split && R <= 16;
-      plans[n] = ctx->plan_o[l]; ga[n] = args_o(ctx, l); sy[n++] = ChainSync{-1, -1, 0, -1, -1};
+      plans[n] = ctx->plan_o[l]; ga[n] = args_o(ctx, l); ga[n].pan_ready = o_panel ? 1 : 0; sy[n++] = ChainSync{-1, -1, 0, -1, -1};
       if (split) {
         plans[n] = ctx->plan_gu_half[0][l]; ga[n] = args_gu_half(ctx, l, 0); sy[n++] = ChainSync{-1, 0, -1, 0, -1};
         plans[n] = ctx->plan_gu_half[1][l]; ga[n] = args_gu_half(ctx, l, 1); sy[n++] = ChainSync{-1, 1, -1, 0, -1};

@@ -51,6 +51,7 @@ struct GemmArgs {
   // and streams by TMA; with the argmax epilogue ss_out then holds the row sums of squares the epilogue reads
   void *pan;
   int pan_rows;
+  int pan_ready;                  // the panel already holds pro(x), written by the kernel before this launch: no conversion
 };
 
 struct ZeroList {       // buffers a kernel clears on the side (fp32 words)
@@ -111,6 +112,10 @@ struct FusedAttnArgs {   // bf16: rotary embedding + K/V write + window attentio
   int pdl;                // launched as a programmatic dependent of the previous kernel
   unsigned int *err;      // device error word, raised when a bounded wait gives up
   float *out;             // [R, hq*hd] fp32
+  // instead of `out`: the result as the bf16 pair high + low in the activation panel [2][pan_rows][hq*hd] that the output
+  // projection streams by TMA (more than 16 rows per forward), which then needs no conversion pass of its own
+  void *out_pan;
+  int pan_rows;
   ZeroList z;
 };
 

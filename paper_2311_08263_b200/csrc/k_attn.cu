@@ -608,8 +608,15 @@ attn_tma_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant_
     const float inv = den > 0.f ? 1.0f / den : 0.f;
     const int g = div_c(qrow), j = qrow - g * c;
     const int r = bl * c + j, h = kvh * group + g;
-    *reinterpret_cast<float4 *>(a.out + (long long)r * qd + h * HD + c4 * 4) =
-        make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    const float o0 = acc.x * inv, o1 = acc.y * inv, o2 = acc.z * inv, o3 = acc.w * inv;
+    if (a.out_pan) {
+      __nv_bfloat16 *ph = (__nv_bfloat16 *)a.out_pan + (long long)r * qd + h * HD + c4 * 4;
+      *reinterpret_cast<uint2 *>(ph) = make_uint2(pack_bf16(o0, o1), pack_bf16(o2, o3));
+      *reinterpret_cast<uint2 *>(ph + (long long)a.pan_rows * qd) =
+          make_uint2(pack_bf16(o0 - bf16_round(o0), o1 - bf16_round(o1)), pack_bf16(o2 - bf16_round(o2), o3 - bf16_round(o3)));
+    } else {
+      *reinterpret_cast<float4 *>(a.out + (long long)r * qd + h * HD + c4 * 4) = make_float4(o0, o1, o2, o3);
+    }
   }
   if (ns > 1) cluster_sync_all();                             // the other splits may still be reading this CTA's memory
 }

@@ -58,6 +58,7 @@ struct PhaseDesc {
   const unsigned int *dep_done;
   unsigned int dep_need;
   int dep_tiles;                      // number of counters behind dep_done
+  int pre_panel;                      // panel mode: the panel was filled by the kernel before this launch
 };
 
 struct MapPack {
@@ -675,12 +676,16 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
         if (!ok) break;
       }
       if constexpr (PANEL) {
-        // ---- (1) this warp's share of the panel conversion
-        convert_share(P, pi, sw);
-        // ---- (2) panel-ready barrier: the converting warps of every CTA have stored their share
-        if (sw == 0) {
-          ok = grid_bar_wait(p.bar_b + pi, gridDim.x, lane, abort_flag);
-          asm volatile("fence.proxy.async;" ::: "memory");
+        if (!P.pre_panel) {
+          // ---- (1) this warp's share of the panel conversion
+          convert_share(P, pi, sw);
+          // ---- (2) panel-ready barrier: the converting warps of every CTA have stored their share
+          if (sw == 0) {
+            ok = grid_bar_wait(p.bar_b + pi, gridDim.x, lane, abort_flag);
+            asm volatile("fence.proxy.async;" ::: "memory");
+          }
+        } else if (sw == 0) {
+          asm volatile("fence.proxy.async;" ::: "memory");    // the previous kernel's stores, complete since griddepcontrol.wait
         }
         // ---- (3) warp 0 streams the activation tiles of every claimed k-block into the ring; the other three
         // staging warps only follow the queue
@@ -863,7 +868,7 @@ gemm_umma_kernel(const __grid_constant__ MapPack maps, const __grid_constant__ U
       if constexpr (PANEL && BN == 128) {
         // the previous phase's sums are complete (a staging warp polls the grid barrier and opens go_bar): this warp's
         // share of the panel conversion
-        if (conv_warps(P) == 8) {
+        if (!P.pre_panel && conv_warps(P) == 8) {
           if (P.wait_bar >= 0 && !mbar_wait_warp(smem_u32(&go_bar[pi]), 0u, abort_flag)) { ok = false; break; }
           convert_share(P, pi, 4 + q);
         }
@@ -1170,6 +1175,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
   bool panel = bar_b != nullptr && args[0].R > 16;
   for (int i = 0; i < n; ++i) panel = panel && plans[i]->has_xmap && args[0].R <= plans[i]->d.g.pan_rows;
   if (panel && epi == EPI_ARGMAX && !args[0].ss_out) return cudaErrorInvalidValue;
+  if (args[0].pan_ready && !panel) return cudaErrorInvalidValue;     // the caller wrote the panel instead of the fp32 input
   if (args[0].R > 16 && !panel && n > 1 && sync) return cudaErrorInvalidValue;   // the caller plans `sync` for <= 16 rows
   const bool explicit_sync = sync && tile_done && !panel && !tile_mode && args[0].R <= 16;
   // CTA pairs: 128-row blocks in panel mode, every matrix a whole number of 256-row tiles
@@ -1199,6 +1205,7 @@ cudaError_t launch_gemm_chain(const UmmaPlan *const *plans, const GemmArgs *args
     d.sig_bar = i + 1 < n ? i : -1;
     d.epi_bar = -1;
     d.tile_done = nullptr; d.dep_done = nullptr; d.dep_need = 0; d.dep_tiles = 0;
+    d.pre_panel = panel && i == 0 && a.pan_ready;
     if (pair) {
       d.tile_rows = 2 * kTileM;
       d.n_tiles = 0;
